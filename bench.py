@@ -1,0 +1,302 @@
+"""Benchmark of the FP8 SLA forward: one step = quantise Q, K, V + block plan + forward on one synthetic batch.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload vggt8] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `value` is dense-equivalent TFLOP/s (4*B*H*N^2*D per step over the step time)
+with the bf16 sources resident in HBM; `e2e` is the same metric with pinned-host sources copied in and the fp32
+output copied out inside the timed region.  `--impl reference` times the CPU oracle on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2605_11354_b200 import dist as pdist  # noqa: E402
+from paper_2605_11354_b200 import workloads as wk  # noqa: E402
+
+METRIC = "sla_fwd_dense_equiv_tflops"
+UNIT = "TFLOP/s"
+L2_FLUSH_BYTES = 512 << 20
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
+FP8_OVER_BF16 = 2.0  # nominal dense ratio (4.5 vs 2.25 PFLOP/s)
+# DRAM bytes (read + write) of one attention-kernel launch from the ncu capture summarised under profiles/;
+# None until a capture of the current kernel exists.
+ATTENTION_DRAM_BYTES_PER_LAUNCH = None
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            return json.load(fh), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            return
+        self.thread = threading.Thread(target=self._pump, daemon=True)
+        self.thread.start()
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) == 7:
+                self.rows.append(parts)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        if self.thread is not None:
+            self.thread.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, r[3:]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def executed_critical_flops(wl, k_crit):
+    return 4.0 * wl.batch * wl.heads * wl.n_blocks * k_crit * wl.block * wl.block * wl.head_dim
+
+
+# ------------------------------------------------------------------------------------------------ CPU oracle timing
+def time_oracle(wl, inputs, n_heads, budget_blocks):
+    """One bounded sample of the step on the host cores: quantiser and plan for the first `n_heads` heads of every
+    batch entry, the forward on a seeded sample of their query blocks; both parts are extrapolated to the whole
+    workload (heads are independent problems of equal size).  Returns (seconds per whole step, description)."""
+    from oracle import sla_oracle as orc
+    n_heads = min(n_heads, wl.heads)
+    sub = {n: np.ascontiguousarray(inputs[n][:, :n_heads]) for n in ("q", "k", "v")}
+    proj = inputs["proj"][:n_heads]
+    t0 = time.perf_counter()
+    r = orc.sla_forward_from_source(sub["q"], sub["k"], sub["v"], proj, wl.block, wl.crit, wl.neg, query_blocks=[])
+    t_front = time.perf_counter() - t0
+    total_sub = wl.batch * n_heads * wl.n_blocks
+    total = wl.batch * wl.heads * wl.n_blocks
+    g = np.random.default_rng(wl.cfg_id)
+    n = min(budget_blocks, total_sub)
+    flat = g.choice(total_sub, size=n, replace=False)
+    qb = [(int(f // (n_heads * wl.n_blocks)), int((f // wl.n_blocks) % n_heads), int(f % wl.n_blocks)) for f in flat]
+    t0 = time.perf_counter()
+    orc.sla_forward(r["qhat"], r["khat"], r["vhat"], proj, r["cls"], wl.block, "softmax", qb)
+    t_blocks = time.perf_counter() - t0
+    seconds = t_front * wl.heads / n_heads + t_blocks * total / n
+    sample = (f"quantise x3 + plan on {n_heads} of {wl.heads} heads ({t_front:.1f} s) + forward on {n} of {total} "
+              f"query blocks ({t_blocks:.1f} s), each extrapolated to the whole step")
+    return seconds, sample
+
+
+def host_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max((p.get("num_threads", 1) for p in threadpool_info()), default=1)
+    except Exception:
+        n = 1
+    return int(n)
+
+
+def run_reference(args, wl):
+    rank, _, world = pdist.env_world()
+    if rank != 0:
+        return
+    inputs = wk.make_inputs(wl)
+    times = []
+    sample = ""
+    for _ in range(args.warmup):
+        time_oracle(wl, inputs, 1, 8)
+    for _ in range(args.steps):
+        sec, sample = time_oracle(wl, inputs, 2, max(16, args.oracle_blocks // 8))
+        times.append(sec)
+    sec = sum(times) / len(times)
+    value = wl.dense_equiv_flops / sec / 1e12
+    cores = host_threads()
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic", "impl": "reference",
+            "config": {"workload": wl.name, "batch": wl.batch, "heads": wl.heads, "tokens": wl.tokens,
+                       "head_dim": wl.head_dim, "block": wl.block, "crit": wl.crit, "neg": wl.neg},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------ CUDA path
+def run_ours(args, wl):
+    from paper_2605_11354_b200 import binding as lt
+    from paper_2605_11354_b200 import build as lb
+
+    rank, local_rank, world = pdist.init()
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the SLA forward has no CPU path")
+    device = torch.device("cuda", local_rank)
+    torch.cuda.set_device(device)
+    if rank == 0:
+        lb.build()
+    pdist.barrier(device)
+    lt.lib()
+
+    inputs = wk.make_inputs(wl)
+    host = {}
+    for name in ("q", "k", "v"):
+        if wl.src_dtype == "bf16":
+            t = torch.from_numpy(wk.bf16_bits(inputs[name]).view(np.int16)).view(torch.bfloat16)
+        else:
+            t = torch.from_numpy(inputs[name])
+        host[name] = t.pin_memory()
+    proj = torch.from_numpy(inputs["proj"]).to(device)
+    dev = {n: host[n].to(device) for n in ("q", "k", "v")}
+    eng = lt.SlaForward(wl.batch, wl.heads, wl.tokens, wl.block, wl.crit, wl.neg, device=device)
+    out_host = torch.empty(eng.out.shape, dtype=torch.float32).pin_memory()
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=device)
+    lt.profile_enable(True)
+
+    def step():
+        return eng.run(dev["q"], dev["k"], dev["v"], proj)
+
+    def step_e2e():
+        for n in ("q", "k", "v"):
+            dev[n].copy_(host[n], non_blocking=True)
+        out = eng.run(dev["q"], dev["k"], dev["v"], proj)
+        out_host.copy_(out, non_blocking=True)
+
+    def timed(fn, steps, collect_stages):
+        total_ms, stages = 0.0, []
+        for _ in range(steps):
+            flush.fill_(1)  # evict L2 between timed iterations (not timed)
+            start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            start.record()
+            fn()
+            end.record()
+            end.synchronize()
+            total_ms += start.elapsed_time(end)
+            if collect_stages:
+                stages.append(lt.profile_stage_ms())
+        return total_ms, stages
+
+    for _ in range(args.warmup):
+        step()
+        step_e2e()
+    torch.cuda.synchronize(device)
+    assert int(eng.status.item()) == 0
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    pdist.barrier(device)
+    torch.cuda.synchronize(device)
+    launches0 = lt.launch_count()
+    ms_total, stages = timed(step, args.steps, True)
+    launches = lt.launch_count() - launches0
+    torch.cuda.synchronize(device)
+    pdist.barrier(device)
+    e2e_total, _ = timed(step_e2e, args.steps, False)
+    torch.cuda.synchronize(device)
+    pdist.barrier(device)
+    clocks = sampler.stop()
+    assert int(eng.status.item()) == 0
+
+    flops = wl.dense_equiv_flops
+    value_flops, worst_s = pdist.aggregate_throughput(flops * args.steps, ms_total / 1e3, device)
+    e2e_flops, _ = pdist.aggregate_throughput(flops * args.steps, e2e_total / 1e3, device)
+
+    peaks, peak_kind = measured_peaks()
+    att_ms = statistics.mean(s[2] for s in stages)
+    crit_flops = executed_critical_flops(wl, eng.plan.k_crit)
+    achieved = crit_flops / (att_ms * 1e-3) / 1e12 if att_ms > 0 else 0.0
+    fp8_peak = peaks["bf16_tflops"] * FP8_OVER_BF16
+    roofline = {"kernel": "attention (critical-block softmax + linear branch + projection)", "bound": "tensor",
+                "achieved": achieved, "peak": fp8_peak, "unit": "TFLOP/s", "frac": achieved / fp8_peak,
+                "peak_source": f"2 x {peak_kind} bf16 burst (no fp8 figure measured; nominal fp8/bf16 ratio)",
+                "traffic": ATTENTION_DRAM_BYTES_PER_LAUNCH, "flops_per_launch": crit_flops,
+                "avg_launch_ms": att_ms,
+                "stage_ms": {"summary": statistics.mean(s[0] for s in stages),
+                             "aggregation": statistics.mean(s[1] for s in stages), "attention": att_ms}}
+
+    if rank != 0:
+        pdist.shutdown()
+        return
+    in_bytes = sum(host[n].numel() * host[n].element_size() for n in ("q", "k", "v"))
+    out_bytes = out_host.numel() * 4
+    line = {"metric": METRIC, "value": value_flops / 1e12, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": worst_s * 1e3 / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "fp8_e4m3", "data": "synthetic",
+            "config": {"workload": wl.name, "batch": wl.batch, "heads": wl.heads, "tokens": wl.tokens,
+                       "head_dim": wl.head_dim, "block": wl.block, "crit": wl.crit, "neg": wl.neg,
+                       "k_crit": eng.plan.k_crit, "k_marg": eng.plan.k_marg, "k_neg": eng.plan.k_neg,
+                       "source_dtype": wl.src_dtype, "l2": f"flushed between timed steps ({L2_FLUSH_BYTES >> 20} MiB write)",
+                       "parallelism": "independent replicas, no collective" if world > 1 else "single GPU"},
+            "e2e": {"value": e2e_flops / 1e12, "unit": UNIT, "h2d_bytes_per_step": in_bytes,
+                    "d2h_bytes_per_step": out_bytes},
+            "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline}
+    if world == 1 and not args.no_cpu_baseline:
+        sec, sample = time_oracle(wl, inputs, wl.heads, args.oracle_blocks)
+        line["cpu_baseline"] = {"value": flops / sec / 1e12, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
+                                "sample": sample}
+    print(json.dumps(line))
+    pdist.shutdown()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="vggt8", choices=sorted(wk.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
+    ap.add_argument("--oracle-blocks", type=int, default=512)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    wl = wk.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

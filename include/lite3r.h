@@ -1,0 +1,152 @@
+/*
+ * lite3r.h -- C ABI of the FP8 Sparse Linear Attention (SLA) forward for NVIDIA B200 (sm_100a).
+ *
+ * The library computes  A_SLA(Q,K,V) = A_sparse(Q,K,V) + Proj(A_lin(Q,K,V))   (paper Eq. 1, Algorithm 1)
+ * in its block-level form: tokens of one (batch, head) are cut into blocks of `block` tokens; Q and K are
+ * mean-pooled per block, every (query-block, key-block) pair is ranked by the pooled score and classified
+ * critical / marginal / negligible; critical pairs run exact softmax attention on the e4m3 operands, marginal
+ * pairs feed a linear-attention branch through the feature map phi, negligible pairs are skipped.
+ *
+ * General conventions (all entry points)
+ *   - Every pointer inside a struct or argument marked DEVICE is a CUDA device pointer owned by the caller.
+ *     The library never allocates or frees device memory, never synchronises the device and never changes
+ *     the current device; work is enqueued on `stream` and the call returns.
+ *   - Shapes: B = batch, H = heads, N = tokens, D = head_dim (must be 64), Bs = block (64 or 128),
+ *     Nb = ceil(N / Bs).  The last block of a sequence may be ragged; only its valid tokens take part.
+ *   - Errors detected on the host (bad argument, unsupported shape, short workspace, failed launch) are
+ *     returned as a lite3r_status; nothing has been enqueued when a call returns an error other than
+ *     LITE3R_ERR_CUDA.  There is no CPU fallback: without a CUDA device the compute calls fail.
+ *   - Same inputs give bit-identical outputs (fixed reduction orders, no floating-point atomics).
+ */
+#ifndef LITE3R_H
+#define LITE3R_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define LITE3R_API __attribute__((visibility("default")))
+#else
+#define LITE3R_API
+#endif
+
+typedef enum {
+  LITE3R_OK = 0,
+  LITE3R_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, misaligned pointer or stride, fraction outside [0,1] */
+  LITE3R_ERR_UNSUPPORTED = 2, /* head_dim != 64, block not in {64,128}, unknown dtype / phi */
+  LITE3R_ERR_WORKSPACE = 3,   /* workspace_bytes smaller than the size query reports */
+  LITE3R_ERR_CUDA = 4,        /* a CUDA call failed; see lite3r_last_cuda_error() */
+  LITE3R_ERR_TIMEOUT = 5      /* a bounded device-side wait expired (reported through device_status) */
+} lite3r_status;
+
+typedef enum { LITE3R_F32 = 0, LITE3R_BF16 = 1 } lite3r_dtype;
+
+/* Feature map of the linear branch.  SOFTMAX: softmax over the head_dim components (the benchmark
+ * contract).  ELU1: ELU(x)+1 (Algorithm 1, line 6). */
+typedef enum { LITE3R_PHI_SOFTMAX = 0, LITE3R_PHI_ELU1 = 1 } lite3r_phi;
+
+typedef struct {
+  int batch, heads, tokens, head_dim, block;
+} lite3r_shape;
+
+/* A source tensor [B, H, N, D] with arbitrary batch/head/token strides (in elements) and contiguous D.
+ * DEVICE pointer, 16-byte aligned; every stride must be a multiple of 8 elements. */
+typedef struct {
+  const void* ptr;
+  lite3r_dtype dtype;
+  long long stride_b, stride_h, stride_n;
+} lite3r_tensor;
+
+/* A block-quantised tensor (all DEVICE pointers, caller-allocated, 16-byte aligned):
+ *   codes  uint8 [B, H, Nb*Bs, D]  e4m3 codes, rows past N are zero
+ *   scales fp32  [B, H, Nb]        one scale per (b, h, token-block) tile of Bs x D:  x ~= value(code) * scale
+ *   colsum int32 [B, H, Nb, D]     per-tile column sums of the code values in units of 2^-9 (exact integers);
+ *                                  the pooled block mean is colsum * 2^-9 * scale / valid_tokens. */
+typedef struct {
+  unsigned char* codes;
+  float* scales;
+  int* colsum;
+} lite3r_fp8;
+
+/* The block plan (all DEVICE pointers, caller-allocated):
+ *   cls       int8  [B, H, Nb, Nb]    class of key block j for query block i: 0 negligible, 1 marginal, 2 critical
+ *   crit_idx  int32 [B, H, Nb, k_crit] key-block indices of the critical blocks of row i, ascending
+ *   marg_idx  int32 [B, H, Nb, k_marg] same for the marginal blocks; may be NULL (not written then)
+ * k_crit / k_marg / k_neg are the per-row counts lite3r_plan_sizes reports. */
+typedef struct {
+  signed char* cls;
+  int* crit_idx;
+  int* marg_idx;
+  int k_crit, k_marg, k_neg;
+} lite3r_plan;
+
+/* Byte sizes of the three buffers of a lite3r_fp8 for `shape`.  Host-only. */
+LITE3R_API lite3r_status lite3r_fp8_sizes(const lite3r_shape* shape, size_t* codes_bytes, size_t* scales_bytes,
+                               size_t* colsum_bytes);
+
+/* Per-row class counts and plan buffer sizes.  Counts: k_crit = 0 if crit == 0, else
+ * min(Nb, max(1, floor(crit*Nb + 0.5))); k_neg = min(Nb - k_crit, floor(neg*Nb + 0.5)); k_marg is the rest
+ * (the row-wise TopKMask of Algorithm 1 line 3 with its keep ratio, applied to blocks).  Host-only. */
+LITE3R_API lite3r_status lite3r_plan_sizes(const lite3r_shape* shape, double crit, double neg, size_t* cls_bytes,
+                                size_t* crit_idx_bytes, size_t* marg_idx_bytes, int* k_crit, int* k_marg,
+                                int* k_neg);
+
+/* Bytes of scratch lite3r_sla_forward needs for `shape` and these fractions.  Host-only. */
+LITE3R_API lite3r_status lite3r_forward_workspace(const lite3r_shape* shape, double crit, double neg, size_t* bytes);
+
+/* Scaled FP8 quantisation (paper appendix "Scaled FP8 Quantization" with the epsilon of "Implementation
+ * Details"), one scale per (b, h, token-block) tile, all in fp32:
+ *   amax = max |x| over the valid tokens of the tile;  scale = (amax + 1e-8) / 448;
+ *   code = e4m3_round_to_nearest_even(clamp(x / scale, -448, 448))   (IEEE fp32 division).
+ * Writes out.codes, out.scales and, when out.colsum is not NULL, out.colsum.  x: DEVICE source tensor. */
+LITE3R_API lite3r_status lite3r_quantize_fp8(const lite3r_tensor* x, const lite3r_shape* shape, lite3r_fp8 out, void* stream);
+
+/* Pooled scores and row-wise top-k classification (Algorithm 1 lines 2-3 on block means):
+ *   s_ij = mean_i(q_hat) . mean_j(k_hat) / sqrt(D), means over valid tokens of the dequantised blocks;
+ *   row i ranks j by (s_ij descending, j ascending); first k_crit critical, last k_neg negligible.
+ * Scores are evaluated from the exact integer column sums in fp64, so the ranking can differ from an exact
+ * evaluation only between scores that agree to ~1e-15 relative.  q, k need scales and colsum only.
+ * Fills plan->cls, plan->crit_idx, plan->marg_idx (if not NULL) and the three counts. */
+LITE3R_API lite3r_status lite3r_sla_plan(const lite3r_fp8* q, const lite3r_fp8* k, const lite3r_shape* shape, double crit,
+                              double neg, lite3r_plan* plan, void* stream);
+
+/* The SLA forward (Eq. 1; Algorithm 1 lines 4-10) for a given plan.
+ *   sparse branch: per query token, softmax over exactly the valid keys of the critical blocks of
+ *     (q_hat . k_hat) / sqrt(D), times v_hat;
+ *   linear branch: (phi(q_hat) G_i) / (phi(q_hat) . zeta_i) with G_i = sum over marginal blocks of
+ *     phi(K_j)^T V_j and zeta_i = sum of phi(K_j)^T 1;
+ *   out = sparse + linear @ proj[h]   (no bias).
+ * proj: DEVICE fp32 [H, D, D] row-major [d_in][d_out]; proj_head_stride in elements (D*D for per-head
+ * matrices, 0 for one matrix shared by all heads).
+ * out: DEVICE fp32 [B, H, N, D] with the given strides (elements, multiples of 4); rows past N are not written.
+ * workspace: DEVICE, 256-byte aligned, at least lite3r_forward_workspace() bytes; its contents are scratch.
+ * device_status: optional DEVICE int, set non-zero by the kernels if a bounded wait expired (read it after
+ * synchronising); may be NULL. */
+LITE3R_API lite3r_status lite3r_sla_forward(const lite3r_fp8* q, const lite3r_fp8* k, const lite3r_fp8* v, const float* proj,
+                                 long long proj_head_stride, const lite3r_shape* shape, lite3r_phi phi,
+                                 const lite3r_plan* plan, float* out, long long out_stride_b,
+                                 long long out_stride_h, long long out_stride_n, void* workspace,
+                                 size_t workspace_bytes, int* device_status, void* stream);
+
+/* Text for a status code; the last CUDA error code (cudaError_t as int) recorded by this thread. */
+LITE3R_API const char* lite3r_status_string(lite3r_status status);
+LITE3R_API int lite3r_last_cuda_error(void);
+
+/* Stage timing for benchmarks.  After lite3r_profile_enable(1) (call it with the device current; it creates CUDA
+ * events, no device memory), every lite3r_sla_forward brackets its three stages -- key-block summaries, marginal
+ * aggregation, attention -- with event records on the call's stream.  lite3r_profile_stage_ms waits for the last
+ * forward's events (the only blocking call of the library) and writes the three durations in milliseconds to
+ * ms (HOST, 3 floats; a stage that did not run reports 0).  Not thread-safe; meant for one benchmarking thread. */
+LITE3R_API lite3r_status lite3r_profile_enable(int enable);
+LITE3R_API lite3r_status lite3r_profile_stage_ms(float* ms);
+
+/* Number of kernel launches the library has enqueued since it was loaded (all threads). */
+LITE3R_API long long lite3r_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LITE3R_H */

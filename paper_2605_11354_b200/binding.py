@@ -1,0 +1,247 @@
+"""ctypes binding of liblite3r.so: argument marshalling only, every step runs in the CUDA kernels.
+
+The functions carry the C names (``lite3r_quantize_fp8``, ``lite3r_sla_plan``, ``lite3r_sla_forward``);
+torch is used for device memory and streams.  There is no fallback: if the shared library is missing
+the import of any compute function raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblite3r.so")
+_lib = None
+
+F32, BF16 = 0, 1
+PHI_SOFTMAX, PHI_ELU1 = 0, 1
+PHI_CODES = {"softmax": PHI_SOFTMAX, "elu1": PHI_ELU1}
+
+
+class Lite3rError(RuntimeError):
+    pass
+
+
+class Shape(C.Structure):
+    _fields_ = [("batch", C.c_int), ("heads", C.c_int), ("tokens", C.c_int), ("head_dim", C.c_int), ("block", C.c_int)]
+
+
+class Tensor(C.Structure):
+    _fields_ = [("ptr", C.c_void_p), ("dtype", C.c_int), ("stride_b", C.c_longlong), ("stride_h", C.c_longlong),
+                ("stride_n", C.c_longlong)]
+
+
+class Fp8(C.Structure):
+    _fields_ = [("codes", C.c_void_p), ("scales", C.c_void_p), ("colsum", C.c_void_p)]
+
+
+class Plan(C.Structure):
+    _fields_ = [("cls", C.c_void_p), ("crit_idx", C.c_void_p), ("marg_idx", C.c_void_p), ("k_crit", C.c_int),
+                ("k_marg", C.c_int), ("k_neg", C.c_int)]
+
+
+EXPORTS = ("lite3r_fp8_sizes", "lite3r_plan_sizes", "lite3r_forward_workspace", "lite3r_quantize_fp8",
+           "lite3r_sla_plan", "lite3r_sla_forward", "lite3r_status_string", "lite3r_last_cuda_error",
+           "lite3r_launch_count", "lite3r_profile_enable", "lite3r_profile_stage_ms")
+
+
+def lib() -> C.CDLL:
+    """Loads the shared library once; raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise Lite3rError(f"{_LIB_PATH} is missing: build it with `python -m paper_2605_11354_b200.build`")
+    L = C.CDLL(_LIB_PATH)
+    sz = C.POINTER(C.c_size_t)
+    ip = C.POINTER(C.c_int)
+    L.lite3r_fp8_sizes.argtypes = [C.POINTER(Shape), sz, sz, sz]
+    L.lite3r_plan_sizes.argtypes = [C.POINTER(Shape), C.c_double, C.c_double, sz, sz, sz, ip, ip, ip]
+    L.lite3r_forward_workspace.argtypes = [C.POINTER(Shape), C.c_double, C.c_double, sz]
+    L.lite3r_quantize_fp8.argtypes = [C.POINTER(Tensor), C.POINTER(Shape), Fp8, C.c_void_p]
+    L.lite3r_sla_plan.argtypes = [C.POINTER(Fp8), C.POINTER(Fp8), C.POINTER(Shape), C.c_double, C.c_double,
+                                  C.POINTER(Plan), C.c_void_p]
+    L.lite3r_sla_forward.argtypes = [C.POINTER(Fp8), C.POINTER(Fp8), C.POINTER(Fp8), C.c_void_p, C.c_longlong,
+                                     C.POINTER(Shape), C.c_int, C.POINTER(Plan), C.c_void_p, C.c_longlong,
+                                     C.c_longlong, C.c_longlong, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+    L.lite3r_status_string.argtypes = [C.c_int]
+    L.lite3r_status_string.restype = C.c_char_p
+    L.lite3r_last_cuda_error.restype = C.c_int
+    L.lite3r_launch_count.restype = C.c_longlong
+    L.lite3r_profile_enable.argtypes = [C.c_int]
+    L.lite3r_profile_enable.restype = C.c_int
+    L.lite3r_profile_stage_ms.argtypes = [C.POINTER(C.c_float)]
+    L.lite3r_profile_stage_ms.restype = C.c_int
+    for name in EXPORTS[:6]:
+        getattr(L, name).restype = C.c_int
+    _lib = L
+    return L
+
+
+def _check(status: int, what: str) -> None:
+    if status != 0:
+        L = lib()
+        msg = L.lite3r_status_string(status).decode()
+        extra = f" (cudaError {L.lite3r_last_cuda_error()})" if status == 4 else ""
+        raise Lite3rError(f"{what}: {msg}{extra}")
+
+
+def _stream_ptr(stream) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(s.cuda_stream)
+
+
+def launch_count() -> int:
+    return int(lib().lite3r_launch_count())
+
+
+def profile_enable(on: bool) -> None:
+    _check(lib().lite3r_profile_enable(1 if on else 0), "lite3r_profile_enable")
+
+
+def profile_stage_ms():
+    """(summary, aggregation, attention) milliseconds of the last forward; blocks until it has finished."""
+    ms = (C.c_float * 3)()
+    _check(lib().lite3r_profile_stage_ms(ms), "lite3r_profile_stage_ms")
+    return tuple(float(x) for x in ms)
+
+
+# ----------------------------------------------------------------------------- size queries (host only)
+def lite3r_fp8_sizes(shape: Shape):
+    a, b, c = C.c_size_t(), C.c_size_t(), C.c_size_t()
+    _check(lib().lite3r_fp8_sizes(C.byref(shape), C.byref(a), C.byref(b), C.byref(c)), "lite3r_fp8_sizes")
+    return a.value, b.value, c.value
+
+
+def lite3r_plan_sizes(shape: Shape, crit: float, neg: float):
+    a, b, c = C.c_size_t(), C.c_size_t(), C.c_size_t()
+    kc, km, kn = C.c_int(), C.c_int(), C.c_int()
+    _check(lib().lite3r_plan_sizes(C.byref(shape), crit, neg, C.byref(a), C.byref(b), C.byref(c), C.byref(kc),
+                                   C.byref(km), C.byref(kn)), "lite3r_plan_sizes")
+    return a.value, b.value, c.value, kc.value, km.value, kn.value
+
+
+def lite3r_forward_workspace(shape: Shape, crit: float, neg: float) -> int:
+    a = C.c_size_t()
+    _check(lib().lite3r_forward_workspace(C.byref(shape), crit, neg, C.byref(a)), "lite3r_forward_workspace")
+    return a.value
+
+
+# ----------------------------------------------------------------------------- device buffers
+@dataclass
+class Fp8Tensor:
+    codes: torch.Tensor  # uint8 [B,H,Nb*Bs,D]
+    scales: torch.Tensor  # fp32 [B,H,Nb]
+    colsum: torch.Tensor  # int32 [B,H,Nb,D]
+
+    def c_struct(self) -> Fp8:
+        return Fp8(self.codes.data_ptr(), self.scales.data_ptr(), self.colsum.data_ptr())
+
+
+@dataclass
+class PlanBuffers:
+    cls: torch.Tensor  # int8 [B,H,Nb,Nb]
+    crit_idx: torch.Tensor  # int32 [B,H,Nb,k_crit]
+    marg_idx: torch.Tensor  # int32 [B,H,Nb,k_marg]
+    k_crit: int
+    k_marg: int
+    k_neg: int
+
+    def c_struct(self) -> Plan:
+        return Plan(self.cls.data_ptr(), self.crit_idx.data_ptr() if self.k_crit else None,
+                    self.marg_idx.data_ptr() if self.k_marg else None, self.k_crit, self.k_marg, self.k_neg)
+
+
+def alloc_fp8(shape: Shape, device) -> Fp8Tensor:
+    nb = -(-shape.tokens // shape.block)
+    B, H, D = shape.batch, shape.heads, shape.head_dim
+    return Fp8Tensor(torch.empty((B, H, nb * shape.block, D), dtype=torch.uint8, device=device),
+                     torch.empty((B, H, nb), dtype=torch.float32, device=device),
+                     torch.empty((B, H, nb, D), dtype=torch.int32, device=device))
+
+
+def alloc_plan(shape: Shape, crit: float, neg: float, device) -> PlanBuffers:
+    _, _, _, kc, km, kn = lite3r_plan_sizes(shape, crit, neg)
+    nb = -(-shape.tokens // shape.block)
+    B, H = shape.batch, shape.heads
+    return PlanBuffers(torch.empty((B, H, nb, nb), dtype=torch.int8, device=device),
+                       torch.empty((B, H, nb, max(kc, 1)), dtype=torch.int32, device=device)[..., :kc],
+                       torch.empty((B, H, nb, max(km, 1)), dtype=torch.int32, device=device)[..., :km], kc, km, kn)
+
+
+# ----------------------------------------------------------------------------- the three calls
+def lite3r_quantize_fp8(x: torch.Tensor, shape: Shape, out: Fp8Tensor, stream=None) -> None:
+    """x: CUDA tensor [B,H,N,D] (any b/h/n strides, contiguous D), fp32 or bf16."""
+    if not x.is_cuda or x.dim() != 4 or x.stride(3) != 1:
+        raise Lite3rError("lite3r_quantize_fp8: x must be a CUDA tensor [B,H,N,D] with contiguous D")
+    dtype = {torch.float32: F32, torch.bfloat16: BF16}.get(x.dtype)
+    if dtype is None:
+        raise Lite3rError("lite3r_quantize_fp8: dtype must be float32 or bfloat16")
+    t = Tensor(x.data_ptr(), dtype, x.stride(0), x.stride(1), x.stride(2))
+    _check(lib().lite3r_quantize_fp8(C.byref(t), C.byref(shape), out.c_struct(), _stream_ptr(stream)),
+           "lite3r_quantize_fp8")
+
+
+def lite3r_sla_plan(q: Fp8Tensor, k: Fp8Tensor, shape: Shape, crit: float, neg: float, plan: PlanBuffers,
+                    stream=None) -> None:
+    p = plan.c_struct()
+    qs, ks = q.c_struct(), k.c_struct()
+    _check(lib().lite3r_sla_plan(C.byref(qs), C.byref(ks), C.byref(shape), crit, neg, C.byref(p),
+                                 _stream_ptr(stream)), "lite3r_sla_plan")
+    assert (p.k_crit, p.k_marg, p.k_neg) == (plan.k_crit, plan.k_marg, plan.k_neg)
+
+
+def lite3r_sla_forward(q: Fp8Tensor, k: Fp8Tensor, v: Fp8Tensor, proj: torch.Tensor, shape: Shape, phi: int,
+                       plan: PlanBuffers, out: torch.Tensor, workspace: torch.Tensor, device_status=None,
+                       stream=None) -> None:
+    """proj: CUDA fp32 [H,D,D] or [D,D] (shared); out: CUDA fp32 [B,H,N,D] view with contiguous D."""
+    if proj.dtype != torch.float32 or not proj.is_cuda or not proj.is_contiguous():
+        raise Lite3rError("lite3r_sla_forward: proj must be a contiguous CUDA float32 tensor")
+    if out.dtype != torch.float32 or not out.is_cuda or out.stride(3) != 1:
+        raise Lite3rError("lite3r_sla_forward: out must be a CUDA float32 tensor [B,H,N,D] with contiguous D")
+    head_stride = proj.stride(0) if proj.dim() == 3 else 0
+    p = plan.c_struct()
+    qs, ks, vs = q.c_struct(), k.c_struct(), v.c_struct()
+    _check(lib().lite3r_sla_forward(C.byref(qs), C.byref(ks), C.byref(vs), proj.data_ptr(), head_stride,
+                                    C.byref(shape), phi, C.byref(p), out.data_ptr(), out.stride(0), out.stride(1),
+                                    out.stride(2), workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                    device_status.data_ptr() if device_status is not None else None,
+                                    _stream_ptr(stream)), "lite3r_sla_forward")
+
+
+# ----------------------------------------------------------------------------- whole path
+class SlaForward:
+    """Pre-allocated buffers for one shape; ``run`` enqueues quantise x3 + plan + forward and returns ``out``."""
+
+    def __init__(self, batch, heads, tokens, block, crit, neg, phi="softmax", device="cuda:0", head_dim=64):
+        self.shape = Shape(batch, heads, tokens, head_dim, block)
+        self.crit, self.neg, self.phi = float(crit), float(neg), PHI_CODES[phi]
+        self.device = torch.device(device)
+        self.q8, self.k8, self.v8 = (alloc_fp8(self.shape, self.device) for _ in range(3))
+        self.plan = alloc_plan(self.shape, self.crit, self.neg, self.device)
+        nbytes = lite3r_forward_workspace(self.shape, self.crit, self.neg)
+        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+        off = (-self.workspace.data_ptr()) % 256
+        self.workspace = self.workspace[off:off + nbytes]
+        self.out = torch.empty((batch, heads, tokens, head_dim), dtype=torch.float32, device=self.device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=self.device)
+
+    def quantize(self, q, k, v, stream=None):
+        lite3r_quantize_fp8(q, self.shape, self.q8, stream)
+        lite3r_quantize_fp8(k, self.shape, self.k8, stream)
+        lite3r_quantize_fp8(v, self.shape, self.v8, stream)
+
+    def make_plan(self, stream=None):
+        lite3r_sla_plan(self.q8, self.k8, self.shape, self.crit, self.neg, self.plan, stream)
+
+    def forward(self, proj, stream=None):
+        lite3r_sla_forward(self.q8, self.k8, self.v8, proj, self.shape, self.phi, self.plan, self.out,
+                           self.workspace, self.status, stream)
+        return self.out
+
+    def run(self, q, k, v, proj, stream=None):
+        self.quantize(q, k, v, stream)
+        self.make_plan(stream)
+        return self.forward(proj, stream)

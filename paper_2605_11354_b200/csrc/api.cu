@@ -1,0 +1,237 @@
+// C-ABI entry points of the lite3r library: argument validation, size queries and dispatch.
+#include <atomic>
+#include <cmath>
+
+#include "common.cuh"
+
+namespace lite3r {
+
+static thread_local int g_last_cuda_error = 0;
+static std::atomic<long long> g_launches{0};
+
+lite3r_status record_cuda(cudaError_t err) {
+  if (err == cudaSuccess) return LITE3R_OK;
+  g_last_cuda_error = static_cast<int>(err);
+  return LITE3R_ERR_CUDA;
+}
+
+lite3r_status after_launch() {
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return record_cuda(cudaGetLastError());
+}
+
+static bool g_profile = false;
+static cudaEvent_t g_events[6] = {};
+static bool g_marked[6] = {};
+
+void profile_mark(int idx, cudaStream_t stream) {
+  if (!g_profile) return;
+  if (idx == 0)
+    for (bool& m : g_marked) m = false;
+  if (cudaEventRecord(g_events[idx], stream) == cudaSuccess) g_marked[idx] = true;
+}
+
+Counts class_counts(int nb, double crit, double neg) {
+  Counts c;
+  if (crit == 0.0) {
+    c.k_crit = 0;
+  } else {
+    long long kc = static_cast<long long>(std::floor(crit * nb + 0.5));
+    if (kc < 1) kc = 1;
+    if (kc > nb) kc = nb;
+    c.k_crit = static_cast<int>(kc);
+  }
+  long long kn = static_cast<long long>(std::floor(neg * nb + 0.5));
+  if (kn > nb - c.k_crit) kn = nb - c.k_crit;
+  c.k_neg = static_cast<int>(kn);
+  c.k_marg = nb - c.k_crit - c.k_neg;
+  return c;
+}
+
+static lite3r_status check_shape(const lite3r_shape* s) {
+  if (s == nullptr) return LITE3R_ERR_INVALID_ARG;
+  if (s->batch <= 0 || s->heads <= 0 || s->tokens <= 0) return LITE3R_ERR_INVALID_ARG;
+  if (s->head_dim != kHeadDim) return LITE3R_ERR_UNSUPPORTED;
+  if (s->block != 64 && s->block != 128) return LITE3R_ERR_UNSUPPORTED;
+  const long long rows = static_cast<long long>(s->batch) * s->heads * ceil_div(s->tokens, s->block);
+  if (rows > 0x7FFFFFFFLL / 4) return LITE3R_ERR_UNSUPPORTED;  // tile ids are 32-bit
+  return LITE3R_OK;
+}
+
+static lite3r_status check_fractions(double crit, double neg) {
+  if (!(crit >= 0.0 && crit <= 1.0) || !(neg >= 0.0 && neg <= 1.0)) return LITE3R_ERR_INVALID_ARG;
+  return LITE3R_OK;
+}
+
+static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+static lite3r_status check_fp8(const lite3r_fp8* t, bool need_codes, bool need_colsum) {
+  if (t == nullptr || t->scales == nullptr) return LITE3R_ERR_INVALID_ARG;
+  if (need_codes && (t->codes == nullptr || !aligned(t->codes, 16))) return LITE3R_ERR_INVALID_ARG;
+  if (need_colsum && t->colsum == nullptr) return LITE3R_ERR_INVALID_ARG;
+  if (!aligned(t->scales, 4) || (t->colsum != nullptr && !aligned(t->colsum, 16))) return LITE3R_ERR_INVALID_ARG;
+  return LITE3R_OK;
+}
+
+}  // namespace lite3r
+
+using namespace lite3r;
+
+extern "C" {
+
+lite3r_status lite3r_fp8_sizes(const lite3r_shape* shape, size_t* codes_bytes, size_t* scales_bytes,
+                               size_t* colsum_bytes) {
+  lite3r_status st = check_shape(shape);
+  if (st != LITE3R_OK) return st;
+  const size_t bh = static_cast<size_t>(shape->batch) * shape->heads;
+  const size_t nb = ceil_div(shape->tokens, shape->block);
+  if (codes_bytes) *codes_bytes = bh * nb * shape->block * kHeadDim;
+  if (scales_bytes) *scales_bytes = bh * nb * sizeof(float);
+  if (colsum_bytes) *colsum_bytes = bh * nb * kHeadDim * sizeof(int);
+  return LITE3R_OK;
+}
+
+lite3r_status lite3r_plan_sizes(const lite3r_shape* shape, double crit, double neg, size_t* cls_bytes,
+                                size_t* crit_idx_bytes, size_t* marg_idx_bytes, int* k_crit, int* k_marg,
+                                int* k_neg) {
+  lite3r_status st = check_shape(shape);
+  if (st != LITE3R_OK) return st;
+  st = check_fractions(crit, neg);
+  if (st != LITE3R_OK) return st;
+  const size_t bh = static_cast<size_t>(shape->batch) * shape->heads;
+  const size_t nb = ceil_div(shape->tokens, shape->block);
+  const Counts c = class_counts(static_cast<int>(nb), crit, neg);
+  if (cls_bytes) *cls_bytes = bh * nb * nb;
+  if (crit_idx_bytes) *crit_idx_bytes = bh * nb * c.k_crit * sizeof(int);
+  if (marg_idx_bytes) *marg_idx_bytes = bh * nb * c.k_marg * sizeof(int);
+  if (k_crit) *k_crit = c.k_crit;
+  if (k_marg) *k_marg = c.k_marg;
+  if (k_neg) *k_neg = c.k_neg;
+  return LITE3R_OK;
+}
+
+lite3r_status lite3r_forward_workspace(const lite3r_shape* shape, double crit, double neg, size_t* bytes) {
+  lite3r_status st = check_shape(shape);
+  if (st != LITE3R_OK) return st;
+  st = check_fractions(crit, neg);
+  if (st != LITE3R_OK) return st;
+  if (bytes == nullptr) return LITE3R_ERR_INVALID_ARG;
+  *bytes = forward_workspace_bytes(*shape, class_counts(ceil_div(shape->tokens, shape->block), crit, neg));
+  return LITE3R_OK;
+}
+
+lite3r_status lite3r_quantize_fp8(const lite3r_tensor* x, const lite3r_shape* shape, lite3r_fp8 out, void* stream) {
+  lite3r_status st = check_shape(shape);
+  if (st != LITE3R_OK) return st;
+  if (x == nullptr || x->ptr == nullptr || !aligned(x->ptr, 16)) return LITE3R_ERR_INVALID_ARG;
+  if (x->dtype != LITE3R_F32 && x->dtype != LITE3R_BF16) return LITE3R_ERR_UNSUPPORTED;
+  if (x->stride_n < kHeadDim || x->stride_b < 0 || x->stride_h < 0) return LITE3R_ERR_INVALID_ARG;
+  if ((x->stride_b % 8) || (x->stride_h % 8) || (x->stride_n % 8)) return LITE3R_ERR_INVALID_ARG;
+  st = check_fp8(&out, true, false);
+  if (st != LITE3R_OK) return st;
+  return launch_quantize(*x, *shape, out, static_cast<cudaStream_t>(stream));
+}
+
+lite3r_status lite3r_sla_plan(const lite3r_fp8* q, const lite3r_fp8* k, const lite3r_shape* shape, double crit,
+                              double neg, lite3r_plan* plan, void* stream) {
+  lite3r_status st = check_shape(shape);
+  if (st != LITE3R_OK) return st;
+  st = check_fractions(crit, neg);
+  if (st != LITE3R_OK) return st;
+  if ((st = check_fp8(q, false, true)) != LITE3R_OK) return st;
+  if ((st = check_fp8(k, false, true)) != LITE3R_OK) return st;
+  if (plan == nullptr || plan->cls == nullptr) return LITE3R_ERR_INVALID_ARG;
+  const Counts c = class_counts(ceil_div(shape->tokens, shape->block), crit, neg);
+  if (c.k_crit > 0 && plan->crit_idx == nullptr) return LITE3R_ERR_INVALID_ARG;
+  plan->k_crit = c.k_crit;
+  plan->k_marg = c.k_marg;
+  plan->k_neg = c.k_neg;
+  return launch_plan(*q, *k, *shape, c, *plan, static_cast<cudaStream_t>(stream));
+}
+
+lite3r_status lite3r_sla_forward(const lite3r_fp8* q, const lite3r_fp8* k, const lite3r_fp8* v, const float* proj,
+                                 long long proj_head_stride, const lite3r_shape* shape, lite3r_phi phi,
+                                 const lite3r_plan* plan, float* out, long long out_stride_b,
+                                 long long out_stride_h, long long out_stride_n, void* workspace,
+                                 size_t workspace_bytes, int* device_status, void* stream) {
+  lite3r_status st = check_shape(shape);
+  if (st != LITE3R_OK) return st;
+  if ((st = check_fp8(q, true, false)) != LITE3R_OK) return st;
+  if ((st = check_fp8(k, true, false)) != LITE3R_OK) return st;
+  if ((st = check_fp8(v, true, false)) != LITE3R_OK) return st;
+  if (phi != LITE3R_PHI_SOFTMAX && phi != LITE3R_PHI_ELU1) return LITE3R_ERR_UNSUPPORTED;
+  if (proj == nullptr || !aligned(proj, 16) || proj_head_stride < 0 || (proj_head_stride % 4)) return LITE3R_ERR_INVALID_ARG;
+  if (out == nullptr || !aligned(out, 16)) return LITE3R_ERR_INVALID_ARG;
+  if (out_stride_n < kHeadDim || out_stride_b < 0 || out_stride_h < 0) return LITE3R_ERR_INVALID_ARG;
+  if ((out_stride_b % 4) || (out_stride_h % 4) || (out_stride_n % 4)) return LITE3R_ERR_INVALID_ARG;
+  if (plan == nullptr || plan->cls == nullptr) return LITE3R_ERR_INVALID_ARG;
+  const int nb = ceil_div(shape->tokens, shape->block);
+  if (plan->k_crit < 0 || plan->k_marg < 0 || plan->k_neg < 0 || plan->k_crit + plan->k_marg + plan->k_neg != nb)
+    return LITE3R_ERR_INVALID_ARG;
+  if (plan->k_crit > 0 && plan->crit_idx == nullptr) return LITE3R_ERR_INVALID_ARG;
+  const Counts c{plan->k_crit, plan->k_marg, plan->k_neg};
+  if (workspace == nullptr || !aligned(workspace, 256)) return LITE3R_ERR_INVALID_ARG;
+  if (workspace_bytes < forward_workspace_bytes(*shape, c)) return LITE3R_ERR_WORKSPACE;
+  ForwardArgs a;
+  a.q = *q;
+  a.k = *k;
+  a.v = *v;
+  a.proj = proj;
+  a.proj_head_stride = proj_head_stride;
+  a.s = *shape;
+  a.phi = static_cast<int>(phi);
+  a.plan = *plan;
+  a.out = out;
+  a.out_stride_b = out_stride_b;
+  a.out_stride_h = out_stride_h;
+  a.out_stride_n = out_stride_n;
+  a.workspace = workspace;
+  a.workspace_bytes = workspace_bytes;
+  a.device_status = device_status;
+  return launch_forward(a, static_cast<cudaStream_t>(stream));
+}
+
+lite3r_status lite3r_profile_enable(int enable) {
+  if (enable && !g_profile) {
+    for (cudaEvent_t& e : g_events) {
+      lite3r_status st = record_cuda(cudaEventCreate(&e));
+      if (st != LITE3R_OK) return st;
+    }
+  } else if (!enable && g_profile) {
+    for (cudaEvent_t& e : g_events) cudaEventDestroy(e);
+  }
+  g_profile = enable != 0;
+  return LITE3R_OK;
+}
+
+lite3r_status lite3r_profile_stage_ms(float* ms) {
+  if (ms == nullptr || !g_profile) return LITE3R_ERR_INVALID_ARG;
+  for (int s = 0; s < 3; ++s) {
+    ms[s] = 0.f;
+    if (g_marked[2 * s] && g_marked[2 * s + 1]) {
+      lite3r_status st = record_cuda(cudaEventSynchronize(g_events[2 * s + 1]));
+      if (st != LITE3R_OK) return st;
+      st = record_cuda(cudaEventElapsedTime(&ms[s], g_events[2 * s], g_events[2 * s + 1]));
+      if (st != LITE3R_OK) return st;
+    }
+  }
+  return LITE3R_OK;
+}
+
+const char* lite3r_status_string(lite3r_status status) {
+  switch (status) {
+    case LITE3R_OK: return "ok";
+    case LITE3R_ERR_INVALID_ARG: return "invalid argument";
+    case LITE3R_ERR_UNSUPPORTED: return "unsupported shape, dtype or option";
+    case LITE3R_ERR_WORKSPACE: return "workspace too small";
+    case LITE3R_ERR_CUDA: return "CUDA error";
+    case LITE3R_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+int lite3r_last_cuda_error(void) { return g_last_cuda_error; }
+
+long long lite3r_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

@@ -1,0 +1,85 @@
+// Shared host/device helpers of the lite3r library (internal; the public surface is include/lite3r.h).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_fp8.h>
+#include <stdint.h>
+
+#include "lite3r.h"
+
+namespace lite3r {
+
+constexpr int kHeadDim = 64;
+// One row of per-key-block linear-branch summaries: (H_j W)^T as [e][d] (4096 values) followed by z_j[d] (64).
+constexpr int kSummaryRow = kHeadDim * kHeadDim + kHeadDim;
+
+// Records a CUDA error for lite3r_last_cuda_error(); returns LITE3R_ERR_CUDA if err != cudaSuccess.
+lite3r_status record_cuda(cudaError_t err);
+// Counts one enqueued kernel launch and returns the launch's error state as a status.
+lite3r_status after_launch();
+
+// Benchmark stage timing: records event `idx` (0..5) on `stream` when profiling is enabled.
+void profile_mark(int idx, cudaStream_t stream);
+
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+struct Counts {
+  int k_crit, k_marg, k_neg;
+};
+Counts class_counts(int nb, double crit, double neg);
+
+// Value of an e4m3 code in units of 2^-9 (an exact integer, |v| <= 448 * 512).
+__device__ __forceinline__ int e4m3_units(uint32_t code) {
+  const int e = (code >> 3) & 0xF;
+  const int m = code & 0x7;
+  const int mag = e ? ((8 | m) << (e - 1)) : m;
+  return (code & 0x80) ? -mag : mag;
+}
+
+// Decodes four packed e4m3 codes to fp32 (exact).
+__device__ __forceinline__ void e4m3x4_to_float(uint32_t packed, float out[4]) {
+  const __half2_raw lo = __nv_cvt_fp8x2_to_halfraw2(static_cast<__nv_fp8x2_storage_t>(packed & 0xFFFFu), __NV_E4M3);
+  const __half2_raw hi = __nv_cvt_fp8x2_to_halfraw2(static_cast<__nv_fp8x2_storage_t>(packed >> 16), __NV_E4M3);
+  const float2 a = __half22float2(__half2(lo));
+  const float2 b = __half22float2(__half2(hi));
+  out[0] = a.x;
+  out[1] = a.y;
+  out[2] = b.x;
+  out[3] = b.y;
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  return v;
+}
+
+// Kernel launchers (one per translation unit).  All enqueue on `stream` and return a status.
+lite3r_status launch_quantize(const lite3r_tensor& x, const lite3r_shape& s, const lite3r_fp8& out, cudaStream_t stream);
+lite3r_status launch_plan(const lite3r_fp8& q, const lite3r_fp8& k, const lite3r_shape& s, const Counts& c,
+                          const lite3r_plan& plan, cudaStream_t stream);
+
+struct ForwardArgs {
+  lite3r_fp8 q, k, v;
+  const float* proj;
+  long long proj_head_stride;
+  lite3r_shape s;
+  int phi;
+  lite3r_plan plan;
+  float* out;
+  long long out_stride_b, out_stride_h, out_stride_n;
+  void* workspace;
+  size_t workspace_bytes;
+  int* device_status;
+};
+size_t forward_workspace_bytes(const lite3r_shape& s, const Counts& c);
+lite3r_status launch_forward(const ForwardArgs& a, cudaStream_t stream);
+
+}  // namespace lite3r
