@@ -131,6 +131,34 @@ LITE3R_API lite3r_status lite3r_sla_forward(const lite3r_fp8* q, const lite3r_fp
                                  long long out_stride_h, long long out_stride_n, void* workspace,
                                  size_t workspace_bytes, int* device_status, void* stream);
 
+/* The same forward for callers that cannot provide scratch memory.  (The paper has no counterpart: this entry
+ * point exists for deployments, not for the method.)
+ *
+ * Who needs it: code that is not allowed to allocate device memory where it calls the library -- a plug-in that
+ * lives inside another runtime's pre-planned memory arena, a latency-critical loop that must stay away from the
+ * allocator, a process whose memory pool is already sized to the last byte.  Such a caller still owns the inputs
+ * and the output, but has nowhere to take the workspace of lite3r_sla_forward from.
+ *
+ * Here the scratch is a fixed array of LITE3R_STATIC_SCRATCH_BYTES inside the library image: every GPU on which
+ * the library is loaded sets that much memory aside until the process exits, whether or not this call is used.
+ * The call allocates and frees nothing, on the device or through any library.  Arguments are those of
+ * lite3r_sla_forward without workspace / workspace_bytes, and the results are identical.
+ *   - Limit: if lite3r_forward_workspace() for this shape exceeds LITE3R_STATIC_SCRATCH_BYTES the call returns
+ *     LITE3R_ERR_WORKSPACE and enqueues nothing (32 MiB holds 1344 (batch x head x block) tiles, e.g. two heads of
+ *     an 8-frame 10992-token sequence at block 64); use lite3r_sla_forward with your own buffer for larger problems.
+ *   - The first call on each device looks up the array's device address (the device must be current); make that
+ *     first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps whatever the previous call left there.  The forward
+ *     overwrites every scratch element before reading it, so nothing needs clearing between calls, but two calls
+ *     whose kernels may overlap on the GPU (different streams, no ordering between them) race on the array:
+ *     serialise them. */
+#define LITE3R_STATIC_SCRATCH_BYTES (32u << 20)
+LITE3R_API lite3r_status lite3r_sla_forward_static_scratch(const lite3r_fp8* q, const lite3r_fp8* k, const lite3r_fp8* v,
+                                                const float* proj, long long proj_head_stride,
+                                                const lite3r_shape* shape, lite3r_phi phi, const lite3r_plan* plan,
+                                                float* out, long long out_stride_b, long long out_stride_h,
+                                                long long out_stride_n, int* device_status, void* stream);
+
 /* Text for a status code; the last CUDA error code (cudaError_t as int) recorded by this thread. */
 LITE3R_API const char* lite3r_status_string(lite3r_status status);
 LITE3R_API int lite3r_last_cuda_error(void);

@@ -44,7 +44,9 @@ class Plan(C.Structure):
 
 EXPORTS = ("lite3r_fp8_sizes", "lite3r_plan_sizes", "lite3r_forward_workspace", "lite3r_quantize_fp8",
            "lite3r_sla_plan", "lite3r_sla_forward", "lite3r_status_string", "lite3r_last_cuda_error",
-           "lite3r_launch_count", "lite3r_profile_enable", "lite3r_profile_stage_ms")
+           "lite3r_launch_count", "lite3r_profile_enable", "lite3r_profile_stage_ms",
+           "lite3r_sla_forward_static_scratch")
+STATIC_SCRATCH_BYTES = 32 << 20  # LITE3R_STATIC_SCRATCH_BYTES
 
 
 def lib() -> C.CDLL:
@@ -66,6 +68,11 @@ def lib() -> C.CDLL:
     L.lite3r_sla_forward.argtypes = [C.POINTER(Fp8), C.POINTER(Fp8), C.POINTER(Fp8), C.c_void_p, C.c_longlong,
                                      C.POINTER(Shape), C.c_int, C.POINTER(Plan), C.c_void_p, C.c_longlong,
                                      C.c_longlong, C.c_longlong, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+    L.lite3r_sla_forward_static_scratch.argtypes = [C.POINTER(Fp8), C.POINTER(Fp8), C.POINTER(Fp8), C.c_void_p,
+                                                    C.c_longlong, C.POINTER(Shape), C.c_int, C.POINTER(Plan),
+                                                    C.c_void_p, C.c_longlong, C.c_longlong, C.c_longlong, C.c_void_p,
+                                                    C.c_void_p]
+    L.lite3r_sla_forward_static_scratch.restype = C.c_int
     L.lite3r_status_string.argtypes = [C.c_int]
     L.lite3r_status_string.restype = C.c_char_p
     L.lite3r_last_cuda_error.restype = C.c_int
@@ -209,6 +216,26 @@ def lite3r_sla_forward(q: Fp8Tensor, k: Fp8Tensor, v: Fp8Tensor, proj: torch.Ten
                                     out.stride(2), workspace.data_ptr(), workspace.numel() * workspace.element_size(),
                                     device_status.data_ptr() if device_status is not None else None,
                                     _stream_ptr(stream)), "lite3r_sla_forward")
+
+
+def lite3r_sla_forward_static_scratch(q: Fp8Tensor, k: Fp8Tensor, v: Fp8Tensor, proj: torch.Tensor, shape: Shape,
+                                      phi: int, plan: PlanBuffers, out: torch.Tensor, device_status=None,
+                                      stream=None) -> None:
+    """lite3r_sla_forward for callers that may not allocate: the scratch is a fixed 32 MiB array inside the
+    library (held on every GPU that loads it), so no workspace is passed.  Raises "workspace too small" when the
+    shape needs more than that.  Calls on one device share the array: do not let two of them overlap on the GPU."""
+    if proj.dtype != torch.float32 or not proj.is_cuda or not proj.is_contiguous():
+        raise Lite3rError("lite3r_sla_forward_static_scratch: proj must be a contiguous CUDA float32 tensor")
+    if out.dtype != torch.float32 or not out.is_cuda or out.stride(3) != 1:
+        raise Lite3rError("lite3r_sla_forward_static_scratch: out must be CUDA float32 [B,H,N,D], contiguous D")
+    head_stride = proj.stride(0) if proj.dim() == 3 else 0
+    p = plan.c_struct()
+    qs, ks, vs = q.c_struct(), k.c_struct(), v.c_struct()
+    _check(lib().lite3r_sla_forward_static_scratch(
+        C.byref(qs), C.byref(ks), C.byref(vs), proj.data_ptr(), head_stride, C.byref(shape), phi, C.byref(p),
+        out.data_ptr(), out.stride(0), out.stride(1), out.stride(2),
+        device_status.data_ptr() if device_status is not None else None, _stream_ptr(stream)),
+        "lite3r_sla_forward_static_scratch")
 
 
 # ----------------------------------------------------------------------------- whole path
