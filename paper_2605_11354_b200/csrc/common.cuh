@@ -79,6 +79,25 @@ struct ForwardArgs {
   size_t workspace_bytes;
   int* device_status;
 };
+struct AttentionLaunch {
+  lite3r_shape shape;
+  const uint8_t* q_codes;
+  const uint8_t* k_codes;
+  const float* q_scales;
+  const float* k_scales;
+  const float* v_scales;
+  const __half* v16;          // [tiles*Bs][64] V code values as fp16
+  const __nv_bfloat16* g16;   // [tiles][64][64] aggregated projected summaries, [e][d]
+  const float* zeta;          // [tiles][64]
+  const float* vref;          // [B*H]
+  const int* crit_idx;
+  int k_crit, k_marg, phi;
+  float* out;
+  long long out_stride_b, out_stride_h, out_stride_n;
+  int* device_status;
+};
+lite3r_status launch_attention(const AttentionLaunch& a, cudaStream_t stream);
+
 size_t forward_workspace_bytes(const lite3r_shape& s, const Counts& c);
 lite3r_status launch_forward(const ForwardArgs& a, cudaStream_t stream);
 

@@ -7,6 +7,8 @@
 //   K4  attention_kernel  per query block i: online-softmax attention over the critical key blocks (lines 4-5),
 //                         then the linear branch (line 9) phi(q) G_i / (phi(q) . zeta_i), the sum of the two
 //                         (line 10) and the store.
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace lite3r {
@@ -132,7 +134,8 @@ constexpr int kAggPer = (kSummaryRow / 2 + kAggThreads - 1) / kAggThreads;  // b
 __global__ void __launch_bounds__(kAggThreads) aggregate_kernel(const __nv_bfloat16* __restrict__ hws,
                                                                 const int* __restrict__ marg_idx,
                                                                 const signed char* __restrict__ cls, int nb, int k_marg,
-                                                                float* __restrict__ g) {
+                                                                __nv_bfloat16* __restrict__ g16,
+                                                                float* __restrict__ zeta) {
   extern __shared__ int s_list[];  // [k_marg]
   const int row = blockIdx.x;      // (b*H + h) * nb + i
   const size_t bh_rows = static_cast<size_t>(row / nb) * nb;
@@ -160,197 +163,122 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_kernel(const __nv_bfloa
       }
     }
   }
-  float2* dst = reinterpret_cast<float2*>(g + static_cast<size_t>(row) * kSummaryRow);
+  __nv_bfloat162* dst = reinterpret_cast<__nv_bfloat162*>(g16 + static_cast<size_t>(row) * kHeadDim * kHeadDim);
+  float2* dst_z = reinterpret_cast<float2*>(zeta + static_cast<size_t>(row) * kHeadDim);
 #pragma unroll
   for (int x = 0; x < kAggPer; ++x) {
     const int n = threadIdx.x + x * kAggThreads;
-    if (n < kSummaryRow / 2) dst[n] = acc[x];
+    if (n < kHeadDim * kHeadDim / 2) {
+      dst[n] = __floats2bfloat162_rn(acc[x].x, acc[x].y);
+    } else if (n < kSummaryRow / 2) {
+      dst_z[n - kHeadDim * kHeadDim / 2] = acc[x];
+    }
   }
 }
 
-// ------------------------------------------------------------------------------------------------ K4
-template <int BS>
-__global__ void __launch_bounds__(BS) attention_kernel(const uint8_t* __restrict__ q_codes,
-                                                       const float* __restrict__ q_scales,
-                                                       const uint8_t* __restrict__ k_codes,
-                                                       const float* __restrict__ k_scales,
-                                                       const uint8_t* __restrict__ v_codes,
-                                                       const float* __restrict__ v_scales,
-                                                       const int* __restrict__ crit_idx, const float* __restrict__ g,
-                                                       int heads, int tokens, int nb, int k_crit, int k_marg, int phi,
-                                                       float* __restrict__ out, long long out_stride_b,
-                                                       long long out_stride_h, long long out_stride_n) {
-  extern __shared__ __align__(16) float smem_f[];
-  float* s_k = smem_f;               // [BS][64]
-  float* s_v = s_k + BS * kHeadDim;  // [BS][64]
-
-  const int row_tile = blockIdx.x;  // (b*H + h) * nb + i
-  const int i = row_tile % nb;
-  const int bh = row_tile / nb;
-  const int h = bh % heads, b = bh / heads;
-  const size_t bh_rows = static_cast<size_t>(bh) * nb;
-  const int t = threadIdx.x;
-  const int token = i * BS + t;
-  const bool live = token < tokens;
-
-  // The query row: decoded codes times scale^Q, kept twice: plain (for phi) and pre-multiplied by log2(e)/sqrt(D).
-  float qv[kHeadDim];
-  {
-    const uint4* src = reinterpret_cast<const uint4*>(q_codes + (static_cast<size_t>(row_tile) * BS + t) * kHeadDim);
-    const float sq = q_scales[row_tile];
-#pragma unroll
-    for (int w = 0; w < 4; ++w) {
-      const uint4 raw = __ldg(src + w);
-      const uint32_t words[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-      for (int x = 0; x < 4; ++x) {
-        float f[4];
-        e4m3x4_to_float(words[x], f);
-#pragma unroll
-        for (int y = 0; y < 4; ++y) qv[w * 16 + x * 4 + y] = f[y] * sq;
-      }
-    }
+// ------------------------------------------------------------------------------------------------ prep
+// V code values as fp16 (exact) for the P V tensor-core product, and the largest V block scale of every head.
+__global__ void __launch_bounds__(256) prep_kernel(const uint8_t* __restrict__ v_codes, const float* __restrict__ v_scales,
+                                                   size_t words, int tiles, int nb, __half* __restrict__ v16,
+                                                   float* __restrict__ vref) {
+  const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
+  for (size_t w = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; w < words; w += stride) {
+    const uint32_t packed = __ldg(reinterpret_cast<const uint32_t*>(v_codes) + w);
+    const __half2_raw lo = __nv_cvt_fp8x2_to_halfraw2(static_cast<__nv_fp8x2_storage_t>(packed & 0xFFFFu), __NV_E4M3);
+    const __half2_raw hi = __nv_cvt_fp8x2_to_halfraw2(static_cast<__nv_fp8x2_storage_t>(packed >> 16), __NV_E4M3);
+    uint2 out;
+    out.x = static_cast<uint32_t>(lo.x) | (static_cast<uint32_t>(lo.y) << 16);
+    out.y = static_cast<uint32_t>(hi.x) | (static_cast<uint32_t>(hi.y) << 16);
+    reinterpret_cast<uint2*>(v16)[w] = out;
   }
-  const float qk_scale = kLog2e * 0.125f;  // 1/sqrt(64) in the base-2 exponent domain
-
-  float o[kHeadDim];
-#pragma unroll
-  for (int e = 0; e < kHeadDim; ++e) o[e] = 0.f;
-  float m = -INFINITY, l = 0.f;
-
-  for (int c = 0; c < k_crit; ++c) {
-    const int j = crit_idx[static_cast<size_t>(row_tile) * k_crit + c];
-    const float sk = k_scales[bh_rows + j], sv = v_scales[bh_rows + j];
-    const int valid = min(BS, tokens - j * BS);
-    const uint32_t* kc = reinterpret_cast<const uint32_t*>(k_codes + (bh_rows + j) * BS * kHeadDim);
-    const uint32_t* vc = reinterpret_cast<const uint32_t*>(v_codes + (bh_rows + j) * BS * kHeadDim);
-    __syncthreads();
-#pragma unroll 4
-    for (int w = t; w < BS * kHeadDim / 4; w += BS) {
-      float f[4];
-      e4m3x4_to_float(__ldg(kc + w), f);
-      *reinterpret_cast<float4*>(s_k + 4 * w) = make_float4(f[0] * sk, f[1] * sk, f[2] * sk, f[3] * sk);
-      e4m3x4_to_float(__ldg(vc + w), f);
-      *reinterpret_cast<float4*>(s_v + 4 * w) = make_float4(f[0] * sv, f[1] * sv, f[2] * sv, f[3] * sv);
-    }
-    __syncthreads();
-    for (int s = 0; s < valid; ++s) {
-      const float4* kr = reinterpret_cast<const float4*>(s_k + s * kHeadDim);
-      float acc = 0.f;
-#pragma unroll
-      for (int d4 = 0; d4 < kHeadDim / 4; ++d4) {
-        const float4 kk = kr[d4];
-        acc = fmaf(qv[4 * d4], kk.x, acc);
-        acc = fmaf(qv[4 * d4 + 1], kk.y, acc);
-        acc = fmaf(qv[4 * d4 + 2], kk.z, acc);
-        acc = fmaf(qv[4 * d4 + 3], kk.w, acc);
-      }
-      acc *= qk_scale;
-      if (acc > m) {
-        const float corr = exp2f(m - acc);
-        l *= corr;
-#pragma unroll
-        for (int e = 0; e < kHeadDim; ++e) o[e] *= corr;
-        m = acc;
-      }
-      const float p = exp2f(acc - m);
-      l += p;
-      const float4* vr = reinterpret_cast<const float4*>(s_v + s * kHeadDim);
-#pragma unroll
-      for (int e4 = 0; e4 < kHeadDim / 4; ++e4) {
-        const float4 vv = vr[e4];
-        o[4 * e4] = fmaf(p, vv.x, o[4 * e4]);
-        o[4 * e4 + 1] = fmaf(p, vv.y, o[4 * e4 + 1]);
-        o[4 * e4 + 2] = fmaf(p, vv.z, o[4 * e4 + 2]);
-        o[4 * e4 + 3] = fmaf(p, vv.w, o[4 * e4 + 3]);
-      }
-    }
-  }
-  if (k_crit > 0) {
-    const float inv = 1.f / l;
-#pragma unroll
-    for (int e = 0; e < kHeadDim; ++e) o[e] *= inv;
-  }
-
-  if (k_marg > 0) {
-    __syncthreads();
-    const float4* src = reinterpret_cast<const float4*>(g + static_cast<size_t>(row_tile) * kSummaryRow);
-    for (int w = t; w < kSummaryRow / 4; w += BS) reinterpret_cast<float4*>(smem_f)[w] = __ldg(src + w);
-    __syncthreads();
-    if (phi == LITE3R_PHI_SOFTMAX) {
-      float mx = qv[0];
-#pragma unroll
-      for (int d = 1; d < kHeadDim; ++d) mx = fmaxf(mx, qv[d]);
-#pragma unroll
-      for (int d = 0; d < kHeadDim; ++d) qv[d] = expf(qv[d] - mx);  // normalisation cancels in the ratio
-    } else {
-#pragma unroll
-      for (int d = 0; d < kHeadDim; ++d) qv[d] = phi_elu1(qv[d]);
-    }
-    float den = 0.f;
-    const float* zeta = smem_f + kHeadDim * kHeadDim;
-#pragma unroll
-    for (int d = 0; d < kHeadDim; ++d) den = fmaf(qv[d], zeta[d], den);
-    const float inv = 1.f / den;
-#pragma unroll
-    for (int e = 0; e < kHeadDim; ++e) {
-      const float4* gr = reinterpret_cast<const float4*>(smem_f + e * kHeadDim);
-      float num = 0.f;
-#pragma unroll
-      for (int d4 = 0; d4 < kHeadDim / 4; ++d4) {
-        const float4 gg = gr[d4];
-        num = fmaf(qv[4 * d4], gg.x, num);
-        num = fmaf(qv[4 * d4 + 1], gg.y, num);
-        num = fmaf(qv[4 * d4 + 2], gg.z, num);
-        num = fmaf(qv[4 * d4 + 3], gg.w, num);
-      }
-      o[e] = fmaf(num, inv, o[e]);
-    }
-  }
-  if (live) {
-    float4* dst = reinterpret_cast<float4*>(out + b * out_stride_b + h * out_stride_h + token * out_stride_n);
-#pragma unroll
-    for (int e4 = 0; e4 < kHeadDim / 4; ++e4) dst[e4] = make_float4(o[4 * e4], o[4 * e4 + 1], o[4 * e4 + 2], o[4 * e4 + 3]);
-  }
+  // scales are positive, so their bit patterns order like integers; max is order-independent (deterministic)
+  for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < tiles; t += static_cast<int>(stride))
+    atomicMax(reinterpret_cast<int*>(vref) + t / nb, __float_as_int(v_scales[t]));
 }
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Workspace {
+  __nv_bfloat16* hws;  // [tiles][4160]   per-key-block summaries
+  __nv_bfloat16* g16;  // [tiles][64][64] aggregated summaries, [e][d]
+  float* zeta;         // [tiles][64]
+  __half* v16;         // [tiles*Bs][64]  V code values as fp16
+  float* vref;         // [B*H]
+  size_t bytes;
+};
+
+Workspace carve(void* base, const lite3r_shape& s) {
+  const size_t tiles = static_cast<size_t>(s.batch) * s.heads * ceil_div(s.tokens, s.block);
+  char* p = static_cast<char*>(base);
+  size_t off = 0;
+  Workspace w;
+  auto take = [&](size_t bytes) {
+    char* r = p + off;
+    off += align_up(bytes, 1024);
+    return r;
+  };
+  w.hws = reinterpret_cast<__nv_bfloat16*>(take(tiles * kSummaryRow * sizeof(__nv_bfloat16)));
+  w.g16 = reinterpret_cast<__nv_bfloat16*>(take(tiles * kHeadDim * kHeadDim * sizeof(__nv_bfloat16)));
+  w.zeta = reinterpret_cast<float*>(take(tiles * kHeadDim * sizeof(float)));
+  w.v16 = reinterpret_cast<__half*>(take(tiles * s.block * kHeadDim * sizeof(__half)));
+  w.vref = reinterpret_cast<float*>(take(static_cast<size_t>(s.batch) * s.heads * sizeof(float)));
+  w.bytes = off;
+  return w;
+}
 
 template <int BS>
 lite3r_status run_forward(const ForwardArgs& a, cudaStream_t stream) {
   const lite3r_shape& s = a.s;
   const int nb = ceil_div(s.tokens, BS);
   const int rows = s.batch * s.heads * nb;
-  __nv_bfloat16* hws = static_cast<__nv_bfloat16*>(a.workspace);
-  float* g = reinterpret_cast<float*>(static_cast<char*>(a.workspace) +
-                                      align_up(static_cast<size_t>(rows) * kSummaryRow * sizeof(__nv_bfloat16), 256));
+  const Workspace w = carve(a.workspace, s);
   lite3r_status st;
+  profile_mark(0, stream);
+  if (a.plan.k_crit > 0) {
+    st = record_cuda(cudaMemsetAsync(w.vref, 0, static_cast<size_t>(s.batch) * s.heads * sizeof(float), stream));
+    if (st != LITE3R_OK) return st;
+    const size_t words = static_cast<size_t>(rows) * BS * kHeadDim / 4;
+    const int blocks = static_cast<int>(std::min<size_t>((words + 255) / 256, 148 * 16));
+    prep_kernel<<<blocks, 256, 0, stream>>>(a.v.codes, a.v.scales, words, rows, nb, w.v16, w.vref);
+    if ((st = after_launch()) != LITE3R_OK) return st;
+  }
   if (a.plan.k_marg > 0) {
     const size_t smem = (2 * BS * kHeadDim + kHeadDim * 68 + kHeadDim * kHeadDim) * sizeof(float);
     st = record_cuda(cudaFuncSetAttribute(summary_kernel<BS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           static_cast<int>(smem)));
     if (st != LITE3R_OK) return st;
-    profile_mark(0, stream);
     summary_kernel<BS><<<rows, kSumThreads, smem, stream>>>(a.k.codes, a.k.scales, a.v.codes, a.v.scales, a.proj,
-                                                            a.proj_head_stride, s.heads, s.tokens, nb, a.phi, hws);
+                                                            a.proj_head_stride, s.heads, s.tokens, nb, a.phi, w.hws);
     if ((st = after_launch()) != LITE3R_OK) return st;
     profile_mark(1, stream);
     profile_mark(2, stream);
-    aggregate_kernel<<<rows, kAggThreads, a.plan.k_marg * sizeof(int), stream>>>(hws, a.plan.marg_idx, a.plan.cls, nb,
-                                                                                   a.plan.k_marg, g);
+    aggregate_kernel<<<rows, kAggThreads, a.plan.k_marg * sizeof(int), stream>>>(w.hws, a.plan.marg_idx, a.plan.cls, nb,
+                                                                                   a.plan.k_marg, w.g16, w.zeta);
     if ((st = after_launch()) != LITE3R_OK) return st;
     profile_mark(3, stream);
   }
-  const size_t smem = align_up(2 * BS * kHeadDim * sizeof(float), 16) + 1024;
-  st = record_cuda(cudaFuncSetAttribute(attention_kernel<BS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        static_cast<int>(smem)));
-  if (st != LITE3R_OK) return st;
+  AttentionLaunch att;
+  att.shape = s;
+  att.q_codes = a.q.codes;
+  att.k_codes = a.k.codes;
+  att.q_scales = a.q.scales;
+  att.k_scales = a.k.scales;
+  att.v_scales = a.v.scales;
+  att.v16 = w.v16;
+  att.g16 = w.g16;
+  att.zeta = w.zeta;
+  att.vref = w.vref;
+  att.crit_idx = a.plan.crit_idx;
+  att.k_crit = a.plan.k_crit;
+  att.k_marg = a.plan.k_marg;
+  att.phi = a.phi;
+  att.out = a.out;
+  att.out_stride_b = a.out_stride_b;
+  att.out_stride_h = a.out_stride_h;
+  att.out_stride_n = a.out_stride_n;
+  att.device_status = a.device_status;
   profile_mark(4, stream);
-  attention_kernel<BS><<<rows, BS, smem, stream>>>(a.q.codes, a.q.scales, a.k.codes, a.k.scales, a.v.codes, a.v.scales,
-                                                   a.plan.crit_idx, g, s.heads, s.tokens, nb, a.plan.k_crit,
-                                                   a.plan.k_marg, a.phi, a.out, a.out_stride_b, a.out_stride_h,
-                                                   a.out_stride_n);
-  st = after_launch();
+  st = launch_attention(att, stream);
   profile_mark(5, stream);
   return st;
 }
@@ -359,8 +287,7 @@ lite3r_status run_forward(const ForwardArgs& a, cudaStream_t stream) {
 
 size_t forward_workspace_bytes(const lite3r_shape& s, const Counts& c) {
   (void)c;
-  const size_t rows = static_cast<size_t>(s.batch) * s.heads * ceil_div(s.tokens, s.block);
-  return align_up(rows * kSummaryRow * sizeof(__nv_bfloat16), 256) + align_up(rows * kSummaryRow * sizeof(float), 256);
+  return carve(nullptr, s).bytes;
 }
 
 lite3r_status launch_forward(const ForwardArgs& a, cudaStream_t stream) {
