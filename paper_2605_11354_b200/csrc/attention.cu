@@ -40,7 +40,7 @@ constexpr uint32_t kOffK = kOffQ + kQBytes;
 constexpr uint32_t kOffV = kOffK + kStages * kKStage;
 constexpr uint32_t kOffP = kOffV + kStages * kVStage;
 constexpr uint32_t kOffBar = kOffP + 2 * kPBuf;
-constexpr uint32_t kSmemBytes = kOffBar + 256 + 1024;  // barriers + slack for the 1024-byte alignment
+constexpr uint32_t kSmemBytes = kOffBar + 256;  // two CTAs per SM: 2 * (114944 + 1024 reserved) <= 232448
 
 struct Bars {
   uint64_t q_full, g_full, phi_full, l_full;
@@ -84,10 +84,14 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   constexpr int kM = kPair ? 64 : 128;
   constexpr uint32_t kKTx = kHalves * 4096, kVTx = kHalves * 8192;
 
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  extern __shared__ __align__(1024) uint8_t smem[];
   Bars* bars = reinterpret_cast<Bars*>(smem + kOffBar);
   volatile int* abort_flag = &bars->abort;
+  // The swizzled operand tiles need a 1024-byte aligned base; refuse to run on anything else.
+  if ((smem_u32(smem) & 1023u) != 0) {
+    if (threadIdx.x == 0 && p.status != nullptr) atomicCAS(p.status, 0, 900);
+    return;
+  }
 
   // A wait that expired in an earlier CTA of this launch stops the rest of the grid before it touches anything.
   if (p.status != nullptr && *reinterpret_cast<volatile int*>(p.status) != 0) return;
@@ -292,20 +296,22 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       tc_fence_before();
       mbar_arrive(&bars->s_empty[buf]);
 
-      float x[64];
-      float tile_max = -INFINITY;
+      float sv[64];
 #pragma unroll
       for (int k = 0; k < 32; ++k) {
-        x[k] = __uint_as_float(s_lo[k]) * c;
-        x[k + 32] = __uint_as_float(s_hi[k]) * c;
+        sv[k] = __uint_as_float(s_lo[k]);
+        sv[k + 32] = __uint_as_float(s_hi[k]);
       }
       if (valid < kStepKeys) {
 #pragma unroll
         for (int k = 0; k < 64; ++k)
-          if (k >= valid) x[k] = -INFINITY;
+          if (k >= valid) sv[k] = -INFINITY;
       }
+      // row maximum of the raw scores (c > 0 commutes with max), four independent chains
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int k = 0; k < 64; ++k) tile_max = fmaxf(tile_max, x[k]);
+      for (int k = 0; k < 64; ++k) mx4[k & 3] = fmaxf(mx4[k & 3], sv[k]);
+      const float tile_max = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * c;
 
       bool need = false;
       float alpha = 1.f;
@@ -317,16 +323,16 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         m_ref = tile_max;
         l *= alpha;
       }
-      const float shift = m_ref - __log2f(f);
-      float sum = 0.f;
+      const float neg_shift = __log2f(f) - m_ref;
+      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
       uint32_t packed[32];
 #pragma unroll
       for (int k = 0; k < 64; k += 2) {
-        const float p0 = ex2(x[k] - shift), p1 = ex2(x[k + 1] - shift);
-        sum += p0 + p1;
+        const float p0 = ex2(fmaf(sv[k], c, neg_shift)), p1 = ex2(fmaf(sv[k + 1], c, neg_shift));
+        sum4[(k >> 1) & 3] += p0 + p1;
         packed[k >> 1] = pack_half2(p0, p1);
       }
-      l += sum / f;
+      l += ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3])) / f;
 
       // P[buf] is free once the P V product of step t-2 has completed
       if (!(ok = mbar_wait(&bars->p_empty[buf], ((t >> 1) & 1) ^ 1, abort_flag, p.status, 302))) break;
@@ -455,36 +461,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 }
 
 // ------------------------------------------------------------------------------------------------ host side
-using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = [] {
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult res;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &res) != cudaSuccess ||
-        res != cudaDriverEntryPointSuccess)
-      ptr = nullptr;
-    return reinterpret_cast<EncodeTiledFn>(ptr);
-  }();
-  return fn;
-}
-
-// Row-major 2-D tensor [rows][64 elements] with a box of 64 x 64 elements.
-lite3r_status make_map(CUtensorMap* map, CUtensorMapDataType type, int elem_bytes, const void* base, uint64_t rows,
-                       CUtensorMapSwizzle swizzle) {
-  EncodeTiledFn fn = encode_fn();
-  if (fn == nullptr) return LITE3R_ERR_CUDA;
-  const cuuint64_t dims[2] = {64, rows};
-  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(64 * elem_bytes)};
-  const cuuint32_t box[2] = {64, 64};
-  const cuuint32_t estr[2] = {1, 1};
-  const CUresult r = fn(map, type, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                        swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? LITE3R_OK : LITE3R_ERR_CUDA;
-}
-
 template <int BS>
 lite3r_status launch(const AttentionLaunch& a, cudaStream_t stream) {
   const lite3r_shape& s = a.shape;
@@ -492,10 +468,10 @@ lite3r_status launch(const AttentionLaunch& a, cudaStream_t stream) {
   const uint64_t tiles = static_cast<uint64_t>(s.batch) * s.heads * nb;
   alignas(64) CUtensorMap map_q, map_k, map_v, map_g;
   lite3r_status st;
-  if ((st = make_map(&map_q, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.q_codes, tiles * BS, CU_TENSOR_MAP_SWIZZLE_64B)) != LITE3R_OK) return st;
-  if ((st = make_map(&map_k, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.k_codes, tiles * BS, CU_TENSOR_MAP_SWIZZLE_64B)) != LITE3R_OK) return st;
-  if ((st = make_map(&map_v, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, a.v16, tiles * BS, CU_TENSOR_MAP_SWIZZLE_128B)) != LITE3R_OK) return st;
-  if ((st = make_map(&map_g, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.g16, tiles * 64, CU_TENSOR_MAP_SWIZZLE_128B)) != LITE3R_OK) return st;
+  if ((st = make_tensor_map_2d(&map_q, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.q_codes, 64, tiles * BS, 64, 64, CU_TENSOR_MAP_SWIZZLE_64B)) != LITE3R_OK) return st;
+  if ((st = make_tensor_map_2d(&map_k, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.k_codes, 64, tiles * BS, 64, 64, CU_TENSOR_MAP_SWIZZLE_64B)) != LITE3R_OK) return st;
+  if ((st = make_tensor_map_2d(&map_v, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, a.v16, 64, tiles * BS, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B)) != LITE3R_OK) return st;
+  if ((st = make_tensor_map_2d(&map_g, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.g16, 64, tiles * 64, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B)) != LITE3R_OK) return st;
   AttnParams p;
   p.q_codes = a.q_codes;
   p.q_scales = a.q_scales;

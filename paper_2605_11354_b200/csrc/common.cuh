@@ -1,6 +1,7 @@
 // Shared host/device helpers of the lite3r library (internal; the public surface is include/lite3r.h).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
@@ -97,6 +98,16 @@ struct AttentionLaunch {
   int* device_status;
 };
 lite3r_status launch_attention(const AttentionLaunch& a, cudaStream_t stream);
+
+// Marginal aggregation G_i = sum over marginal j of the summary rows, as a 0/1-mask GEMM on tensor cores.
+lite3r_status launch_aggregate(const __nv_bfloat16* hws, const signed char* cls, const lite3r_shape& s, int nb,
+                               __nv_bfloat16* g16, float* zeta, int* device_status, cudaStream_t stream);
+
+// TMA descriptor of a row-major 2-D tensor [rows][inner] (row pitch = inner * elem_bytes, a multiple of 16 bytes)
+// with a box of box_inner x box_rows elements.
+lite3r_status make_tensor_map_2d(CUtensorMap* map, CUtensorMapDataType type, int elem_bytes, const void* base,
+                                 uint64_t inner, uint64_t rows, uint32_t box_inner, uint32_t box_rows,
+                                 CUtensorMapSwizzle swizzle);
 
 size_t forward_workspace_bytes(const lite3r_shape& s, const Counts& c);
 lite3r_status launch_forward(const ForwardArgs& a, cudaStream_t stream);

@@ -3,10 +3,11 @@
 //   K3  summary_kernel    per key block j:  H_j = phi(K_j)^T V_j, z_j = phi(K_j)^T 1  (lines 7-8 per block), with the
 //                         output projection folded in early: the kernel stores (H_j W)^T and z_j in bf16.  Folding
 //                         is exact algebra: (phi(q) sum_j H_j) W = phi(q) sum_j (H_j W).
-//   K3b aggregate_kernel  per query block i:  G_i = sum over marginal j of (H_j W)^T,  zeta_i = sum of z_j  (fp32).
-//   K4  attention_kernel  per query block i: online-softmax attention over the critical key blocks (lines 4-5),
+//   K3b aggregate.cu      per query block i:  G_i = sum over marginal j of (H_j W)^T,  zeta_i = sum of z_j.
+//   K4  attention.cu      per query block i: online-softmax attention over the critical key blocks (lines 4-5),
 //                         then the linear branch (line 9) phi(q) G_i / (phi(q) . zeta_i), the sum of the two
 //                         (line 10) and the store.
+//   prep_kernel           V code values as fp16 and the per-head reference V scale for the attention kernel.
 #include <algorithm>
 
 #include "common.cuh"
@@ -127,55 +128,6 @@ __global__ void __launch_bounds__(kSumThreads) summary_kernel(const uint8_t* __r
   }
 }
 
-// ------------------------------------------------------------------------------------------------ K3b
-constexpr int kAggThreads = 256;
-constexpr int kAggPer = (kSummaryRow / 2 + kAggThreads - 1) / kAggThreads;  // bf16 pairs per thread
-
-__global__ void __launch_bounds__(kAggThreads) aggregate_kernel(const __nv_bfloat16* __restrict__ hws,
-                                                                const int* __restrict__ marg_idx,
-                                                                const signed char* __restrict__ cls, int nb, int k_marg,
-                                                                __nv_bfloat16* __restrict__ g16,
-                                                                float* __restrict__ zeta) {
-  extern __shared__ int s_list[];  // [k_marg]
-  const int row = blockIdx.x;      // (b*H + h) * nb + i
-  const size_t bh_rows = static_cast<size_t>(row / nb) * nb;
-  if (marg_idx != nullptr) {
-    for (int t = threadIdx.x; t < k_marg; t += kAggThreads) s_list[t] = marg_idx[static_cast<size_t>(row) * k_marg + t];
-  } else if (threadIdx.x == 0) {  // rebuild the ascending list from the class row
-    int n = 0;
-    const signed char* c = cls + static_cast<size_t>(row) * nb;
-    for (int j = 0; j < nb; ++j)
-      if (c[j] == 1) s_list[n++] = j;
-  }
-  __syncthreads();
-  float2 acc[kAggPer];
-#pragma unroll
-  for (int x = 0; x < kAggPer; ++x) acc[x] = make_float2(0.f, 0.f);
-  for (int t = 0; t < k_marg; ++t) {
-    const __nv_bfloat162* src = reinterpret_cast<const __nv_bfloat162*>(hws + (bh_rows + s_list[t]) * kSummaryRow);
-#pragma unroll
-    for (int x = 0; x < kAggPer; ++x) {
-      const int n = threadIdx.x + x * kAggThreads;
-      if (n < kSummaryRow / 2) {
-        const float2 v = __bfloat1622float2(src[n]);
-        acc[x].x += v.x;
-        acc[x].y += v.y;
-      }
-    }
-  }
-  __nv_bfloat162* dst = reinterpret_cast<__nv_bfloat162*>(g16 + static_cast<size_t>(row) * kHeadDim * kHeadDim);
-  float2* dst_z = reinterpret_cast<float2*>(zeta + static_cast<size_t>(row) * kHeadDim);
-#pragma unroll
-  for (int x = 0; x < kAggPer; ++x) {
-    const int n = threadIdx.x + x * kAggThreads;
-    if (n < kHeadDim * kHeadDim / 2) {
-      dst[n] = __floats2bfloat162_rn(acc[x].x, acc[x].y);
-    } else if (n < kSummaryRow / 2) {
-      dst_z[n - kHeadDim * kHeadDim / 2] = acc[x];
-    }
-  }
-}
-
 // ------------------------------------------------------------------------------------------------ prep
 // V code values as fp16 (exact) for the P V tensor-core product, and the largest V block scale of every head.
 __global__ void __launch_bounds__(256) prep_kernel(const uint8_t* __restrict__ v_codes, const float* __restrict__ v_scales,
@@ -252,9 +204,7 @@ lite3r_status run_forward(const ForwardArgs& a, cudaStream_t stream) {
     if ((st = after_launch()) != LITE3R_OK) return st;
     profile_mark(1, stream);
     profile_mark(2, stream);
-    aggregate_kernel<<<rows, kAggThreads, a.plan.k_marg * sizeof(int), stream>>>(w.hws, a.plan.marg_idx, a.plan.cls, nb,
-                                                                                   a.plan.k_marg, w.g16, w.zeta);
-    if ((st = after_launch()) != LITE3R_OK) return st;
+    if ((st = launch_aggregate(w.hws, a.plan.cls, s, nb, w.g16, w.zeta, a.device_status, stream)) != LITE3R_OK) return st;
     profile_mark(3, stream);
   }
   AttentionLaunch att;
