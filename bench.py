@@ -31,9 +31,9 @@ UNIT = "TFLOP/s"
 L2_FLUSH_BYTES = 512 << 20
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 FP8_OVER_BF16 = 2.0  # nominal dense ratio (4.5 vs 2.25 PFLOP/s)
-# DRAM bytes (read + write) of one attention-kernel launch from the ncu capture summarised under profiles/;
-# None until a capture of the current kernel exists.
-ATTENTION_DRAM_BYTES_PER_LAUNCH = None
+# DRAM bytes (read + write) of one launch, keyed by (workload, kernel), from the ncu captures summarised under
+# profiles/; a kernel that changed since its capture has no entry.
+DRAM_BYTES_PER_LAUNCH = {}
 
 
 def measured_peaks():
@@ -100,6 +100,64 @@ class ClockSampler:
 
 def executed_critical_flops(wl, k_crit):
     return 4.0 * wl.batch * wl.heads * wl.n_blocks * k_crit * wl.block * wl.block * wl.head_dim
+
+
+def kernel_work(wl, plan):
+    """Algorithmic work of one launch of each kernel of the step: (bound, amount, unit of the amount).
+    HBM kernels: compulsory bytes (inputs read once + outputs written once).  Tensor kernels: executed flops."""
+    tiles = wl.batch * wl.heads * wl.n_blocks
+    elems = tiles * wl.block * wl.head_dim          # padded element count of one tensor
+    src_bytes = 2 if wl.src_dtype == "bf16" else 4
+    valid_elems = wl.batch * wl.heads * wl.tokens * wl.head_dim
+    nb = wl.n_blocks
+    return {
+        # three launches: read the source, write codes + scale + 64 column sums per tile
+        "quantize_x3": ("hbm", 3 * (valid_elems * src_bytes + elems + tiles * (4 + 256))),
+        # fp64 FMAs of the pooled scores (the selection itself is integer work on top)
+        "plan": ("alu_fp64", 2.0 * wl.batch * wl.heads * nb * nb * wl.head_dim),
+        # read V codes, write fp16 operand
+        "prep": ("hbm", elems * 3),
+        # read K and V codes, write one bf16 summary row per tile
+        "summary": ("hbm", 2 * elems + tiles * 4160 * 2),
+        # 0/1-mask GEMM over the summaries
+        "aggregation": ("tensor_bf16", 2.0 * wl.batch * wl.heads * nb * nb * 4160),
+        # QK^T and PV of every (query block, critical key block) pair
+        "attention": ("tensor_fp8", executed_critical_flops(wl, plan.k_crit)),
+    }
+
+
+def build_roofline(wl, plan, stage_ms, peaks, peak_kind):
+    """Roofline of the dominant kernel (largest share of the step) plus a per-kernel table."""
+    work = kernel_work(wl, plan)
+    hbm = peaks["hbm_gbs"]
+    bf16 = peaks["bf16_tflops"]
+    table = {}
+    for name, (bound, amount) in work.items():
+        ms = stage_ms[name]
+        if ms <= 0:
+            continue
+        if bound == "hbm":
+            ach, peak, unit, b = amount / (ms * 1e-3) / 1e9, hbm, "GB/s", "hbm"
+        elif bound == "tensor_bf16":
+            ach, peak, unit, b = amount / (ms * 1e-3) / 1e12, bf16, "TFLOP/s", "tensor"
+        elif bound == "tensor_fp8":
+            ach, peak, unit, b = amount / (ms * 1e-3) / 1e12, bf16 * FP8_OVER_BF16, "TFLOP/s", "tensor"
+        else:  # fp64 FMA pipe: 64 lanes per SM per clock, 148 SMs, at the maximum SM clock
+            ach, peak, unit, b = amount / (ms * 1e-3) / 1e12, 2 * 64 * 148 * 1.965e9 / 1e12, "TFLOP/s", "alu"
+        table[name] = {"bound": b, "ms": ms, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
+                       "work_per_launch": amount}
+    top = max(table, key=lambda n: table[n]["ms"])
+    t = table[top]
+    launches = 3 if top == "quantize_x3" else 1
+    return {"kernel": top, "bound": t["bound"], "achieved": t["achieved"], "peak": t["peak"], "unit": t["unit"],
+            "frac": t["frac"],
+            "peak_source": (f"{peak_kind} HBM copy" if t["bound"] == "hbm" else
+                            f"{peak_kind} bf16 burst x {FP8_OVER_BF16:g} (nominal fp8/bf16 ratio; no fp8 figure measured)"
+                            if top == "attention" else f"{peak_kind} bf16 burst" if t["bound"] == "tensor" else
+                            "64 fp64 FMA lanes x 148 SMs x 1.965 GHz"),
+            "traffic": DRAM_BYTES_PER_LAUNCH.get((wl.name, top)),
+            "work_per_launch": t["work_per_launch"] / launches, "avg_launch_ms": t["ms"] / launches,
+            "stage_ms": stage_ms, "kernels": table}
 
 
 # ------------------------------------------------------------------------------------------------ CPU oracle timing
@@ -238,22 +296,33 @@ def run_ours(args, wl):
     clocks = sampler.stop()
     assert int(eng.status.item()) == 0
 
+    # Per-kernel breakdown (outside the timed region, L2 flushed before each sample): quantiser and plan with CUDA
+    # events on the launching stream, the forward's four stages from the library's own event marks.
+    def sample(fn, reps):
+        acc = 0.0
+        for _ in range(reps):
+            flush.fill_(1)
+            start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            start.record()
+            fn()
+            end.record()
+            end.synchronize()
+            acc += start.elapsed_time(end)
+        return acc / reps
+
+    reps = max(3, min(args.steps, 10))
+    quant_ms = sample(lambda: eng.quantize(dev["q"], dev["k"], dev["v"]), reps)
+    plan_ms = sample(eng.make_plan, reps)
+
     flops = wl.dense_equiv_flops
     value_flops, worst_s = pdist.aggregate_throughput(flops * args.steps, ms_total / 1e3, device)
     e2e_flops, _ = pdist.aggregate_throughput(flops * args.steps, e2e_total / 1e3, device)
 
     peaks, peak_kind = measured_peaks()
-    att_ms = statistics.mean(s[2] for s in stages)
-    crit_flops = executed_critical_flops(wl, eng.plan.k_crit)
-    achieved = crit_flops / (att_ms * 1e-3) / 1e12 if att_ms > 0 else 0.0
-    fp8_peak = peaks["bf16_tflops"] * FP8_OVER_BF16
-    roofline = {"kernel": "attention (critical-block softmax + linear branch + projection)", "bound": "tensor",
-                "achieved": achieved, "peak": fp8_peak, "unit": "TFLOP/s", "frac": achieved / fp8_peak,
-                "peak_source": f"2 x {peak_kind} bf16 burst (no fp8 figure measured; nominal fp8/bf16 ratio)",
-                "traffic": ATTENTION_DRAM_BYTES_PER_LAUNCH, "flops_per_launch": crit_flops,
-                "avg_launch_ms": att_ms,
-                "stage_ms": {"summary": statistics.mean(s[0] for s in stages),
-                             "aggregation": statistics.mean(s[1] for s in stages), "attention": att_ms}}
+    stage = {"quantize_x3": quant_ms, "plan": plan_ms,
+             "prep": statistics.mean(s[0] for s in stages), "summary": statistics.mean(s[1] for s in stages),
+             "aggregation": statistics.mean(s[2] for s in stages), "attention": statistics.mean(s[3] for s in stages)}
+    roofline = build_roofline(wl, eng.plan, stage, peaks, peak_kind)
 
     if rank != 0:
         pdist.shutdown()

@@ -164,10 +164,11 @@ LITE3R_API const char* lite3r_status_string(lite3r_status status);
 LITE3R_API int lite3r_last_cuda_error(void);
 
 /* Stage timing for benchmarks.  After lite3r_profile_enable(1) (call it with the device current; it creates CUDA
- * events, no device memory), every lite3r_sla_forward brackets its three stages -- key-block summaries, marginal
- * aggregation, attention -- with event records on the call's stream.  lite3r_profile_stage_ms waits for the last
- * forward's events (the only blocking call of the library) and writes the three durations in milliseconds to
- * ms (HOST, 3 floats; a stage that did not run reports 0).  Not thread-safe; meant for one benchmarking thread. */
+ * events, no device memory), every lite3r_sla_forward brackets its four stages -- V operand preparation, key-block
+ * summaries, marginal aggregation, attention -- with event records on the call's stream.  lite3r_profile_stage_ms
+ * waits for the last forward's events (the only blocking call of the library) and writes the four durations in
+ * milliseconds to ms (HOST, 4 floats; a stage that did not run reports 0).  Not thread-safe; meant for one
+ * benchmarking thread. */
 LITE3R_API lite3r_status lite3r_profile_enable(int enable);
 LITE3R_API lite3r_status lite3r_profile_stage_ms(float* ms);
 

@@ -109,8 +109,8 @@ def profile_enable(on: bool) -> None:
 
 
 def profile_stage_ms():
-    """(summary, aggregation, attention) milliseconds of the last forward; blocks until it has finished."""
-    ms = (C.c_float * 3)()
+    """(prep, summary, aggregation, attention) milliseconds of the last forward; blocks until it has finished."""
+    ms = (C.c_float * 4)()
     _check(lib().lite3r_profile_stage_ms(ms), "lite3r_profile_stage_ms")
     return tuple(float(x) for x in ms)
 

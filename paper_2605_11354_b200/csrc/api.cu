@@ -20,9 +20,16 @@ lite3r_status after_launch() {
   return record_cuda(cudaGetLastError());
 }
 
+lite3r_status sm_count(int* count) {
+  int device = 0;
+  lite3r_status st = record_cuda(cudaGetDevice(&device));
+  if (st != LITE3R_OK) return st;
+  return record_cuda(cudaDeviceGetAttribute(count, cudaDevAttrMultiProcessorCount, device));
+}
+
 static bool g_profile = false;
-static cudaEvent_t g_events[6] = {};
-static bool g_marked[6] = {};
+static cudaEvent_t g_events[8] = {};
+static bool g_marked[8] = {};
 
 void profile_mark(int idx, cudaStream_t stream) {
   if (!g_profile) return;
@@ -237,7 +244,7 @@ lite3r_status lite3r_profile_enable(int enable) {
 
 lite3r_status lite3r_profile_stage_ms(float* ms) {
   if (ms == nullptr || !g_profile) return LITE3R_ERR_INVALID_ARG;
-  for (int s = 0; s < 3; ++s) {
+  for (int s = 0; s < 4; ++s) {
     ms[s] = 0.f;
     if (g_marked[2 * s] && g_marked[2 * s + 1]) {
       lite3r_status st = record_cuda(cudaEventSynchronize(g_events[2 * s + 1]));

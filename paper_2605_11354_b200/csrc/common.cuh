@@ -21,8 +21,12 @@ lite3r_status record_cuda(cudaError_t err);
 // Counts one enqueued kernel launch and returns the launch's error state as a status.
 lite3r_status after_launch();
 
-// Benchmark stage timing: records event `idx` (0..5) on `stream` when profiling is enabled.
+// Benchmark stage timing: records event `idx` (0..7; stage s runs from event 2s to 2s+1) on `stream` when
+// profiling is enabled.
 void profile_mark(int idx, cudaStream_t stream);
+
+// Number of SMs of the current device.
+lite3r_status sm_count(int* count);
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
@@ -98,6 +102,11 @@ struct AttentionLaunch {
   int* device_status;
 };
 lite3r_status launch_attention(const AttentionLaunch& a, cudaStream_t stream);
+
+// Per-key-block summaries ((H_j W)^T | z_j) in bf16, one kSummaryRow-wide row per (b, h, key block).
+lite3r_status launch_summary(const lite3r_fp8& k, const lite3r_fp8& v, const float* proj, long long proj_head_stride,
+                             const lite3r_shape& s, int phi, __nv_bfloat16* hws, int* device_status,
+                             cudaStream_t stream);
 
 // Marginal aggregation G_i = sum over marginal j of the summary rows, as a 0/1-mask GEMM on tensor cores.
 lite3r_status launch_aggregate(const __nv_bfloat16* hws, const signed char* cls, const lite3r_shape& s, int nb,

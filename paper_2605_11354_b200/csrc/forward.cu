@@ -1,8 +1,7 @@
 // K3 / K3b / K4: the SLA forward for a given block plan (Eq. 1; Algorithm 1 lines 4-10).
 //
-//   K3  summary_kernel    per key block j:  H_j = phi(K_j)^T V_j, z_j = phi(K_j)^T 1  (lines 7-8 per block), with the
-//                         output projection folded in early: the kernel stores (H_j W)^T and z_j in bf16.  Folding
-//                         is exact algebra: (phi(q) sum_j H_j) W = phi(q) sum_j (H_j W).
+//   K3  summary.cu        per key block j:  H_j = phi(K_j)^T V_j, z_j = phi(K_j)^T 1  (lines 7-8 per block), stored as
+//                         (H_j W)^T and z_j in bf16 (output projection folded in early).
 //   K3b aggregate.cu      per query block i:  G_i = sum over marginal j of (H_j W)^T,  zeta_i = sum of z_j.
 //   K4  attention.cu      per query block i: online-softmax attention over the critical key blocks (lines 4-5),
 //                         then the linear branch (line 9) phi(q) G_i / (phi(q) . zeta_i), the sum of the two
@@ -15,118 +14,6 @@
 namespace lite3r {
 
 namespace {
-
-constexpr float kLog2e = 1.4426950408889634f;
-
-__device__ __forceinline__ float phi_elu1(float x) { return x > 0.f ? x + 1.f : expf(x); }
-
-// ------------------------------------------------------------------------------------------------ K3
-constexpr int kSumThreads = 256;
-
-template <int BS>
-__global__ void __launch_bounds__(kSumThreads) summary_kernel(const uint8_t* __restrict__ k_codes,
-                                                              const float* __restrict__ k_scales,
-                                                              const uint8_t* __restrict__ v_codes,
-                                                              const float* __restrict__ v_scales,
-                                                              const float* __restrict__ proj,
-                                                              long long proj_head_stride, int heads, int tokens, int nb,
-                                                              int phi, __nv_bfloat16* __restrict__ hws) {
-  extern __shared__ __align__(16) float smem_f[];
-  float* s_phi = smem_f;                 // [BS][64]
-  float* s_v = s_phi + BS * kHeadDim;    // [BS][64]
-  float* s_h = s_v + BS * kHeadDim;      // [64][68]
-  float* s_w = s_h + kHeadDim * 68;      // [64][64]
-
-  const int tile = blockIdx.x;  // (b*H + h) * nb + j
-  const int j = tile % nb;
-  const int h = (tile / nb) % heads;
-  const int valid = min(BS, tokens - j * BS);
-  const float sk = k_scales[tile];
-  const float sv = v_scales[tile];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-  const uint8_t* kc = k_codes + static_cast<size_t>(tile) * BS * kHeadDim;
-  const uint8_t* vc = v_codes + static_cast<size_t>(tile) * BS * kHeadDim;
-  for (int r = warp; r < BS; r += kSumThreads / 32) {
-    float p0 = 0.f, p1 = 0.f;
-    if (r < valid) {
-      const uint32_t two = *reinterpret_cast<const uint16_t*>(kc + r * kHeadDim + 2 * lane);
-      float x[4];
-      e4m3x4_to_float(two, x);
-      const float x0 = x[0] * sk, x1 = x[1] * sk;
-      if (phi == LITE3R_PHI_SOFTMAX) {
-        const float m = warp_max(fmaxf(x0, x1));
-        const float e0 = expf(x0 - m), e1 = expf(x1 - m);
-        const float inv = 1.f / warp_sum(e0 + e1);
-        p0 = e0 * inv;
-        p1 = e1 * inv;
-      } else {
-        p0 = phi_elu1(x0);
-        p1 = phi_elu1(x1);
-      }
-    }
-    *reinterpret_cast<float2*>(s_phi + r * kHeadDim + 2 * lane) = make_float2(p0, p1);
-  }
-  for (int w = threadIdx.x; w < BS * kHeadDim / 4; w += kSumThreads) {
-    float x[4];
-    e4m3x4_to_float(*reinterpret_cast<const uint32_t*>(vc + 4 * w), x);
-    *reinterpret_cast<float4*>(s_v + 4 * w) = make_float4(x[0] * sv, x[1] * sv, x[2] * sv, x[3] * sv);
-  }
-  const float* w_h = proj + h * proj_head_stride;
-  for (int w = threadIdx.x; w < kHeadDim * kHeadDim / 4; w += kSumThreads) {
-    *reinterpret_cast<float4*>(s_w + 4 * w) = __ldg(reinterpret_cast<const float4*>(w_h) + w);
-  }
-  __syncthreads();
-
-  const int d0 = (threadIdx.x >> 4) * 4, e0 = (threadIdx.x & 15) * 4;
-  float acc[4][4] = {};
-  float z[4] = {};
-  for (int s = 0; s < valid; ++s) {
-    const float4 a = *reinterpret_cast<const float4*>(s_phi + s * kHeadDim + d0);
-    const float4 b = *reinterpret_cast<const float4*>(s_v + s * kHeadDim + e0);
-    const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-    for (int x = 0; x < 4; ++x) {
-      z[x] += av[x];
-#pragma unroll
-      for (int y = 0; y < 4; ++y) acc[x][y] = fmaf(av[x], bv[y], acc[x][y]);
-    }
-  }
-#pragma unroll
-  for (int x = 0; x < 4; ++x)
-    *reinterpret_cast<float4*>(s_h + (d0 + x) * 68 + e0) = make_float4(acc[x][0], acc[x][1], acc[x][2], acc[x][3]);
-  __syncthreads();
-
-  float out[4][4] = {};
-  for (int f = 0; f < kHeadDim; ++f) {
-    const float4 b = *reinterpret_cast<const float4*>(s_w + f * kHeadDim + e0);
-    const float bv[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-    for (int x = 0; x < 4; ++x) {
-      const float a = s_h[(d0 + x) * 68 + f];
-#pragma unroll
-      for (int y = 0; y < 4; ++y) out[x][y] = fmaf(a, bv[y], out[x][y]);
-    }
-  }
-  __nv_bfloat16* dst = hws + static_cast<size_t>(tile) * kSummaryRow;
-#pragma unroll
-  for (int y = 0; y < 4; ++y) {  // row e0+y of (H W)^T holds d0..d0+3 contiguously
-    __nv_bfloat162 lo = __floats2bfloat162_rn(out[0][y], out[1][y]);
-    __nv_bfloat162 hi = __floats2bfloat162_rn(out[2][y], out[3][y]);
-    uint2 pk;
-    pk.x = *reinterpret_cast<uint32_t*>(&lo);
-    pk.y = *reinterpret_cast<uint32_t*>(&hi);
-    *reinterpret_cast<uint2*>(dst + (e0 + y) * kHeadDim + d0) = pk;
-  }
-  if ((threadIdx.x & 15) == 0) {
-    __nv_bfloat162 lo = __floats2bfloat162_rn(z[0], z[1]);
-    __nv_bfloat162 hi = __floats2bfloat162_rn(z[2], z[3]);
-    uint2 pk;
-    pk.x = *reinterpret_cast<uint32_t*>(&lo);
-    pk.y = *reinterpret_cast<uint32_t*>(&hi);
-    *reinterpret_cast<uint2*>(dst + kHeadDim * kHeadDim + d0) = pk;
-  }
-}
 
 // ------------------------------------------------------------------------------------------------ prep
 // V code values as fp16 (exact) for the P V tensor-core product, and the largest V block scale of every head.
@@ -193,19 +80,16 @@ lite3r_status run_forward(const ForwardArgs& a, cudaStream_t stream) {
     const int blocks = static_cast<int>(std::min<size_t>((words + 255) / 256, 148 * 16));
     prep_kernel<<<blocks, 256, 0, stream>>>(a.v.codes, a.v.scales, words, rows, nb, w.v16, w.vref);
     if ((st = after_launch()) != LITE3R_OK) return st;
+    profile_mark(1, stream);
   }
   if (a.plan.k_marg > 0) {
-    const size_t smem = (2 * BS * kHeadDim + kHeadDim * 68 + kHeadDim * kHeadDim) * sizeof(float);
-    st = record_cuda(cudaFuncSetAttribute(summary_kernel<BS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          static_cast<int>(smem)));
-    if (st != LITE3R_OK) return st;
-    summary_kernel<BS><<<rows, kSumThreads, smem, stream>>>(a.k.codes, a.k.scales, a.v.codes, a.v.scales, a.proj,
-                                                            a.proj_head_stride, s.heads, s.tokens, nb, a.phi, w.hws);
-    if ((st = after_launch()) != LITE3R_OK) return st;
-    profile_mark(1, stream);
     profile_mark(2, stream);
-    if ((st = launch_aggregate(w.hws, a.plan.cls, s, nb, w.g16, w.zeta, a.device_status, stream)) != LITE3R_OK) return st;
+    st = launch_summary(a.k, a.v, a.proj, a.proj_head_stride, s, a.phi, w.hws, a.device_status, stream);
+    if (st != LITE3R_OK) return st;
     profile_mark(3, stream);
+    profile_mark(4, stream);
+    if ((st = launch_aggregate(w.hws, a.plan.cls, s, nb, w.g16, w.zeta, a.device_status, stream)) != LITE3R_OK) return st;
+    profile_mark(5, stream);
   }
   AttentionLaunch att;
   att.shape = s;
@@ -227,9 +111,9 @@ lite3r_status run_forward(const ForwardArgs& a, cudaStream_t stream) {
   att.out_stride_h = a.out_stride_h;
   att.out_stride_n = a.out_stride_n;
   att.device_status = a.device_status;
-  profile_mark(4, stream);
+  profile_mark(6, stream);
   st = launch_attention(att, stream);
-  profile_mark(5, stream);
+  profile_mark(7, stream);
   return st;
 }
 
