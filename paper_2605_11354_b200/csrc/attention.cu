@@ -3,18 +3,22 @@
 // One CTA owns 128 query rows of one (b, h): at block 64 a PAIR of query blocks (two M=64 accumulators interleaved
 // in the two 16-lane halves of every TMEM sub-partition), at block 128 one query block (M=128).  Work advances in
 // steps of 64 keys.  Per step t:
-//   TMA      K tile(s) (e4m3, 64-byte rows, 64B swizzle) and V tile(s) (code values as fp16, 128B swizzle) -> smem ring
+//   TMA      K tile(s) (e4m3, 64-byte rows, 64B swizzle) and V tile(s) (dequantised fp16, 128B swizzle) -> smem ring
 //   tcgen05  S[t&1] = Q K^T        kind::f8f6f4, fp32 accumulators in TMEM (64 columns)
-//   softmax  128 threads, one query row each (TMEM lane = thread): scale, mask padded keys, running max with lazy
-//            rescale, exp2, row sum; P goes to shared memory as fp16 in the MMA's K-major 128B-swizzled layout
+//   softmax  256 threads, two per query row (TMEM lane = thread, 32 of the 64 columns each): scale, mask padded
+//            keys, running max with lazy rescale, exp2, row sum; P goes to shared memory as fp16 in the MMA's
+//            K-major 128B-swizzled layout.  Both threads of a row read all 64 scores for the maximum, so they
+//            take identical rescale decisions without exchanging anything; only the exponentials are split.
 //   tcgen05  O += P V              kind::f16, V as MN-major B operand, fp32 accumulators in TMEM (64 columns)
 // P is carried in fp16 (not e4m3): one e4m3 term has a 2.6 % rounding error per probability, which alone is ten
-// times the output tolerance; V's code values are exact in fp16, and the V block scale rides on P
-// (P' = P * scale_j / scale_ref, row sums corrected by the inverse), so O needs one final scale.
+// times the output tolerance.  V travels as the dequantised value in fp16 (2^-12 relative rounding).
 // Tail: phi(Q) (bf16) times the aggregated, projected summaries G_i (bf16) as one more MMA, divided by
-// phi(Q) . zeta_i, added to O / l and stored.
+// phi(Q) . zeta_i, added to O / l and stored; the two threads of a row swap their partial row sums once.
 //
-// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner, warps 2-5 = softmax/epilogue.
+// Warp roles (352 threads): warp 0 = TMA producer, warp 1 = Q K^T issuer and TMEM owner, warp 2 = P V issuer (and the
+// linear-branch MMA), warps 3-10 = softmax/epilogue.  A single thread can issue one small tcgen05.mma roughly every
+// 50 clocks, so the two products have an issuing thread each; "product t done" is one barrier per product (rings of
+// six, committed once) on which both the softmax threads and the TMA producer wait.
 // Every mbarrier wait is bounded (1 s); on expiry the CTA sets *device_status and all roles leave their loops.
 #include "common.cuh"
 #include "sm100.cuh"
@@ -26,12 +30,17 @@ namespace {
 using namespace sm100;
 
 constexpr int kStages = 3;
-constexpr int kThreads = 192;
+constexpr int kSoftmaxThreads = 256;
+constexpr int kCtrlWarps = 3;
+constexpr int kThreads = kCtrlWarps * 32 + kSoftmaxThreads;
+constexpr uint32_t kBackoffNs = 100;  // sleep between polls of the single-thread roles
+constexpr int kRing = 6;  // lcm of the S/P double buffers and the three K/V stages
 constexpr int kStepKeys = 64;
 constexpr uint32_t kTmemCols = 256;
 constexpr uint32_t kColS = 0, kColO = 128, kColL = 192;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRescaleThreshold = 8.0f;  // lazy rescale: keep the old reference max until it is beaten by 2^8
+constexpr uint32_t kOffX = 8192;           // row-sum exchange of the epilogue: reuses K stage 0 (2 KB)
 
 // shared-memory map (bytes from a 1024-aligned base)
 constexpr uint32_t kQBytes = 8192, kKStage = 8192, kVStage = 16384, kPBuf = 16384;
@@ -43,9 +52,10 @@ constexpr uint32_t kOffBar = kOffP + 2 * kPBuf;
 constexpr uint32_t kSmemBytes = kOffBar + 256;  // two CTAs per SM: 2 * (114944 + 1024 reserved) <= 232448
 
 struct Bars {
-  uint64_t q_full, g_full, phi_full, l_full;
-  uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
-  uint64_t s_full[2], s_empty[2], p_full[2], p_empty[2];
+  uint64_t q_full, g_full, phi_full, l_full, x_full;
+  uint64_t k_full[kStages], v_full[kStages];  // TMA -> issuers
+  uint64_t qk_done[kRing], pv_done[kRing];    // product of step t complete: barrier t % 6, phase (t / 6)
+  uint64_t s_empty[2], p_full[2];             // softmax -> issuers
   uint32_t tmem_base;
   int abort;
 };
@@ -55,7 +65,6 @@ struct AttnParams {
   const float* q_scales;
   const float* k_scales;
   const float* v_scales;
-  const float* vref;   // [B*H] largest V block scale of the head
   const int* crit_idx; // [B*H*Nb][k_crit]
   const float* zeta;   // [B*H*Nb][64]
   float* out;
@@ -67,6 +76,11 @@ struct AttnParams {
 __device__ __forceinline__ uint32_t pack_half2(float a, float b) {
   __half2 h = __floats2half2_rn(a, b);
   return *reinterpret_cast<uint32_t*>(&h);
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
 }
 __device__ __forceinline__ uint32_t pack_bf162(float a, float b) {
   __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
@@ -107,19 +121,20 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   if (threadIdx.x == 0) {
     mbar_init(&bars->q_full, 1);
     mbar_init(&bars->g_full, 1);
-    mbar_init(&bars->phi_full, 128);
+    mbar_init(&bars->phi_full, kSoftmaxThreads);
     mbar_init(&bars->l_full, 1);
+    mbar_init(&bars->x_full, kSoftmaxThreads);
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&bars->k_full[s], 1);
-      mbar_init(&bars->k_empty[s], 1);
       mbar_init(&bars->v_full[s], 1);
-      mbar_init(&bars->v_empty[s], 1);
+    }
+    for (int r = 0; r < kRing; ++r) {
+      mbar_init(&bars->qk_done[r], 1);
+      mbar_init(&bars->pv_done[r], 1);
     }
     for (int b = 0; b < 2; ++b) {
-      mbar_init(&bars->s_full[b], 1);
-      mbar_init(&bars->s_empty[b], 128);
-      mbar_init(&bars->p_full[b], 128);
-      mbar_init(&bars->p_empty[b], 1);
+      mbar_init(&bars->s_empty[b], kSoftmaxThreads);
+      mbar_init(&bars->p_full[b], kSoftmaxThreads);
     }
     bars->abort = 0;
     mbar_fence_init();
@@ -152,7 +167,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       bool ok = true;
       for (int t = 0; t < steps && ok; ++t) {
         const int st = t % kStages;
-        const uint32_t par = ((t / kStages) & 1) ^ 1;
         int row[2];
         if (kPair) {
           row[0] = static_cast<int>((bh_rows + __ldg(list0 + t)) * 64);
@@ -161,13 +175,13 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           row[0] = static_cast<int>((bh_rows + __ldg(list0 + t / 2)) * 128 + (t & 1) * 64);
           row[1] = 0;
         }
-        ok = mbar_wait(&bars->k_empty[st], par, abort_flag, p.status, 101);
-        if (!ok) break;
+        // stage st was last used by step t-3: its K tile is free after that step's Q K^T, its V tile after its P V
+        const int u = t - kStages;
+        if (u >= 0 && !(ok = mbar_wait(&bars->qk_done[u % kRing], (u / kRing) & 1, abort_flag, p.status, 101, kBackoffNs))) break;
         mbar_arrive_expect_tx(&bars->k_full[st], kKTx);
         for (int hf = 0; hf < kHalves; ++hf)
           tma_load_2d(smem + kOffK + st * kKStage + hf * 4096, &map_k, &bars->k_full[st], 0, row[hf]);
-        ok = mbar_wait(&bars->v_empty[st], par, abort_flag, p.status, 102);
-        if (!ok) break;
+        if (u >= 0 && !(ok = mbar_wait(&bars->pv_done[u % kRing], (u / kRing) & 1, abort_flag, p.status, 102, kBackoffNs))) break;
         mbar_arrive_expect_tx(&bars->v_full[st], kVTx);
         for (int hf = 0; hf < kHalves; ++hf)
           tma_load_2d(smem + kOffV + st * kVStage + hf * 8192, &map_v, &bars->v_full[st], 0, row[hf]);
@@ -176,7 +190,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         // The aggregated summaries reuse V stage 0; it is free once the last P V product has completed.
         if (steps > 0) {
           const int last = steps - 1;
-          ok = mbar_wait(&bars->v_empty[last % kStages], (last / kStages) & 1, abort_flag, p.status, 103);
+          ok = mbar_wait(&bars->pv_done[last % kRing], (last / kRing) & 1, abort_flag, p.status, 103);
         }
         if (ok) {
           mbar_arrive_expect_tx(&bars->g_full, kHalves * 8192);
@@ -186,61 +200,65 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------------------------------ MMA issuer
+    // ------------------------------------------------------------------------------------------ Q K^T issuer
     if (lane == 0) {
       constexpr uint32_t idesc_qk = instr_desc(0, kM, 64, 0, 0);   // e4m3 x e4m3, both K-major
-      constexpr uint32_t idesc_pv = instr_desc(0, kM, 64, 0, 1);   // f16 x f16, V MN-major
-      constexpr uint32_t idesc_lin = instr_desc(1, kM, 64, 0, 0);  // bf16 x bf16, both K-major
       const uint32_t q_addr = smem_u32(smem + kOffQ), k_addr = smem_u32(smem + kOffK);
-      const uint32_t v_addr = smem_u32(smem + kOffV), p_addr = smem_u32(smem + kOffP);
       bool ok = mbar_wait(&bars->q_full, 0, abort_flag, p.status, 201);
-      auto issue_qk = [&](int t) {
+      // Gated only by the K tile and by the softmax threads having pulled S(t-2) into registers, so this runs up
+      // to two steps ahead of the softmax.
+      for (int t = 0; t < steps && ok; ++t) {
         const int st = t % kStages, buf = t & 1;
-        if (!mbar_wait(&bars->k_full[st], (t / kStages) & 1, abort_flag, p.status, 202)) return false;
-        if (!mbar_wait(&bars->s_empty[buf], ((t >> 1) & 1) ^ 1, abort_flag, p.status, 203)) return false;
+        if (!(ok = mbar_wait(&bars->k_full[st], (t / kStages) & 1, abort_flag, p.status, 202, kBackoffNs))) break;
+        if (!(ok = mbar_wait(&bars->s_empty[buf], ((t >> 1) & 1) ^ 1, abort_flag, p.status, 203, kBackoffNs))) break;
         tc_fence_after();
-        for (int hf = 0; hf < kHalves; ++hf) {
-          const uint32_t d = tmem + kColS + buf * 64 + ((hf * 16u) << 16);
-          for (int kk = 0; kk < 2; ++kk) {
+#pragma unroll
+        for (int kk = 0; kk < 2; ++kk) {
+#pragma unroll
+          for (int hf = 0; hf < kHalves; ++hf) {
+            const uint32_t d = tmem + kColS + buf * 64 + ((hf * 16u) << 16);
             const uint64_t a = smem_desc(q_addr + (kPair ? hf * 4096 : 0) + kk * 32, 16, 512, kSwizzle64);
             const uint64_t b = smem_desc(k_addr + st * kKStage + hf * 4096 + kk * 32, 16, 512, kSwizzle64);
             mma_f8(d, a, b, idesc_qk, kk);
           }
         }
-        mma_commit(&bars->k_empty[st]);
-        mma_commit(&bars->s_full[buf]);
-        return true;
-      };
-      auto issue_pv = [&](int t) {
+        mma_commit(&bars->qk_done[t % kRing]);
+      }
+    }
+  } else if (warp == 2) {
+    // ------------------------------------------------------------------------------------------ P V issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_pv = instr_desc(0, kM, 64, 0, 1);   // f16 x f16, V MN-major
+      constexpr uint32_t idesc_lin = instr_desc(1, kM, 64, 0, 0);  // bf16 x bf16, both K-major
+      const uint32_t v_addr = smem_u32(smem + kOffV), p_addr = smem_u32(smem + kOffP);
+      bool ok = true;
+      for (int t = 0; t < steps && ok; ++t) {
         const int st = t % kStages, buf = t & 1;
-        if (!mbar_wait(&bars->v_full[st], (t / kStages) & 1, abort_flag, p.status, 204)) return false;
-        if (!mbar_wait(&bars->p_full[buf], (t >> 1) & 1, abort_flag, p.status, 205)) return false;
+        if (!(ok = mbar_wait(&bars->v_full[st], (t / kStages) & 1, abort_flag, p.status, 204, kBackoffNs))) break;
+        if (!(ok = mbar_wait(&bars->p_full[buf], (t >> 1) & 1, abort_flag, p.status, 205, kBackoffNs))) break;
         tc_fence_after();
-        for (int hf = 0; hf < kHalves; ++hf) {
-          const uint32_t d = tmem + kColO + ((hf * 16u) << 16);
-          for (int kk = 0; kk < 4; ++kk) {
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+#pragma unroll
+          for (int hf = 0; hf < kHalves; ++hf) {
+            const uint32_t d = tmem + kColO + ((hf * 16u) << 16);
             const uint64_t a = smem_desc(p_addr + buf * kPBuf + (kPair ? hf * 8192 : 0) + kk * 32, 16, 1024, kSwizzle128);
             const uint64_t b = smem_desc(v_addr + st * kVStage + hf * 8192 + kk * 2048, 8192, 1024, kSwizzle128);
             mma_f16(d, a, b, idesc_pv, (t > 0 || kk > 0) ? 1u : 0u);
           }
         }
-        mma_commit(&bars->v_empty[st]);
-        mma_commit(&bars->p_empty[buf]);
-        return true;
-      };
-      for (int t = 0; t < steps && ok; ++t) {
-        ok = issue_qk(t);
-        if (ok && t > 0) ok = issue_pv(t - 1);
+        mma_commit(&bars->pv_done[t % kRing]);
       }
-      if (ok && steps > 0) ok = issue_pv(steps - 1);
       if (ok && p.k_marg > 0) {
         ok = mbar_wait(&bars->g_full, 0, abort_flag, p.status, 206) &&
              mbar_wait(&bars->phi_full, 0, abort_flag, p.status, 207);
         if (ok) {
           tc_fence_after();
-          for (int hf = 0; hf < kHalves; ++hf) {
-            const uint32_t d = tmem + kColL + ((hf * 16u) << 16);
-            for (int kk = 0; kk < 4; ++kk) {
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) {
+#pragma unroll
+            for (int hf = 0; hf < kHalves; ++hf) {
+              const uint32_t d = tmem + kColL + ((hf * 16u) << 16);
               const uint64_t a = smem_desc(p_addr + (kPair ? hf * 8192 : 0) + kk * 32, 16, 1024, kSwizzle128);
               const uint64_t b = smem_desc(v_addr + hf * 8192 + kk * 32, 16, 1024, kSwizzle128);
               mma_f16(d, a, b, idesc_lin, kk);
@@ -253,6 +271,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   } else {
     // ------------------------------------------------------------------------------------------ softmax + epilogue
     const int quarter = warp & 3;                       // TMEM sub-partition this warp may touch
+    const int ch = (warp - kCtrlWarps) >> 2;            // which 32 of the 64 columns this thread exponentiates
     const int hf = kPair ? (lane >> 4) : 0;             // which query block of the pair this thread serves
     const int row_in_block = kPair ? quarter * 16 + (lane & 15) : quarter * 32 + lane;
     const int p_row = kPair ? hf * 64 + row_in_block : row_in_block;  // row inside the P / phi tile
@@ -261,102 +280,113 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const uint32_t lane_addr = tmem + ((static_cast<uint32_t>(quarter) * 32u) << 16);
     const int token = iq * BS + row_in_block;
     const float sq = __ldg(p.q_scales + q_tile);
-    const float vref = __ldg(p.vref + bh);
     const float qk_scale = sq * (kLog2e * 0.125f);
     const int* list = p.crit_idx + q_tile * p.k_crit;
-    uint8_t* p_tile = smem + kOffP;
+    // this thread's four 16-byte chunks of its 128-byte P / phi row (128B swizzle)
+    uint8_t* const prow = smem + kOffP + p_row * 128;
+    uint32_t chunk_off[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) chunk_off[i] = static_cast<uint32_t>(((ch * 4 + i) ^ (p_row & 7)) << 4);
 
-    float m_ref = -1.0e30f, l = 0.f;
+    float m_ref = -1.0e30f, l = 0.f;  // l: sum over this thread's 32 columns
     bool ok = true;
 
-    // per-step scalars, fetched one step ahead
-    int j_next = steps > 0 ? __ldg(list) : 0;
-    float sk_next = steps > 0 ? __ldg(p.k_scales + bh_rows + j_next) : 0.f;
-    float sv_next = steps > 0 ? __ldg(p.v_scales + bh_rows + j_next) : 1.f;
+    // per-step scalars: the key-block index is fetched two steps ahead and its scale one step ahead, so that no
+    // load in the loop waits for the address produced by another load of the same iteration
+    int j_cur = steps > 0 ? __ldg(list) : 0;
+    int j_nxt = steps > 1 ? __ldg(list + 1 / kStepsPerBlock) : 0;
+    float sk_cur = steps > 0 ? __ldg(p.k_scales + bh_rows + j_cur) : 0.f;
 
     for (int t = 0; t < steps; ++t) {
       const int buf = t & 1;
-      const int j = j_next;
-      const float c = qk_scale * sk_next;
-      const float f = sv_next / vref;
-      if (t + 1 < steps) {
-        j_next = __ldg(list + (t + 1) / kStepsPerBlock);
-        sk_next = __ldg(p.k_scales + bh_rows + j_next);
-        sv_next = __ldg(p.v_scales + bh_rows + j_next);
-      }
+      const int j = j_cur;
+      const float c = qk_scale * sk_cur;
+      j_cur = j_nxt;
+      if (t + 1 < steps) sk_cur = __ldg(p.k_scales + bh_rows + j_nxt);
+      if (t + 2 < steps) j_nxt = __ldg(list + (t + 2) / kStepsPerBlock);
       int valid = p.tokens - j * BS - (kPair ? 0 : (t & 1) * kStepKeys);
       valid = max(0, min(kStepKeys, valid));
 
-      if (!(ok = mbar_wait(&bars->s_full[buf], (t >> 1) & 1, abort_flag, p.status, 301))) break;
+      // S(t) is ready when Q K^T of step t is done; P[buf] is free when P V of step t-2 is done.  Both are normally
+      // complete by now: try them back to back so that their latencies overlap, and fall into the bounded waits
+      // only if one is not.
+      {
+        uint64_t* const qk_bar = &bars->qk_done[t % kRing];
+        uint64_t* const pv_bar = &bars->pv_done[(t + kRing - 2) % kRing];
+        const uint32_t pv_par = static_cast<uint32_t>(((t - 2) / kRing) & 1);
+        const bool qk_ok = mbar_try_wait(qk_bar, (t / kRing) & 1);
+        const bool pv_ok = t < 2 || mbar_try_wait(pv_bar, pv_par);
+        if (!qk_ok && !(ok = mbar_wait(qk_bar, (t / kRing) & 1, abort_flag, p.status, 301))) break;
+        if (!pv_ok && !(ok = mbar_wait(pv_bar, pv_par, abort_flag, p.status, 302))) break;
+      }
       tc_fence_after();
-      uint32_t s_lo[32], s_hi[32];
-      tmem_ld32(lane_addr + kColS + buf * 64, s_lo);
-      tmem_ld32(lane_addr + kColS + buf * 64 + 32, s_hi);
+      uint32_t mine[32], other[32];
+      tmem_ld32(lane_addr + kColS + buf * 64 + ch * 32, mine);
+      tmem_ld32(lane_addr + kColS + buf * 64 + (ch ^ 1) * 32, other);
       tmem_wait_ld();
       tc_fence_before();
       mbar_arrive(&bars->s_empty[buf]);
 
-      float sv[64];
-#pragma unroll
-      for (int k = 0; k < 32; ++k) {
-        sv[k] = __uint_as_float(s_lo[k]);
-        sv[k + 32] = __uint_as_float(s_hi[k]);
-      }
       if (valid < kStepKeys) {
 #pragma unroll
-        for (int k = 0; k < 64; ++k)
-          if (k >= valid) sv[k] = -INFINITY;
+        for (int k = 0; k < 32; ++k) {
+          if (ch * 32 + k >= valid) mine[k] = 0xFF800000u;         // -inf
+          if ((ch ^ 1) * 32 + k >= valid) other[k] = 0xFF800000u;
+        }
       }
-      // row maximum of the raw scores (c > 0 commutes with max), four independent chains
-      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      // row maximum of the raw scores over all 64 columns (c > 0 commutes with max), four independent chains
+      float mx4[4];
 #pragma unroll
-      for (int k = 0; k < 64; ++k) mx4[k & 3] = fmaxf(mx4[k & 3], sv[k]);
-      const float tile_max = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * c;
+      for (int q = 0; q < 4; ++q) mx4[q] = fmaxf(__uint_as_float(mine[q]), __uint_as_float(other[q]));
+#pragma unroll
+      for (int k = 4; k < 32; k += 4) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) mx4[q] = max3(mx4[q], __uint_as_float(mine[k + q]), __uint_as_float(other[k + q]));
+      }
+      const float tile_max = max3(fmaxf(mx4[0], mx4[1]), mx4[2], mx4[3]) * c;
 
       bool need = false;
       float alpha = 1.f;
       if (t == 0) {
-        m_ref = fmaxf(tile_max, m_ref);
+        m_ref = tile_max;
       } else if (tile_max > m_ref + kRescaleThreshold) {
         need = true;
         alpha = ex2(m_ref - tile_max);
         m_ref = tile_max;
         l *= alpha;
       }
-      const float neg_shift = __log2f(f) - m_ref;
-      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-      uint32_t packed[32];
+      // exponent arguments and row sums on pairs of columns (packed fp32x2 fma / add)
+      const uint64_t c2 = pack_f32x2(c, c), shift2 = pack_f32x2(-m_ref, -m_ref);
+      uint64_t sum2[2] = {0ull, 0ull};  // bit pattern of (0.f, 0.f)
+      uint32_t packed[16];
 #pragma unroll
-      for (int k = 0; k < 64; k += 2) {
-        const float p0 = ex2(fmaf(sv[k], c, neg_shift)), p1 = ex2(fmaf(sv[k + 1], c, neg_shift));
-        sum4[(k >> 1) & 3] += p0 + p1;
+      for (int k = 0; k < 32; k += 2) {
+        float a0, a1;
+        unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(mine[k]), __uint_as_float(mine[k + 1])), c2, shift2), a0, a1);
+        const float p0 = ex2(a0), p1 = ex2(a1);
+        sum2[(k >> 1) & 1] = add_f32x2(sum2[(k >> 1) & 1], pack_f32x2(p0, p1));
         packed[k >> 1] = pack_half2(p0, p1);
       }
-      l += ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3])) / f;
-
-      // P[buf] is free once the P V product of step t-2 has completed
-      if (!(ok = mbar_wait(&bars->p_empty[buf], ((t >> 1) & 1) ^ 1, abort_flag, p.status, 302))) break;
-      uint8_t* prow = p_tile + buf * kPBuf + p_row * 128;
-#pragma unroll
-      for (int ch = 0; ch < 8; ++ch) {
-        const uint4 v4 = make_uint4(packed[4 * ch], packed[4 * ch + 1], packed[4 * ch + 2], packed[4 * ch + 3]);
-        *reinterpret_cast<uint4*>(prow + ((ch ^ (p_row & 7)) << 4)) = v4;
+      {
+        float s0, s1;
+        unpack_f32x2(add_f32x2(sum2[0], sum2[1]), s0, s1);
+        l += s0 + s1;
       }
+
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        *reinterpret_cast<uint4*>(prow + buf * kPBuf + chunk_off[i]) =
+            make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
       if (__any_sync(0xFFFFFFFFu, need)) {
-        // O may only be touched between the P V products of steps t-1 and t
-        if (!(ok = mbar_wait(&bars->p_empty[buf ^ 1], ((t - 1) >> 1) & 1, abort_flag, p.status, 303))) break;
+        // O may only be touched between the P V products of steps t-1 and t; each thread rescales its 32 columns
+        if (!(ok = mbar_wait(&bars->pv_done[(t - 1) % kRing], ((t - 1) / kRing) & 1, abort_flag, p.status, 303))) break;
         tc_fence_after();
-        uint32_t o_lo[32], o_hi[32];
-        tmem_ld32(lane_addr + kColO, o_lo);
-        tmem_ld32(lane_addr + kColO + 32, o_hi);
+        uint32_t o[32];
+        tmem_ld32(lane_addr + kColO + ch * 32, o);
         tmem_wait_ld();
 #pragma unroll
-        for (int k = 0; k < 32; ++k) {
-          o_lo[k] = __float_as_uint(__uint_as_float(o_lo[k]) * alpha);
-          o_hi[k] = __float_as_uint(__uint_as_float(o_hi[k]) * alpha);
-        }
-        tmem_st32(lane_addr + kColO, o_lo);
-        tmem_st32(lane_addr + kColO + 32, o_hi);
+        for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
+        tmem_st32(lane_addr + kColO + ch * 32, o);
         tmem_wait_st();
         tc_fence_before();
       }
@@ -367,16 +397,16 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     // wait for the last P V product
     if (ok && steps > 0) {
       const int last = steps - 1;
-      ok = mbar_wait(&bars->p_empty[last & 1], (last >> 1) & 1, abort_flag, p.status, 304);
+      ok = mbar_wait(&bars->pv_done[last % kRing], (last / kRing) & 1, abort_flag, p.status, 304);
       tc_fence_after();
     }
 
-    // linear branch: phi(q) as bf16 A operand, denominators on the side
-    float den = 1.f;
+    // linear branch: this thread's 32 columns of phi(q) as bf16 A operand, partial denominator on the side
+    float den = 0.f;
     if (ok && p.k_marg > 0) {
       const uint4* qsrc = reinterpret_cast<const uint4*>(p.q_codes + (q_tile * BS + row_in_block) * kHeadDim);
-      const float* zeta = p.zeta + q_tile * kHeadDim;
-      float e[64];
+      const float* zeta = p.zeta + q_tile * kHeadDim + ch * 32;
+      float e[32];
       float mx = -INFINITY;
 #pragma unroll
       for (int w = 0; w < 4; ++w) {
@@ -388,22 +418,22 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           e4m3x4_to_float(words[xw], fv);
 #pragma unroll
           for (int y = 0; y < 4; ++y) {
-            e[w * 16 + xw * 4 + y] = fv[y] * sq;
-            mx = fmaxf(mx, fv[y] * sq);
+            mx = fmaxf(mx, fv[y]);
+            if ((w >> 1) == ch) e[(w & 1) * 16 + xw * 4 + y] = fv[y];
           }
         }
       }
-      uint32_t packed[32];
-      den = 0.f;
+      const float cq = sq * kLog2e, shift = mx * cq;  // sq > 0 commutes with max
+      uint32_t packed[16];
 #pragma unroll
-      for (int d = 0; d < 64; d += 2) {
+      for (int d = 0; d < 32; d += 2) {
         float e0, e1;
         if (p.phi == LITE3R_PHI_SOFTMAX) {  // the softmax normaliser cancels in the ratio
-          e0 = ex2((e[d] - mx) * kLog2e);
-          e1 = ex2((e[d + 1] - mx) * kLog2e);
+          e0 = ex2(fmaf(e[d], cq, -shift));
+          e1 = ex2(fmaf(e[d + 1], cq, -shift));
         } else {
-          e0 = e[d] > 0.f ? e[d] + 1.f : ex2(e[d] * kLog2e);
-          e1 = e[d + 1] > 0.f ? e[d + 1] + 1.f : ex2(e[d + 1] * kLog2e);
+          e0 = e[d] > 0.f ? fmaf(e[d], sq, 1.f) : ex2(e[d] * cq);
+          e1 = e[d + 1] > 0.f ? fmaf(e[d + 1], sq, 1.f) : ex2(e[d + 1] * cq);
         }
         const uint32_t pk = pack_bf162(e0, e1);
         packed[d >> 1] = pk;
@@ -411,14 +441,28 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         den = fmaf(__uint_as_float(pk << 16), __ldg(zeta + d), den);
         den = fmaf(__uint_as_float(pk & 0xFFFF0000u), __ldg(zeta + d + 1), den);
       }
-      uint8_t* prow = p_tile + p_row * 128;
 #pragma unroll
-      for (int ch = 0; ch < 8; ++ch) {
-        const uint4 v4 = make_uint4(packed[4 * ch], packed[4 * ch + 1], packed[4 * ch + 2], packed[4 * ch + 3]);
-        *reinterpret_cast<uint4*>(prow + ((ch ^ (p_row & 7)) << 4)) = v4;
-      }
+      for (int i = 0; i < 4; ++i)
+        *reinterpret_cast<uint4*>(prow + chunk_off[i]) =
+            make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
       fence_proxy_async_smem();
       mbar_arrive(&bars->phi_full);
+    }
+
+    // the two threads of a row swap their partial softmax sums and denominators (K stage 0 is free by now:
+    // every Q K^T product has completed before the last P V product did)
+    if (ok) {
+      float2* xbuf = reinterpret_cast<float2*>(smem + kOffX);
+      xbuf[ch * 128 + p_row] = make_float2(l, den);
+      mbar_arrive(&bars->x_full);
+      ok = mbar_wait(&bars->x_full, 0, abort_flag, p.status, 306);
+      if (ok) {
+        const float2 partner = xbuf[(ch ^ 1) * 128 + p_row];
+        l += partner.x;
+        den += partner.y;
+      }
+    }
+    if (ok && p.k_marg > 0) {
       ok = mbar_wait(&bars->l_full, 0, abort_flag, p.status, 305);
       tc_fence_after();
     }
@@ -426,27 +470,25 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     if (ok) {
       const bool live = token < p.tokens && (!kPair || hf == 0 || i_q[1] != i_q[0]);
       const int b = bh / p.heads, h = bh % p.heads;
-      float* dst = p.out + b * p.out_stride_b + h * p.out_stride_h + static_cast<long long>(token) * p.out_stride_n;
-      const float o_scale = steps > 0 ? vref / l : 0.f;
+      float* dst = p.out + b * p.out_stride_b + h * p.out_stride_h + static_cast<long long>(token) * p.out_stride_n +
+                   ch * 32;
+      const float o_scale = steps > 0 ? 1.f / l : 0.f;
       const float l_scale = p.k_marg > 0 ? 1.f / den : 0.f;
+      uint32_t o[32], ln[32];
+      if (steps > 0) tmem_ld32(lane_addr + kColO + ch * 32, o);
+      if (p.k_marg > 0) tmem_ld32(lane_addr + kColL + ch * 32, ln);
+      tmem_wait_ld();
+      if (live) {
 #pragma unroll
-      for (int part = 0; part < 2; ++part) {
-        uint32_t o[32], ln[32];
-        if (steps > 0) tmem_ld32(lane_addr + kColO + part * 32, o);
-        if (p.k_marg > 0) tmem_ld32(lane_addr + kColL + part * 32, ln);
-        tmem_wait_ld();
-        if (live) {
+        for (int k = 0; k < 32; k += 4) {
+          float r[4];
 #pragma unroll
-          for (int k = 0; k < 32; k += 4) {
-            float r[4];
-#pragma unroll
-            for (int y = 0; y < 4; ++y) {
-              const float a = steps > 0 ? __uint_as_float(o[k + y]) * o_scale : 0.f;
-              const float bb = p.k_marg > 0 ? __uint_as_float(ln[k + y]) * l_scale : 0.f;
-              r[y] = a + bb;
-            }
-            *reinterpret_cast<float4*>(dst + part * 32 + k) = make_float4(r[0], r[1], r[2], r[3]);
+          for (int y = 0; y < 4; ++y) {
+            const float a = steps > 0 ? __uint_as_float(o[k + y]) * o_scale : 0.f;
+            const float bb = p.k_marg > 0 ? __uint_as_float(ln[k + y]) * l_scale : 0.f;
+            r[y] = a + bb;
           }
+          *reinterpret_cast<float4*>(dst + k) = make_float4(r[0], r[1], r[2], r[3]);
         }
       }
     }
@@ -477,7 +519,6 @@ lite3r_status launch(const AttentionLaunch& a, cudaStream_t stream) {
   p.q_scales = a.q_scales;
   p.k_scales = a.k_scales;
   p.v_scales = a.v_scales;
-  p.vref = a.vref;
   p.crit_idx = a.crit_idx;
   p.zeta = a.zeta;
   p.out = a.out;

@@ -91,10 +91,9 @@ struct AttentionLaunch {
   const float* q_scales;
   const float* k_scales;
   const float* v_scales;
-  const __half* v16;          // [tiles*Bs][64] V code values as fp16
+  const __half* v16;          // [tiles*Bs][64] dequantised V as fp16
   const __nv_bfloat16* g16;   // [tiles][64][64] aggregated projected summaries, [e][d]
   const float* zeta;          // [tiles][64]
-  const float* vref;          // [B*H]
   const int* crit_idx;
   int k_crit, k_marg, phi;
   float* out;

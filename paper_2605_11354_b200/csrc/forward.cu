@@ -6,7 +6,7 @@
 //   K4  attention.cu      per query block i: online-softmax attention over the critical key blocks (lines 4-5),
 //                         then the linear branch (line 9) phi(q) G_i / (phi(q) . zeta_i), the sum of the two
 //                         (line 10) and the store.
-//   prep_kernel           V code values as fp16 and the per-head reference V scale for the attention kernel.
+//   prep_kernel           dequantised V as fp16 for the attention kernel's P V product.
 #include <algorithm>
 
 #include "common.cuh"
@@ -16,23 +16,27 @@ namespace lite3r {
 namespace {
 
 // ------------------------------------------------------------------------------------------------ prep
-// V code values as fp16 (exact) for the P V tensor-core product, and the largest V block scale of every head.
+// Dequantised V (code value x block scale) as fp16, the B operand of the P V tensor-core product.
 __global__ void __launch_bounds__(256) prep_kernel(const uint8_t* __restrict__ v_codes, const float* __restrict__ v_scales,
-                                                   size_t words, int tiles, int nb, __half* __restrict__ v16,
-                                                   float* __restrict__ vref) {
+                                                   size_t words, int words_per_tile, __half* __restrict__ v16) {
   const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
   for (size_t w = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; w < words; w += stride) {
-    const uint32_t packed = __ldg(reinterpret_cast<const uint32_t*>(v_codes) + w);
-    const __half2_raw lo = __nv_cvt_fp8x2_to_halfraw2(static_cast<__nv_fp8x2_storage_t>(packed & 0xFFFFu), __NV_E4M3);
-    const __half2_raw hi = __nv_cvt_fp8x2_to_halfraw2(static_cast<__nv_fp8x2_storage_t>(packed >> 16), __NV_E4M3);
-    uint2 out;
-    out.x = static_cast<uint32_t>(lo.x) | (static_cast<uint32_t>(lo.y) << 16);
-    out.y = static_cast<uint32_t>(hi.x) | (static_cast<uint32_t>(hi.y) << 16);
-    reinterpret_cast<uint2*>(v16)[w] = out;
+    const uint4 packed = __ldg(reinterpret_cast<const uint4*>(v_codes) + w);
+    const float sv = __ldg(v_scales + w / words_per_tile);
+    const uint32_t in[4] = {packed.x, packed.y, packed.z, packed.w};
+    uint32_t out[8];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      float f[4];
+      e4m3x4_to_float(in[q], f);
+      const __half2 lo = __floats2half2_rn(f[0] * sv, f[1] * sv), hi = __floats2half2_rn(f[2] * sv, f[3] * sv);
+      out[2 * q] = *reinterpret_cast<const uint32_t*>(&lo);
+      out[2 * q + 1] = *reinterpret_cast<const uint32_t*>(&hi);
+    }
+    uint4* dst = reinterpret_cast<uint4*>(v16) + 2 * w;
+    dst[0] = make_uint4(out[0], out[1], out[2], out[3]);
+    dst[1] = make_uint4(out[4], out[5], out[6], out[7]);
   }
-  // scales are positive, so their bit patterns order like integers; max is order-independent (deterministic)
-  for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < tiles; t += static_cast<int>(stride))
-    atomicMax(reinterpret_cast<int*>(vref) + t / nb, __float_as_int(v_scales[t]));
 }
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -41,8 +45,7 @@ struct Workspace {
   __nv_bfloat16* hws;  // [tiles][4160]   per-key-block summaries
   __nv_bfloat16* g16;  // [tiles][64][64] aggregated summaries, [e][d]
   float* zeta;         // [tiles][64]
-  __half* v16;         // [tiles*Bs][64]  V code values as fp16
-  float* vref;         // [B*H]
+  __half* v16;         // [tiles*Bs][64]  dequantised V as fp16
   size_t bytes;
 };
 
@@ -60,7 +63,6 @@ Workspace carve(void* base, const lite3r_shape& s) {
   w.g16 = reinterpret_cast<__nv_bfloat16*>(take(tiles * kHeadDim * kHeadDim * sizeof(__nv_bfloat16)));
   w.zeta = reinterpret_cast<float*>(take(tiles * kHeadDim * sizeof(float)));
   w.v16 = reinterpret_cast<__half*>(take(tiles * s.block * kHeadDim * sizeof(__half)));
-  w.vref = reinterpret_cast<float*>(take(static_cast<size_t>(s.batch) * s.heads * sizeof(float)));
   w.bytes = off;
   return w;
 }
@@ -74,11 +76,11 @@ lite3r_status run_forward(const ForwardArgs& a, cudaStream_t stream) {
   lite3r_status st;
   profile_mark(0, stream);
   if (a.plan.k_crit > 0) {
-    st = record_cuda(cudaMemsetAsync(w.vref, 0, static_cast<size_t>(s.batch) * s.heads * sizeof(float), stream));
-    if (st != LITE3R_OK) return st;
-    const size_t words = static_cast<size_t>(rows) * BS * kHeadDim / 4;
-    const int blocks = static_cast<int>(std::min<size_t>((words + 255) / 256, 148 * 16));
-    prep_kernel<<<blocks, 256, 0, stream>>>(a.v.codes, a.v.scales, words, rows, nb, w.v16, w.vref);
+    const size_t words = static_cast<size_t>(rows) * BS * kHeadDim / 16;  // 16 codes per thread and pass
+    int sms = 0;
+    if ((st = sm_count(&sms)) != LITE3R_OK) return st;
+    const int blocks = static_cast<int>(std::min<size_t>((words + 255) / 256, static_cast<size_t>(sms) * 8));
+    prep_kernel<<<blocks, 256, 0, stream>>>(a.v.codes, a.v.scales, words, BS * kHeadDim / 16, w.v16);
     if ((st = after_launch()) != LITE3R_OK) return st;
     profile_mark(1, stream);
   }
@@ -101,7 +103,6 @@ lite3r_status run_forward(const ForwardArgs& a, cudaStream_t stream) {
   att.v16 = w.v16;
   att.g16 = w.g16;
   att.zeta = w.zeta;
-  att.vref = w.vref;
   att.crit_idx = a.plan.crit_idx;
   att.k_crit = a.plan.k_crit;
   att.k_marg = a.plan.k_marg;
