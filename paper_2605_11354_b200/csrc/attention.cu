@@ -2,23 +2,27 @@
 //
 // One CTA owns 128 query rows of one (b, h): at block 64 a PAIR of query blocks (two M=64 accumulators interleaved
 // in the two 16-lane halves of every TMEM sub-partition), at block 128 one query block (M=128).  Work advances in
-// steps of 64 keys.  Per step t:
+// steps of 64 keys.  The steps are dealt alternately to two independent "sets" (even steps -> set 0, odd steps ->
+// set 1).  A set is 128 softmax threads (one query row each, TMEM lane = thread) plus one MMA-issuing thread, with
+// its own score buffer S, probability buffer P, output accumulator O and online-softmax state (reference maximum and
+// row sum); the two partial results are merged exactly at the end, O = (w0 O0 + w1 O1) / (w0 l0 + w1 l1) with
+// w = 2^(m_set - m).  Because the sets never wait for each other, an SM (two CTAs) always has four softmax streams
+// in different phases, which keeps the exponential unit busy while other streams wait on barriers, TMEM loads or
+// shared-memory stores.  Per step t of set b = t & 1:
 //   TMA      K tile(s) (e4m3, 64-byte rows, 64B swizzle) and V tile(s) (dequantised fp16, 128B swizzle) -> smem ring
-//   tcgen05  S[t&1] = Q K^T        kind::f8f6f4, fp32 accumulators in TMEM (64 columns)
-//   softmax  256 threads, two per query row (TMEM lane = thread, 32 of the 64 columns each): scale, mask padded
-//            keys, running max with lazy rescale, exp2, row sum; P goes to shared memory as fp16 in the MMA's
-//            K-major 128B-swizzled layout.  Both threads of a row read all 64 scores for the maximum, so they
-//            take identical rescale decisions without exchanging anything; only the exponentials are split.
-//   tcgen05  O += P V              kind::f16, V as MN-major B operand, fp32 accumulators in TMEM (64 columns)
+//   tcgen05  S_b = Q K^T           kind::f8f6f4, fp32 accumulators in TMEM (64 columns)
+//   softmax  pass 1: row maximum of the 64 scores, lazy-rescale decision; pass 2: exp2 and row sum, 32 columns at a
+//            time; P goes to shared memory as fp16 in the MMA's K-major 128B-swizzled layout
+//   tcgen05  O_b += P V            kind::f16, V as MN-major B operand, fp32 accumulators in TMEM (64 columns)
 // P is carried in fp16 (not e4m3): one e4m3 term has a 2.6 % rounding error per probability, which alone is ten
 // times the output tolerance.  V travels as the dequantised value in fp16 (2^-12 relative rounding).
 // Tail: phi(Q) (bf16) times the aggregated, projected summaries G_i (bf16) as one more MMA, divided by
-// phi(Q) . zeta_i, added to O / l and stored; the two threads of a row swap their partial row sums once.
+// phi(Q) . zeta_i, added to the merged softmax output and stored (each set stores 32 of the 64 output columns).
 //
-// Warp roles (352 threads): warp 0 = TMA producer, warp 1 = Q K^T issuer and TMEM owner, warp 2 = P V issuer (and the
-// linear-branch MMA), warps 3-10 = softmax/epilogue.  A single thread can issue one small tcgen05.mma roughly every
-// 50 clocks, so the two products have an issuing thread each; "product t done" is one barrier per product (rings of
-// six, committed once) on which both the softmax threads and the TMA producer wait.
+// Warp roles (352 threads): warp 0 = TMA producer; warps 1 and 2 = MMA issuers of set 0 and set 1 (a single thread
+// can issue a small tcgen05.mma only every ~50 clocks, so each set has its own); warps 3-6 = softmax set 0,
+// warps 7-10 = softmax set 1.  "Product of step t done" is one barrier per product (rings of six) on which the
+// softmax threads and the TMA producer wait.
 // Every mbarrier wait is bounded (1 s); on expiry the CTA sets *device_status and all roles leave their loops.
 #include "common.cuh"
 #include "sm100.cuh"
@@ -30,17 +34,19 @@ namespace {
 using namespace sm100;
 
 constexpr int kStages = 3;
-constexpr int kSoftmaxThreads = 256;
+constexpr int kSetThreads = 128;
+constexpr int kSoftmaxThreads = 2 * kSetThreads;
 constexpr int kCtrlWarps = 3;
 constexpr int kThreads = kCtrlWarps * 32 + kSoftmaxThreads;
 constexpr uint32_t kBackoffNs = 100;  // sleep between polls of the single-thread roles
-constexpr int kRing = 6;  // lcm of the S/P double buffers and the three K/V stages
+constexpr int kRing = 6;              // lcm of the two sets and the three K/V stages
 constexpr int kStepKeys = 64;
 constexpr uint32_t kTmemCols = 256;
-constexpr uint32_t kColS = 0, kColO = 128, kColL = 192;
+constexpr uint32_t kColS = 0, kColO = 128, kColL = 0;  // S_b at 64 b, O_b at 128 + 64 b; the linear branch reuses S_0
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRescaleThreshold = 8.0f;  // lazy rescale: keep the old reference max until it is beaten by 2^8
-constexpr uint32_t kOffX = 8192;           // row-sum exchange of the epilogue: reuses K stage 0 (2 KB)
+constexpr float kNoMax = -1.0e30f;         // reference maximum of a row that has seen no valid key yet
+constexpr uint32_t kOffX = 8192;           // epilogue exchange between the sets: reuses K stage 0 (4 KB)
 
 // shared-memory map (bytes from a 1024-aligned base)
 constexpr uint32_t kQBytes = 8192, kKStage = 8192, kVStage = 16384, kPBuf = 16384;
@@ -55,7 +61,7 @@ struct Bars {
   uint64_t q_full, g_full, phi_full, l_full, x_full;
   uint64_t k_full[kStages], v_full[kStages];  // TMA -> issuers
   uint64_t qk_done[kRing], pv_done[kRing];    // product of step t complete: barrier t % 6, phase (t / 6)
-  uint64_t s_empty[2], p_full[2];             // softmax -> issuers
+  uint64_t s_empty[2], p_full[2];             // softmax set b -> issuer b
   uint32_t tmem_base;
   int abort;
 };
@@ -64,7 +70,6 @@ struct AttnParams {
   const uint8_t* q_codes;
   const float* q_scales;
   const float* k_scales;
-  const float* v_scales;
   const int* crit_idx; // [B*H*Nb][k_crit]
   const float* zeta;   // [B*H*Nb][64]
   float* out;
@@ -85,6 +90,24 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 __device__ __forceinline__ uint32_t pack_bf162(float a, float b) {
   __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<uint32_t*>(&h);
+}
+
+// exp2 of 32 scaled scores, packed to fp16 pairs; returns the sum.  Arguments and sums run on pairs of columns
+// (packed fp32x2 fma / add).
+__device__ __forceinline__ float exp_half_row(const uint32_t (&x)[32], float c, float neg_ref, uint32_t* packed) {
+  const uint64_t c2 = pack_f32x2(c, c), shift2 = pack_f32x2(neg_ref, neg_ref);
+  uint64_t sum2[2] = {0ull, 0ull};  // bit pattern of (0.f, 0.f)
+#pragma unroll
+  for (int k = 0; k < 32; k += 2) {
+    float a0, a1;
+    unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(x[k]), __uint_as_float(x[k + 1])), c2, shift2), a0, a1);
+    const float p0 = ex2(a0), p1 = ex2(a1);
+    sum2[(k >> 1) & 1] = add_f32x2(sum2[(k >> 1) & 1], pack_f32x2(p0, p1));
+    packed[k >> 1] = pack_half2(p0, p1);
+  }
+  float s0, s1;
+  unpack_f32x2(add_f32x2(sum2[0], sum2[1]), s0, s1);
+  return s0 + s1;
 }
 
 template <int BS>
@@ -133,8 +156,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       mbar_init(&bars->pv_done[r], 1);
     }
     for (int b = 0; b < 2; ++b) {
-      mbar_init(&bars->s_empty[b], kSoftmaxThreads);
-      mbar_init(&bars->p_full[b], kSoftmaxThreads);
+      mbar_init(&bars->s_empty[b], kSetThreads);
+      mbar_init(&bars->p_full[b], kSetThreads);
     }
     bars->abort = 0;
     mbar_fence_init();
@@ -187,11 +210,9 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           tma_load_2d(smem + kOffV + st * kVStage + hf * 8192, &map_v, &bars->v_full[st], 0, row[hf]);
       }
       if (ok && p.k_marg > 0) {
-        // The aggregated summaries reuse V stage 0; it is free once the last P V product has completed.
-        if (steps > 0) {
-          const int last = steps - 1;
-          ok = mbar_wait(&bars->pv_done[last % kRing], (last / kRing) & 1, abort_flag, p.status, 103);
-        }
+        // The aggregated summaries reuse V stage 0; it is free once the last two P V products have completed.
+        for (int u = max(0, steps - 2); u < steps && ok; ++u)
+          ok = mbar_wait(&bars->pv_done[u % kRing], (u / kRing) & 1, abort_flag, p.status, 103, kBackoffNs);
         if (ok) {
           mbar_arrive_expect_tx(&bars->g_full, kHalves * 8192);
           for (int hf = 0; hf < kHalves; ++hf)
@@ -199,69 +220,71 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
       }
     }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------------------------------ Q K^T issuer
+  } else if (warp < kCtrlWarps) {
+    // ------------------------------------------------------------------------------------------ MMA issuer of set b
     if (lane == 0) {
+      const int b = warp - 1;
       constexpr uint32_t idesc_qk = instr_desc(0, kM, 64, 0, 0);   // e4m3 x e4m3, both K-major
+      constexpr uint32_t idesc_pv = instr_desc(0, kM, 64, 0, 1);   // f16 x f16, V MN-major
+      constexpr uint32_t idesc_lin = instr_desc(1, kM, 64, 0, 0);  // bf16 x bf16, both K-major
       const uint32_t q_addr = smem_u32(smem + kOffQ), k_addr = smem_u32(smem + kOffK);
-      bool ok = mbar_wait(&bars->q_full, 0, abort_flag, p.status, 201);
-      // Gated only by the K tile and by the softmax threads having pulled S(t-2) into registers, so this runs up
-      // to two steps ahead of the softmax.
-      for (int t = 0; t < steps && ok; ++t) {
-        const int st = t % kStages, buf = t & 1;
-        if (!(ok = mbar_wait(&bars->k_full[st], (t / kStages) & 1, abort_flag, p.status, 202, kBackoffNs))) break;
-        if (!(ok = mbar_wait(&bars->s_empty[buf], ((t >> 1) & 1) ^ 1, abort_flag, p.status, 203, kBackoffNs))) break;
+      const uint32_t v_addr = smem_u32(smem + kOffV), p_addr = smem_u32(smem + kOffP) + b * kPBuf;
+      const uint32_t s_tmem = tmem + kColS + b * 64, o_tmem = tmem + kColO + b * 64;
+      bool ok = mbar_wait(&bars->q_full, 0, abort_flag, p.status, 201, kBackoffNs);
+      auto issue_qk = [&](int t) {  // S_b = Q K(t)^T; needs the K tile and S_b drained by the softmax of step t-2
+        const int st = t % kStages;
+        if (!mbar_wait(&bars->k_full[st], (t / kStages) & 1, abort_flag, p.status, 202, kBackoffNs)) return false;
+        if (!mbar_wait(&bars->s_empty[b], ((t >> 1) & 1) ^ 1, abort_flag, p.status, 203, kBackoffNs)) return false;
         tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < 2; ++kk) {
 #pragma unroll
           for (int hf = 0; hf < kHalves; ++hf) {
-            const uint32_t d = tmem + kColS + buf * 64 + ((hf * 16u) << 16);
             const uint64_t a = smem_desc(q_addr + (kPair ? hf * 4096 : 0) + kk * 32, 16, 512, kSwizzle64);
-            const uint64_t b = smem_desc(k_addr + st * kKStage + hf * 4096 + kk * 32, 16, 512, kSwizzle64);
-            mma_f8(d, a, b, idesc_qk, kk);
+            const uint64_t bd = smem_desc(k_addr + st * kKStage + hf * 4096 + kk * 32, 16, 512, kSwizzle64);
+            mma_f8(s_tmem + ((hf * 16u) << 16), a, bd, idesc_qk, kk);
           }
         }
         mma_commit(&bars->qk_done[t % kRing]);
-      }
-    }
-  } else if (warp == 2) {
-    // ------------------------------------------------------------------------------------------ P V issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc_pv = instr_desc(0, kM, 64, 0, 1);   // f16 x f16, V MN-major
-      constexpr uint32_t idesc_lin = instr_desc(1, kM, 64, 0, 0);  // bf16 x bf16, both K-major
-      const uint32_t v_addr = smem_u32(smem + kOffV), p_addr = smem_u32(smem + kOffP);
-      bool ok = true;
-      for (int t = 0; t < steps && ok; ++t) {
-        const int st = t % kStages, buf = t & 1;
-        if (!(ok = mbar_wait(&bars->v_full[st], (t / kStages) & 1, abort_flag, p.status, 204, kBackoffNs))) break;
-        if (!(ok = mbar_wait(&bars->p_full[buf], (t >> 1) & 1, abort_flag, p.status, 205, kBackoffNs))) break;
+        return true;
+      };
+      auto issue_pv = [&](int t) {  // O_b += P(t) V(t)
+        const int st = t % kStages;
+        if (!mbar_wait(&bars->v_full[st], (t / kStages) & 1, abort_flag, p.status, 204, kBackoffNs)) return false;
+        if (!mbar_wait(&bars->p_full[b], (t >> 1) & 1, abort_flag, p.status, 205, kBackoffNs)) return false;
         tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk) {
 #pragma unroll
           for (int hf = 0; hf < kHalves; ++hf) {
-            const uint32_t d = tmem + kColO + ((hf * 16u) << 16);
-            const uint64_t a = smem_desc(p_addr + buf * kPBuf + (kPair ? hf * 8192 : 0) + kk * 32, 16, 1024, kSwizzle128);
-            const uint64_t b = smem_desc(v_addr + st * kVStage + hf * 8192 + kk * 2048, 8192, 1024, kSwizzle128);
-            mma_f16(d, a, b, idesc_pv, (t > 0 || kk > 0) ? 1u : 0u);
+            const uint64_t a = smem_desc(p_addr + (kPair ? hf * 8192 : 0) + kk * 32, 16, 1024, kSwizzle128);
+            const uint64_t bd = smem_desc(v_addr + st * kVStage + hf * 8192 + kk * 2048, 8192, 1024, kSwizzle128);
+            mma_f16(o_tmem + ((hf * 16u) << 16), a, bd, idesc_pv, (t >= 2 || kk > 0) ? 1u : 0u);
           }
         }
         mma_commit(&bars->pv_done[t % kRing]);
+        return true;
+      };
+      // S_b of the set's next step is produced as soon as the softmax threads have pulled the current one into
+      // registers, i.e. while they exponentiate; P V follows when they hand over the probabilities.
+      if (ok && b < steps) ok = issue_qk(b);
+      for (int t = b; t < steps && ok; t += 2) {
+        if (t + 2 < steps) ok = issue_qk(t + 2);
+        if (ok) ok = issue_pv(t);
       }
-      if (ok && p.k_marg > 0) {
-        ok = mbar_wait(&bars->g_full, 0, abort_flag, p.status, 206) &&
-             mbar_wait(&bars->phi_full, 0, abort_flag, p.status, 207);
+      if (b == 0 && ok && p.k_marg > 0) {
+        ok = mbar_wait(&bars->g_full, 0, abort_flag, p.status, 206, kBackoffNs) &&
+             mbar_wait(&bars->phi_full, 0, abort_flag, p.status, 207, kBackoffNs);
         if (ok) {
           tc_fence_after();
+          const uint32_t phi_addr = smem_u32(smem + kOffP);
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk) {
 #pragma unroll
             for (int hf = 0; hf < kHalves; ++hf) {
-              const uint32_t d = tmem + kColL + ((hf * 16u) << 16);
-              const uint64_t a = smem_desc(p_addr + (kPair ? hf * 8192 : 0) + kk * 32, 16, 1024, kSwizzle128);
-              const uint64_t b = smem_desc(v_addr + hf * 8192 + kk * 32, 16, 1024, kSwizzle128);
-              mma_f16(d, a, b, idesc_lin, kk);
+              const uint64_t a = smem_desc(phi_addr + (kPair ? hf * 8192 : 0) + kk * 32, 16, 1024, kSwizzle128);
+              const uint64_t bd = smem_desc(v_addr + hf * 8192 + kk * 32, 16, 1024, kSwizzle128);
+              mma_f16(tmem + kColL + ((hf * 16u) << 16), a, bd, idesc_lin, kk);
             }
           }
           mma_commit(&bars->l_full);
@@ -271,83 +294,70 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   } else {
     // ------------------------------------------------------------------------------------------ softmax + epilogue
     const int quarter = warp & 3;                       // TMEM sub-partition this warp may touch
-    const int ch = (warp - kCtrlWarps) >> 2;            // which 32 of the 64 columns this thread exponentiates
+    const int b = (warp - kCtrlWarps) >> 2;             // set: steps t with (t & 1) == b
     const int hf = kPair ? (lane >> 4) : 0;             // which query block of the pair this thread serves
     const int row_in_block = kPair ? quarter * 16 + (lane & 15) : quarter * 32 + lane;
     const int p_row = kPair ? hf * 64 + row_in_block : row_in_block;  // row inside the P / phi tile
     const int iq = i_q[hf];
     const size_t q_tile = bh_rows + iq;
     const uint32_t lane_addr = tmem + ((static_cast<uint32_t>(quarter) * 32u) << 16);
+    const uint32_t s_addr = lane_addr + kColS + b * 64, o_addr = lane_addr + kColO + b * 64;
     const int token = iq * BS + row_in_block;
     const float sq = __ldg(p.q_scales + q_tile);
     const float qk_scale = sq * (kLog2e * 0.125f);
     const int* list = p.crit_idx + q_tile * p.k_crit;
-    // this thread's four 16-byte chunks of its 128-byte P / phi row (128B swizzle)
-    uint8_t* const prow = smem + kOffP + p_row * 128;
-    uint32_t chunk_off[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) chunk_off[i] = static_cast<uint32_t>(((ch * 4 + i) ^ (p_row & 7)) << 4);
+    uint8_t* const prow = smem + kOffP + b * kPBuf + p_row * 128;  // this thread's 128-byte row of P_b
+    const int swz = p_row & 7;
 
-    float m_ref = -1.0e30f, l = 0.f;  // l: sum over this thread's 32 columns
+    float m_ref = kNoMax, l = 0.f;
     bool ok = true;
 
-    // per-step scalars: the key-block index is fetched two steps ahead and its scale one step ahead, so that no
-    // load in the loop waits for the address produced by another load of the same iteration
-    int j_cur = steps > 0 ? __ldg(list) : 0;
-    int j_nxt = steps > 1 ? __ldg(list + 1 / kStepsPerBlock) : 0;
-    float sk_cur = steps > 0 ? __ldg(p.k_scales + bh_rows + j_cur) : 0.f;
+    // per-step scalars: the key-block index is fetched two of the set's steps ahead and its scale one ahead, so
+    // that no load in the loop waits for the address produced by another load of the same iteration
+    int j_cur = b < steps ? ldg_pinned(list + b / kStepsPerBlock) : 0;
+    int j_nxt = b + 2 < steps ? ldg_pinned(list + (b + 2) / kStepsPerBlock) : 0;
+    float sk_cur = b < steps ? ldg_pinned(p.k_scales + bh_rows + j_cur) : 0.f;
 
-    for (int t = 0; t < steps; ++t) {
-      const int buf = t & 1;
+    for (int t = b; t < steps; t += 2) {
       const int j = j_cur;
       const float c = qk_scale * sk_cur;
       j_cur = j_nxt;
-      if (t + 1 < steps) sk_cur = __ldg(p.k_scales + bh_rows + j_nxt);
-      if (t + 2 < steps) j_nxt = __ldg(list + (t + 2) / kStepsPerBlock);
+      if (t + 2 < steps) sk_cur = ldg_pinned(p.k_scales + bh_rows + j_nxt);
+      if (t + 4 < steps) j_nxt = ldg_pinned(list + (t + 4) / kStepsPerBlock);
       int valid = p.tokens - j * BS - (kPair ? 0 : (t & 1) * kStepKeys);
       valid = max(0, min(kStepKeys, valid));
 
-      // S(t) is ready when Q K^T of step t is done; P[buf] is free when P V of step t-2 is done.  Both are normally
-      // complete by now: try them back to back so that their latencies overlap, and fall into the bounded waits
-      // only if one is not.
-      {
-        uint64_t* const qk_bar = &bars->qk_done[t % kRing];
-        uint64_t* const pv_bar = &bars->pv_done[(t + kRing - 2) % kRing];
-        const uint32_t pv_par = static_cast<uint32_t>(((t - 2) / kRing) & 1);
-        const bool qk_ok = mbar_try_wait(qk_bar, (t / kRing) & 1);
-        const bool pv_ok = t < 2 || mbar_try_wait(pv_bar, pv_par);
-        if (!qk_ok && !(ok = mbar_wait(qk_bar, (t / kRing) & 1, abort_flag, p.status, 301))) break;
-        if (!pv_ok && !(ok = mbar_wait(pv_bar, pv_par, abort_flag, p.status, 302))) break;
-      }
+      if (!(ok = mbar_wait(&bars->qk_done[t % kRing], (t / kRing) & 1, abort_flag, p.status, 301))) break;
       tc_fence_after();
-      uint32_t mine[32], other[32];
-      tmem_ld32(lane_addr + kColS + buf * 64 + ch * 32, mine);
-      tmem_ld32(lane_addr + kColS + buf * 64 + (ch ^ 1) * 32, other);
-      tmem_wait_ld();
-      tc_fence_before();
-      mbar_arrive(&bars->s_empty[buf]);
 
-      if (valid < kStepKeys) {
+      // pass 1: row maximum of the raw scores (c > 0 commutes with max), four independent chains
+      float tile_max;
+      {
+        uint32_t x[32], y[32];
+        tmem_ld32(s_addr, x);
+        tmem_ld32(s_addr + 32, y);
+        tmem_wait_ld();
+        if (valid < kStepKeys) {
 #pragma unroll
-        for (int k = 0; k < 32; ++k) {
-          if (ch * 32 + k >= valid) mine[k] = 0xFF800000u;         // -inf
-          if ((ch ^ 1) * 32 + k >= valid) other[k] = 0xFF800000u;
+          for (int k = 0; k < 32; ++k) {
+            if (k >= valid) x[k] = 0xFF800000u;  // -inf
+            if (32 + k >= valid) y[k] = 0xFF800000u;
+          }
         }
+        float mx4[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) mx4[q] = fmaxf(__uint_as_float(x[q]), __uint_as_float(y[q]));
+#pragma unroll
+        for (int k = 4; k < 32; k += 4) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) mx4[q] = max3(mx4[q], __uint_as_float(x[k + q]), __uint_as_float(y[k + q]));
+        }
+        // a step without any valid key (second half of a short last block) leaves the reference where it is
+        tile_max = fmaxf(max3(fmaxf(mx4[0], mx4[1]), mx4[2], mx4[3]) * c, kNoMax);
       }
-      // row maximum of the raw scores over all 64 columns (c > 0 commutes with max), four independent chains
-      float mx4[4];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) mx4[q] = fmaxf(__uint_as_float(mine[q]), __uint_as_float(other[q]));
-#pragma unroll
-      for (int k = 4; k < 32; k += 4) {
-#pragma unroll
-        for (int q = 0; q < 4; ++q) mx4[q] = max3(mx4[q], __uint_as_float(mine[k + q]), __uint_as_float(other[k + q]));
-      }
-      const float tile_max = max3(fmaxf(mx4[0], mx4[1]), mx4[2], mx4[3]) * c;
-
       bool need = false;
       float alpha = 1.f;
-      if (t == 0) {
+      if (t < 2) {
         m_ref = tile_max;
       } else if (tile_max > m_ref + kRescaleThreshold) {
         need = true;
@@ -355,57 +365,74 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         m_ref = tile_max;
         l *= alpha;
       }
-      // exponent arguments and row sums on pairs of columns (packed fp32x2 fma / add)
-      const uint64_t c2 = pack_f32x2(c, c), shift2 = pack_f32x2(-m_ref, -m_ref);
-      uint64_t sum2[2] = {0ull, 0ull};  // bit pattern of (0.f, 0.f)
-      uint32_t packed[16];
-#pragma unroll
-      for (int k = 0; k < 32; k += 2) {
-        float a0, a1;
-        unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(mine[k]), __uint_as_float(mine[k + 1])), c2, shift2), a0, a1);
-        const float p0 = ex2(a0), p1 = ex2(a1);
-        sum2[(k >> 1) & 1] = add_f32x2(sum2[(k >> 1) & 1], pack_f32x2(p0, p1));
-        packed[k >> 1] = pack_half2(p0, p1);
-      }
-      {
-        float s0, s1;
-        unpack_f32x2(add_f32x2(sum2[0], sum2[1]), s0, s1);
-        l += s0 + s1;
-      }
+      // P_b is free once the P V product of the set's previous step has completed; asked now, needed after the
+      // first exponentials
+      uint64_t* const pv_bar = &bars->pv_done[(t + kRing - 2) % kRing];
+      const uint32_t pv_par = static_cast<uint32_t>(((t - 2) / kRing) & 1);
+      const bool pv_ok = t < 2 || mbar_try_wait(pv_bar, pv_par);
 
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-        *reinterpret_cast<uint4*>(prow + buf * kPBuf + chunk_off[i]) =
-            make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
-      if (__any_sync(0xFFFFFFFFu, need)) {
-        // O may only be touched between the P V products of steps t-1 and t; each thread rescales its 32 columns
-        if (!(ok = mbar_wait(&bars->pv_done[(t - 1) % kRing], ((t - 1) / kRing) & 1, abort_flag, p.status, 303))) break;
-        tc_fence_after();
-        uint32_t o[32];
-        tmem_ld32(lane_addr + kColO + ch * 32, o);
+      // pass 2: exponentials and row sum, 32 columns at a time; each half row of P is stored as soon as it exists
+      {
+        uint32_t x[32], packed[16];
+        tmem_ld32(s_addr, x);
         tmem_wait_ld();
+        if (valid < 32) {
 #pragma unroll
-        for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
-        tmem_st32(lane_addr + kColO + ch * 32, o);
+          for (int k = 0; k < 32; ++k)
+            if (k >= valid) x[k] = 0xFF800000u;
+        }
+        l += exp_half_row(x, c, -m_ref, packed);
+        if (!pv_ok && !(ok = mbar_wait(pv_bar, pv_par, abort_flag, p.status, 302))) break;
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch)
+          *reinterpret_cast<uint4*>(prow + ((ch ^ swz) << 4)) =
+              make_uint4(packed[4 * ch], packed[4 * ch + 1], packed[4 * ch + 2], packed[4 * ch + 3]);
+        tmem_ld32(s_addr + 32, x);
+        tmem_wait_ld();
+        tc_fence_before();
+        mbar_arrive(&bars->s_empty[b]);  // S_b is in registers: the issuer may overwrite it with the set's next step
+        if (valid < kStepKeys) {
+#pragma unroll
+          for (int k = 0; k < 32; ++k)
+            if (32 + k >= valid) x[k] = 0xFF800000u;
+        }
+        l += exp_half_row(x, c, -m_ref, packed);
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch)
+          *reinterpret_cast<uint4*>(prow + (((4 + ch) ^ swz) << 4)) =
+              make_uint4(packed[4 * ch], packed[4 * ch + 1], packed[4 * ch + 2], packed[4 * ch + 3]);
+      }
+      if (__any_sync(0xFFFFFFFFu, need)) {
+        // O_b is only touched by the set's own P V products: the previous one has completed (pv_bar above) and the
+        // next one waits for this thread's arrival below
+        tc_fence_after();
+#pragma unroll
+        for (int part = 0; part < 2; ++part) {
+          uint32_t o[32];
+          tmem_ld32(o_addr + part * 32, o);
+          tmem_wait_ld();
+#pragma unroll
+          for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
+          tmem_st32(o_addr + part * 32, o);
+        }
         tmem_wait_st();
         tc_fence_before();
       }
       fence_proxy_async_smem();
-      mbar_arrive(&bars->p_full[buf]);
+      mbar_arrive(&bars->p_full[b]);
     }
 
-    // wait for the last P V product
-    if (ok && steps > 0) {
-      const int last = steps - 1;
-      ok = mbar_wait(&bars->pv_done[last % kRing], (last / kRing) & 1, abort_flag, p.status, 304);
-      tc_fence_after();
-    }
+    // both sets' last P V products (the epilogue reads O_0 and O_1)
+    for (int u = max(0, steps - 2); u < steps && ok; ++u)
+      ok = mbar_wait(&bars->pv_done[u % kRing], (u / kRing) & 1, abort_flag, p.status, 304);
+    tc_fence_after();
 
-    // linear branch: this thread's 32 columns of phi(q) as bf16 A operand, partial denominator on the side
+    // linear branch: this thread's 32 columns (set b -> columns 32 b ..) of phi(q) as bf16 A operand, partial
+    // denominator on the side
     float den = 0.f;
     if (ok && p.k_marg > 0) {
       const uint4* qsrc = reinterpret_cast<const uint4*>(p.q_codes + (q_tile * BS + row_in_block) * kHeadDim);
-      const float* zeta = p.zeta + q_tile * kHeadDim + ch * 32;
+      const float* zeta = p.zeta + q_tile * kHeadDim + b * 32;
       float e[32];
       float mx = -INFINITY;
 #pragma unroll
@@ -419,7 +446,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 #pragma unroll
           for (int y = 0; y < 4; ++y) {
             mx = fmaxf(mx, fv[y]);
-            if ((w >> 1) == ch) e[(w & 1) * 16 + xw * 4 + y] = fv[y];
+            if ((w >> 1) == b) e[(w & 1) * 16 + xw * 4 + y] = fv[y];
           }
         }
       }
@@ -441,25 +468,31 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         den = fmaf(__uint_as_float(pk << 16), __ldg(zeta + d), den);
         den = fmaf(__uint_as_float(pk & 0xFFFF0000u), __ldg(zeta + d + 1), den);
       }
+      uint8_t* const phirow = smem + kOffP + p_row * 128;  // the phi operand reuses P_0 (all P V products are done)
 #pragma unroll
       for (int i = 0; i < 4; ++i)
-        *reinterpret_cast<uint4*>(prow + chunk_off[i]) =
+        *reinterpret_cast<uint4*>(phirow + (((b * 4 + i) ^ swz) << 4)) =
             make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
       fence_proxy_async_smem();
       mbar_arrive(&bars->phi_full);
     }
 
-    // the two threads of a row swap their partial softmax sums and denominators (K stage 0 is free by now:
-    // every Q K^T product has completed before the last P V product did)
+    // the two threads of a row (one per set) swap reference maximum, row sum and partial denominator (K stage 0 is
+    // free by now: every Q K^T product has completed before the last P V products did)
+    float w_mine = 0.f, w_other = 0.f, inv_l = 0.f;
     if (ok) {
-      float2* xbuf = reinterpret_cast<float2*>(smem + kOffX);
-      xbuf[ch * 128 + p_row] = make_float2(l, den);
+      float4* xbuf = reinterpret_cast<float4*>(smem + kOffX);
+      xbuf[b * 128 + p_row] = make_float4(m_ref, l, den, 0.f);
       mbar_arrive(&bars->x_full);
       ok = mbar_wait(&bars->x_full, 0, abort_flag, p.status, 306);
       if (ok) {
-        const float2 partner = xbuf[(ch ^ 1) * 128 + p_row];
-        l += partner.x;
-        den += partner.y;
+        const float4 other = xbuf[(b ^ 1) * 128 + p_row];
+        const float m = fmaxf(m_ref, other.x);
+        w_mine = ex2(m_ref - m);    // a set without (valid) steps keeps m_ref = kNoMax and l = 0
+        w_other = ex2(other.x - m);
+        const float l_tot = w_mine * l + w_other * other.y;
+        inv_l = steps > 0 ? 1.f / l_tot : 0.f;
+        den += other.z;
       }
     }
     if (ok && p.k_marg > 0) {
@@ -469,27 +502,39 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
     if (ok) {
       const bool live = token < p.tokens && (!kPair || hf == 0 || i_q[1] != i_q[0]);
-      const int b = bh / p.heads, h = bh % p.heads;
-      float* dst = p.out + b * p.out_stride_b + h * p.out_stride_h + static_cast<long long>(token) * p.out_stride_n +
-                   ch * 32;
-      const float o_scale = steps > 0 ? 1.f / l : 0.f;
+      const int bb = bh / p.heads, h = bh % p.heads;
+      float* dst = p.out + bb * p.out_stride_b + h * p.out_stride_h + static_cast<long long>(token) * p.out_stride_n +
+                   b * 32;
+      // accumulators of a set that ran no step hold no data: they are not read
+      const bool has_mine = steps > b, has_other = steps > (b ^ 1);
       const float l_scale = p.k_marg > 0 ? 1.f / den : 0.f;
-      uint32_t o[32], ln[32];
-      if (steps > 0) tmem_ld32(lane_addr + kColO + ch * 32, o);
-      if (p.k_marg > 0) tmem_ld32(lane_addr + kColL + ch * 32, ln);
-      tmem_wait_ld();
+      const float s_mine = has_mine ? w_mine * inv_l : 0.f, s_other = has_other ? w_other * inv_l : 0.f;
+      float acc[32];
+#pragma unroll
+      for (int k = 0; k < 32; ++k) acc[k] = 0.f;
+      uint32_t v[32];
+      if (has_mine) {
+        tmem_ld32(lane_addr + kColO + b * 64 + b * 32, v);
+        tmem_wait_ld();
+#pragma unroll
+        for (int k = 0; k < 32; ++k) acc[k] = __uint_as_float(v[k]) * s_mine;
+      }
+      if (has_other) {
+        tmem_ld32(lane_addr + kColO + (b ^ 1) * 64 + b * 32, v);
+        tmem_wait_ld();
+#pragma unroll
+        for (int k = 0; k < 32; ++k) acc[k] = fmaf(__uint_as_float(v[k]), s_other, acc[k]);
+      }
+      if (p.k_marg > 0) {
+        tmem_ld32(lane_addr + kColL + b * 32, v);
+        tmem_wait_ld();
+#pragma unroll
+        for (int k = 0; k < 32; ++k) acc[k] = fmaf(__uint_as_float(v[k]), l_scale, acc[k]);
+      }
       if (live) {
 #pragma unroll
-        for (int k = 0; k < 32; k += 4) {
-          float r[4];
-#pragma unroll
-          for (int y = 0; y < 4; ++y) {
-            const float a = steps > 0 ? __uint_as_float(o[k + y]) * o_scale : 0.f;
-            const float bb = p.k_marg > 0 ? __uint_as_float(ln[k + y]) * l_scale : 0.f;
-            r[y] = a + bb;
-          }
-          *reinterpret_cast<float4*>(dst + k) = make_float4(r[0], r[1], r[2], r[3]);
-        }
+        for (int k = 0; k < 32; k += 4)
+          *reinterpret_cast<float4*>(dst + k) = make_float4(acc[k], acc[k + 1], acc[k + 2], acc[k + 3]);
       }
     }
   }
@@ -518,7 +563,6 @@ lite3r_status launch(const AttentionLaunch& a, cudaStream_t stream) {
   p.q_codes = a.q_codes;
   p.q_scales = a.q_scales;
   p.k_scales = a.k_scales;
-  p.v_scales = a.v_scales;
   p.crit_idx = a.crit_idx;
   p.zeta = a.zeta;
   p.out = a.out;
