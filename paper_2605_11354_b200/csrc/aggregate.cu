@@ -19,7 +19,7 @@ namespace {
 
 using namespace sm100;
 
-constexpr int kStages = 3;
+constexpr int kStages = 2;  // 96 KB of operand stages: two CTAs per SM, one's epilogue overlaps the other's main loop
 constexpr int kThreads = 192;
 constexpr int kTileM = 128, kTileN = 256, kChunk = 64;
 constexpr uint32_t kABytes = kTileM * kChunk * 2;   // 16 KB
@@ -36,7 +36,7 @@ struct Bars {
   int abort;
 };
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 aggregate_mma_kernel(const __grid_constant__ CUtensorMap map_s, const signed char* __restrict__ cls, int nb,
                      __nv_bfloat16* __restrict__ g16, float* __restrict__ zeta, int* status) {
   extern __shared__ __align__(1024) uint8_t smem[];

@@ -1,10 +1,11 @@
 // K1: scaled FP8 (e4m3) quantisation, one scale per (b, h, token-block) tile of Bs x 64
 // (paper appendix "Scaled FP8 Quantization"; epsilon from "Implementation Details").
 //
-// One CTA per tile.  The tile (8-32 KB) is read once into registers with 16-byte loads, the tile maximum is
-// reduced through shuffles and shared memory, then every value is divided by the scale (IEEE fp32 division,
-// so the codes equal a plain fp32 program's bit for bit), clamped, cast to e4m3 with round-to-nearest-even
-// and written with 8-byte stores.  The same pass emits the per-tile column sums of the code values as exact
+// One CTA per tile at a time (persistent CTAs).  The tile (8-32 KB) is read once into registers with 16-byte loads,
+// one tile ahead of the tile being processed; the tile maximum is
+// reduced through shuffles and shared memory, then every value is divided by the scale (with the result of an
+// IEEE fp32 division, so the codes equal a plain fp32 program's bit for bit), clamped, cast to e4m3 with
+// round-to-nearest-even and written with 8-byte stores.  The same pass emits the per-tile column sums of the code values as exact
 // integers (units of 2^-9), which is all the block plan needs.  HBM-bound: 2 (bf16) or 4 (fp32) bytes read
 // and 1 byte written per element.
 #include "common.cuh"
@@ -14,101 +15,172 @@ namespace lite3r {
 namespace {
 
 constexpr int kThreads = 256;
+// Ring depth for a tile size: about 32 KB of shared memory per CTA, at least two tiles.
+__host__ __device__ constexpr int ring_depth(int tile_bytes) { return 32768 / tile_bytes >= 2 ? 32768 / tile_bytes : 2; }
 constexpr int kRowsPerPass = kThreads / 8;  // a thread owns one 8-column segment of one row per pass
 
-__device__ __forceinline__ void load8(const float* p, float v[8]) {
-  const float4 a = __ldg(reinterpret_cast<const float4*>(p));
-  const float4 b = __ldg(reinterpret_cast<const float4*>(p) + 1);
+// Asynchronous 16-byte copy global -> shared; with src_bytes = 0 the destination is zero-filled.
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst))),
+               "l"(gsrc), "r"(src_bytes)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+__device__ __forceinline__ void unpack8(const __nv_bfloat16* p, float v[8]) {
+  const uint4 w = *reinterpret_cast<const uint4*>(p);
+  const uint32_t x[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __uint_as_float(x[i] << 16);
+    v[2 * i + 1] = __uint_as_float(x[i] & 0xFFFF0000u);
+  }
+}
+__device__ __forceinline__ void unpack8(const float* p, float v[8]) {
+  const float4 a = *reinterpret_cast<const float4*>(p);
+  const float4 b = *reinterpret_cast<const float4*>(p + 4);
   v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
   v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
 }
 
-__device__ __forceinline__ void load8(const __nv_bfloat16* p, float v[8]) {
-  const uint4 raw = __ldg(reinterpret_cast<const uint4*>(p));
-  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    v[2 * i] = __uint_as_float(w[i] << 16);
-    v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
-  }
-}
-
+// Persistent CTAs walk the tiles with a stride of the grid size.  Tiles travel global -> shared memory through
+// asynchronous copies, kDepth tiles ahead of the one being processed, so the bytes a CTA keeps in flight are set by
+// its shared-memory ring and not by its registers: that, not the arithmetic, is what the HBM rate depends on.  Every
+// thread copies and later reads only its own 8-value segments, so the ring needs no barrier.
 template <int BS, typename SrcT>
 __global__ void __launch_bounds__(kThreads) quantize_kernel(const SrcT* __restrict__ x, long long stride_b,
                                                             long long stride_h, long long stride_n, int heads,
-                                                            int tokens, int nb, uint8_t* __restrict__ codes,
+                                                            int tokens, int nb, int tiles, uint8_t* __restrict__ codes,
                                                             float* __restrict__ scales, int* __restrict__ colsum) {
   constexpr int kPasses = BS / kRowsPerPass;
+  constexpr int kSegBytes = 8 * sizeof(SrcT);                 // one thread's 8 values of one row
+  constexpr int kTileBytes = kPasses * kThreads * kSegBytes;  // = BS * 64 * sizeof(SrcT)
+  constexpr int kDepth = ring_depth(kTileBytes);
+  extern __shared__ __align__(16) uint8_t ring[];
   __shared__ float s_max[kThreads / 32];
   __shared__ int s_col[kHeadDim];
 
-  const int tile = blockIdx.x;
-  const int i = tile % nb;
-  const int bh = tile / nb;
-  const int h = bh % heads;
-  const int b = bh / heads;
-  const int valid = min(BS, tokens - i * BS);
   const int seg = threadIdx.x & 7;
   const int row0 = threadIdx.x >> 3;
+  const int stride = static_cast<int>(gridDim.x);
 
-  const SrcT* src = x + b * stride_b + h * stride_h + static_cast<long long>(i) * BS * stride_n + seg * 8;
-
-  float v[kPasses][8];
-  float amax = 0.f;
+  // Copies this thread's segments of tile `tile` into ring slot `slot` (nothing if the tile does not exist).
+  auto fetch = [&](int tile, int slot) {
+    if (tile < tiles) {
+      const int i = tile % nb;
+      const int bh = tile / nb;
+      const int valid = min(BS, tokens - i * BS);
+      const SrcT* src = x + (bh / heads) * stride_b + (bh % heads) * stride_h +
+                        static_cast<long long>(i) * BS * stride_n + seg * 8;
 #pragma unroll
-  for (int p = 0; p < kPasses; ++p) {
-    const int r = row0 + p * kRowsPerPass;
-    if (r < valid) {
-      load8(src + r * stride_n, v[p]);
-    } else {
+      for (int p = 0; p < kPasses; ++p) {
+        const int r = row0 + p * kRowsPerPass;
+        uint8_t* dst = ring + slot * kTileBytes + (p * kThreads + threadIdx.x) * kSegBytes;
+        const SrcT* g = src + (r < valid ? r : 0) * stride_n;  // rows past the end are zero-filled, not read
 #pragma unroll
-      for (int c = 0; c < 8; ++c) v[p][c] = 0.f;
-    }
-#pragma unroll
-    for (int c = 0; c < 8; ++c) amax = fmaxf(amax, fabsf(v[p][c]));
-  }
-  amax = warp_max(amax);
-  if (threadIdx.x < kHeadDim) s_col[threadIdx.x] = 0;
-  if ((threadIdx.x & 31) == 0) s_max[threadIdx.x >> 5] = amax;
-  __syncthreads();
-  amax = s_max[0];
-#pragma unroll
-  for (int w = 1; w < kThreads / 32; ++w) amax = fmaxf(amax, s_max[w]);
-
-  const float scale = __fdiv_rn(__fadd_rn(amax, 1e-8f), 448.0f);
-  if (threadIdx.x == 0) scales[tile] = scale;
-
-  int sums[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-  uint8_t* dst = codes + (static_cast<size_t>(tile) * BS) * kHeadDim + seg * 8;
-#pragma unroll
-  for (int p = 0; p < kPasses; ++p) {
-    const int r = row0 + p * kRowsPerPass;
-    uint32_t packed[2];
-#pragma unroll
-    for (int c = 0; c < 8; c += 2) {
-      float y0 = fminf(fmaxf(__fdiv_rn(v[p][c], scale), -448.0f), 448.0f);
-      float y1 = fminf(fmaxf(__fdiv_rn(v[p][c + 1], scale), -448.0f), 448.0f);
-      const uint32_t two = __nv_cvt_float2_to_fp8x2(make_float2(y0, y1), __NV_SATFINITE, __NV_E4M3);
-      sums[c] += e4m3_units(two & 0xFFu);
-      sums[c + 1] += e4m3_units(two >> 8);
-      if ((c & 2) == 0) {
-        packed[c >> 2] = two;
-      } else {
-        packed[c >> 2] |= two << 16;
+        for (int q = 0; q < kSegBytes / 16; ++q)
+          cp_async16(dst + 16 * q, reinterpret_cast<const uint8_t*>(g) + 16 * q, r < valid ? 16u : 0u);
       }
     }
-    *reinterpret_cast<uint2*>(dst + static_cast<size_t>(r) * kHeadDim) = make_uint2(packed[0], packed[1]);
-  }
-  if (colsum != nullptr) {
+    cp_async_commit();
+  };
+
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
-      int s = sums[c];
-      s += __shfl_xor_sync(0xFFFFFFFFu, s, 8);
-      s += __shfl_xor_sync(0xFFFFFFFFu, s, 16);
-      if ((threadIdx.x & 31) < 8) atomicAdd(&s_col[seg * 8 + c], s);
+  for (int d = 0; d < kDepth - 1; ++d) fetch(blockIdx.x + d * stride, d);
+
+  int slot = 0;
+  for (int tile = blockIdx.x; tile < tiles; tile += stride) {
+    fetch(tile + (kDepth - 1) * stride, (slot + kDepth - 1) % kDepth);
+    cp_async_wait<kDepth - 1>();  // all but the kDepth-1 newest groups are complete: this tile has landed
+    float v[kPasses][8];
+    float amax = 0.f;
+#pragma unroll
+    for (int p = 0; p < kPasses; ++p) {
+      unpack8(reinterpret_cast<const SrcT*>(ring + slot * kTileBytes + (p * kThreads + threadIdx.x) * kSegBytes), v[p]);
+#pragma unroll
+      for (int c = 0; c < 8; ++c) amax = fmaxf(amax, fabsf(v[p][c]));
     }
+    slot = (slot + 1) % kDepth;
+
+    amax = warp_max(amax);
+    if (threadIdx.x < kHeadDim) s_col[threadIdx.x] = 0;
+    if ((threadIdx.x & 31) == 0) s_max[threadIdx.x >> 5] = amax;
     __syncthreads();
-    if (threadIdx.x < kHeadDim) colsum[static_cast<size_t>(tile) * kHeadDim + threadIdx.x] = s_col[threadIdx.x];
+    amax = s_max[0];
+#pragma unroll
+    for (int w = 1; w < kThreads / 32; ++w) amax = fmaxf(amax, s_max[w]);
+
+    const float scale = __fdiv_rn(__fadd_rn(amax, 1e-8f), 448.0f);
+    if (threadIdx.x == 0) scales[tile] = scale;
+    // x / scale must be the IEEE quotient, but only its e4m3 rounding is kept.  The quotient lies strictly between
+    // x * r_lo and x * r_hi with r = 1 / scale widened by 2^-20 either way (the reciprocal, the product and the
+    // quotient itself are each rounded by at most 2^-24), and rounding to e4m3 is monotone: when both products give
+    // the same code, that is the code of the quotient.  Otherwise (a few elements per 10^5, next to a rounding
+    // boundary of the e4m3 grid) the group of eight is redone with the division.
+    const float r = __frcp_rn(scale);
+    const float r_lo = r * (1.0f - 0x1p-20f), r_hi = r * (1.0f + 0x1p-20f);
+
+    float sums[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};  // exact: at most four code values per column
+    uint8_t* dst = codes + (static_cast<size_t>(tile) * BS) * kHeadDim + seg * 8;
+#pragma unroll
+    for (int p = 0; p < kPasses; ++p) {
+      const int row = row0 + p * kRowsPerPass;
+      uint32_t two[4];
+      bool same = true;
+#pragma unroll
+      for (int c = 0; c < 8; c += 2) {
+        // the saturating conversion clamps to +-448 exactly like clamp-then-cast
+        const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(v[p][c] * r_lo, v[p][c + 1] * r_lo), __NV_SATFINITE, __NV_E4M3);
+        two[c >> 1] = __nv_cvt_float2_to_fp8x2(make_float2(v[p][c] * r_hi, v[p][c + 1] * r_hi), __NV_SATFINITE, __NV_E4M3);
+        same &= lo == two[c >> 1];
+      }
+      if (!same) {
+#pragma unroll
+        for (int c = 0; c < 8; c += 2)
+          two[c >> 1] = __nv_cvt_float2_to_fp8x2(make_float2(__fdiv_rn(v[p][c], scale), __fdiv_rn(v[p][c + 1], scale)),
+                                                 __NV_SATFINITE, __NV_E4M3);
+      }
+#pragma unroll
+      for (int c = 0; c < 8; c += 2) {
+        const __half2_raw back = __nv_cvt_fp8x2_to_halfraw2(static_cast<__nv_fp8x2_storage_t>(two[c >> 1]), __NV_E4M3);
+        const float2 f = __half22float2(__half2(back));
+        sums[c] += f.x;
+        sums[c + 1] += f.y;
+      }
+      *reinterpret_cast<uint2*>(dst + static_cast<size_t>(row) * kHeadDim) =
+          make_uint2(two[0] | (two[1] << 16), two[2] | (two[3] << 16));
+    }
+    if (colsum != nullptr) {
+      // Column sums over the four row groups of the warp (lanes that differ in bits 3 and 4): each exchange halves
+      // the number of columns a lane still carries, so eight columns take six shuffles instead of sixteen.
+      int s8[8];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) s8[c] = __float2int_rn(sums[c] * 512.0f);  // exact integer, units of 2^-9
+      const bool up16 = (threadIdx.x & 16) != 0, up8 = (threadIdx.x & 8) != 0;
+      int s4[4], s2[2];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {  // lanes with bit 4 clear keep columns 0-3, the others columns 4-7
+        const int give = up16 ? s8[c] : s8[c + 4];
+        const int keep = up16 ? s8[c + 4] : s8[c];
+        s4[c] = keep + __shfl_xor_sync(0xFFFFFFFFu, give, 16);
+      }
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {  // lanes with bit 3 clear keep the lower two of those
+        const int give = up8 ? s4[c] : s4[c + 2];
+        const int keep = up8 ? s4[c + 2] : s4[c];
+        s2[c] = keep + __shfl_xor_sync(0xFFFFFFFFu, give, 8);
+      }
+      const int col = seg * 8 + (up16 ? 4 : 0) + (up8 ? 2 : 0);
+      atomicAdd(&s_col[col], s2[0]);
+      atomicAdd(&s_col[col + 1], s2[1]);
+      __syncthreads();
+      if (threadIdx.x < kHeadDim) colsum[static_cast<size_t>(tile) * kHeadDim + threadIdx.x] = s_col[threadIdx.x];
+    }
+    __syncthreads();  // s_max and s_col are reused by the next tile
   }
 }
 
@@ -116,9 +188,21 @@ template <int BS, typename SrcT>
 lite3r_status launch(const lite3r_tensor& x, const lite3r_shape& s, const lite3r_fp8& out, cudaStream_t stream) {
   const int nb = ceil_div(s.tokens, BS);
   const int tiles = s.batch * s.heads * nb;
-  quantize_kernel<BS, SrcT><<<tiles, kThreads, 0, stream>>>(static_cast<const SrcT*>(x.ptr), x.stride_b, x.stride_h,
-                                                             x.stride_n, s.heads, s.tokens, nb, out.codes,
-                                                             out.scales, out.colsum);
+  constexpr int kTileBytes = BS * kHeadDim * static_cast<int>(sizeof(SrcT));
+  constexpr int kSmem = ring_depth(kTileBytes) * kTileBytes;
+  int sms = 0;
+  lite3r_status st = sm_count(&sms);
+  if (st != LITE3R_OK) return st;
+  st = record_cuda(cudaFuncSetAttribute(quantize_kernel<BS, SrcT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem));
+  if (st != LITE3R_OK) return st;
+  int per_sm = 0;
+  st = record_cuda(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, quantize_kernel<BS, SrcT>, kThreads, kSmem));
+  if (st != LITE3R_OK) return st;
+  if (per_sm < 1) per_sm = 1;
+  const int grid = tiles < sms * per_sm ? tiles : sms * per_sm;
+  quantize_kernel<BS, SrcT><<<grid, kThreads, kSmem, stream>>>(static_cast<const SrcT*>(x.ptr), x.stride_b, x.stride_h,
+                                                                x.stride_n, s.heads, s.tokens, nb, tiles, out.codes,
+                                                                out.scales, out.colsum);
   return after_launch();
 }
 
