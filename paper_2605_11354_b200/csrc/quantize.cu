@@ -14,7 +14,7 @@ namespace lite3r {
 
 namespace {
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 128;  // a thread then owns 32-64 values of a tile: the per-tile reductions cost less per value
 // Ring depth for a tile size: about 32 KB of shared memory per CTA, at least two tiles.
 __host__ __device__ constexpr int ring_depth(int tile_bytes) { return 32768 / tile_bytes >= 2 ? 32768 / tile_bytes : 2; }
 constexpr int kRowsPerPass = kThreads / 8;  // a thread owns one 8-column segment of one row per pass
@@ -68,14 +68,16 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const SrcT* __restri
   const int row0 = threadIdx.x >> 3;
   const int stride = static_cast<int>(gridDim.x);
 
-  // Copies this thread's segments of tile `tile` into ring slot `slot` (nothing if the tile does not exist).
-  auto fetch = [&](int tile, int slot) {
-    if (tile < tiles) {
-      const int i = tile % nb;
-      const int bh = tile / nb;
-      const int valid = min(BS, tokens - i * BS);
-      const SrcT* src = x + (bh / heads) * stride_b + (bh % heads) * stride_h +
-                        static_cast<long long>(i) * BS * stride_n + seg * 8;
+  // Copies this thread's segments of the next tile of the walk into ring slot `slot` (nothing once the walk has
+  // ended).  The walk's position (batch*head index and block index) advances by additions only.
+  int f_tile = blockIdx.x, f_bh = f_tile / nb, f_i = f_tile % nb;
+  const int step_bh = stride / nb, step_i = stride % nb;
+  auto fetch = [&](int slot) {
+    if (f_tile < tiles) {
+      const int valid = min(BS, tokens - f_i * BS);
+      const int b = f_bh / heads;
+      const SrcT* src = x + b * stride_b + (f_bh - b * heads) * stride_h + static_cast<long long>(f_i) * BS * stride_n +
+                        seg * 8;
 #pragma unroll
       for (int p = 0; p < kPasses; ++p) {
         const int r = row0 + p * kRowsPerPass;
@@ -87,14 +89,21 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const SrcT* __restri
       }
     }
     cp_async_commit();
+    f_tile += stride;
+    f_bh += step_bh;
+    f_i += step_i;
+    if (f_i >= nb) {
+      f_i -= nb;
+      ++f_bh;
+    }
   };
 
 #pragma unroll
-  for (int d = 0; d < kDepth - 1; ++d) fetch(blockIdx.x + d * stride, d);
+  for (int d = 0; d < kDepth - 1; ++d) fetch(d);
 
   int slot = 0;
   for (int tile = blockIdx.x; tile < tiles; tile += stride) {
-    fetch(tile + (kDepth - 1) * stride, (slot + kDepth - 1) % kDepth);
+    fetch(slot == 0 ? kDepth - 1 : slot - 1);
     cp_async_wait<kDepth - 1>();  // all but the kDepth-1 newest groups are complete: this tile has landed
     float v[kPasses][8];
     float amax = 0.f;
@@ -104,7 +113,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const SrcT* __restri
 #pragma unroll
       for (int c = 0; c < 8; ++c) amax = fmaxf(amax, fabsf(v[p][c]));
     }
-    slot = (slot + 1) % kDepth;
+    slot = slot + 1 == kDepth ? 0 : slot + 1;
 
     amax = warp_max(amax);
     if (threadIdx.x < kHeadDim) s_col[threadIdx.x] = 0;
