@@ -187,27 +187,54 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       }
       const int* list0 = p.crit_idx + (bh_rows + i_q[0]) * p.k_crit;
       const int* list1 = p.crit_idx + (bh_rows + i_q[1]) * p.k_crit;
+      // tile row (in the code tensors) of step t for query block hf
+      auto tile_row = [&](int t, int hf) {
+        if (kPair) return static_cast<int>((bh_rows + ldg_pinned((hf ? list1 : list0) + t)) * 64);
+        return static_cast<int>((bh_rows + ldg_pinned(list0 + t / 2)) * 128 + (t & 1) * 64);
+      };
+      // K and V tiles are loaded by two independent cursors: a K stage is free after the Q K^T of three steps
+      // earlier, a V stage only after that step's P V, and neither load may wait behind the other's condition.
+      // The rows of each cursor's next step are fetched one step ahead.
+      int tk = 0, tv = 0;
+      int rk[2] = {0, 0}, rv[2] = {0, 0};
+      if (steps > 0) {
+        for (int hf = 0; hf < kHalves; ++hf) rk[hf] = rv[hf] = tile_row(0, hf);
+      }
+      IdleGuard guard;
       bool ok = true;
-      for (int t = 0; t < steps && ok; ++t) {
-        const int st = t % kStages;
-        int row[2];
-        if (kPair) {
-          row[0] = static_cast<int>((bh_rows + __ldg(list0 + t)) * 64);
-          row[1] = static_cast<int>((bh_rows + __ldg(list1 + t)) * 64);
-        } else {
-          row[0] = static_cast<int>((bh_rows + __ldg(list0 + t / 2)) * 128 + (t & 1) * 64);
-          row[1] = 0;
+      while (ok && (tk < steps || tv < steps)) {
+        bool moved = false;
+        if (tk < steps) {
+          const int u = tk - kStages;
+          if (u < 0 || mbar_test(&bars->qk_done[u % kRing], (u / kRing) & 1)) {
+            const int st = tk % kStages;
+            mbar_arrive_expect_tx(&bars->k_full[st], kKTx);
+            for (int hf = 0; hf < kHalves; ++hf)
+              tma_load_2d(smem + kOffK + st * kKStage + hf * 4096, &map_k, &bars->k_full[st], 0, rk[hf]);
+            if (++tk < steps) {
+              for (int hf = 0; hf < kHalves; ++hf) rk[hf] = tile_row(tk, hf);
+            }
+            moved = true;
+          }
         }
-        // stage st was last used by step t-3: its K tile is free after that step's Q K^T, its V tile after its P V
-        const int u = t - kStages;
-        if (u >= 0 && !(ok = mbar_wait(&bars->qk_done[u % kRing], (u / kRing) & 1, abort_flag, p.status, 101, kBackoffNs))) break;
-        mbar_arrive_expect_tx(&bars->k_full[st], kKTx);
-        for (int hf = 0; hf < kHalves; ++hf)
-          tma_load_2d(smem + kOffK + st * kKStage + hf * 4096, &map_k, &bars->k_full[st], 0, row[hf]);
-        if (u >= 0 && !(ok = mbar_wait(&bars->pv_done[u % kRing], (u / kRing) & 1, abort_flag, p.status, 102, kBackoffNs))) break;
-        mbar_arrive_expect_tx(&bars->v_full[st], kVTx);
-        for (int hf = 0; hf < kHalves; ++hf)
-          tma_load_2d(smem + kOffV + st * kVStage + hf * 8192, &map_v, &bars->v_full[st], 0, row[hf]);
+        if (tv < steps) {
+          const int u = tv - kStages;
+          if (u < 0 || mbar_test(&bars->pv_done[u % kRing], (u / kRing) & 1)) {
+            const int st = tv % kStages;
+            mbar_arrive_expect_tx(&bars->v_full[st], kVTx);
+            for (int hf = 0; hf < kHalves; ++hf)
+              tma_load_2d(smem + kOffV + st * kVStage + hf * 8192, &map_v, &bars->v_full[st], 0, rv[hf]);
+            if (++tv < steps) {
+              for (int hf = 0; hf < kHalves; ++hf) rv[hf] = tile_row(tv, hf);
+            }
+            moved = true;
+          }
+        }
+        if (moved) {
+          guard.progress();
+        } else {
+          ok = guard.idle(abort_flag, p.status, 101, kBackoffNs);
+        }
       }
       if (ok && p.k_marg > 0) {
         // The aggregated summaries reuse V stage 0; it is free once the last two P V products have completed.
@@ -231,10 +258,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       const uint32_t v_addr = smem_u32(smem + kOffV), p_addr = smem_u32(smem + kOffP) + b * kPBuf;
       const uint32_t s_tmem = tmem + kColS + b * 64, o_tmem = tmem + kColO + b * 64;
       bool ok = mbar_wait(&bars->q_full, 0, abort_flag, p.status, 201, kBackoffNs);
-      auto issue_qk = [&](int t) {  // S_b = Q K(t)^T; needs the K tile and S_b drained by the softmax of step t-2
+      auto issue_qk = [&](int t) {  // S_b = Q K(t)^T
         const int st = t % kStages;
-        if (!mbar_wait(&bars->k_full[st], (t / kStages) & 1, abort_flag, p.status, 202, kBackoffNs)) return false;
-        if (!mbar_wait(&bars->s_empty[b], ((t >> 1) & 1) ^ 1, abort_flag, p.status, 203, kBackoffNs)) return false;
         tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < 2; ++kk) {
@@ -246,12 +271,9 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           }
         }
         mma_commit(&bars->qk_done[t % kRing]);
-        return true;
       };
       auto issue_pv = [&](int t) {  // O_b += P(t) V(t)
         const int st = t % kStages;
-        if (!mbar_wait(&bars->v_full[st], (t / kStages) & 1, abort_flag, p.status, 204, kBackoffNs)) return false;
-        if (!mbar_wait(&bars->p_full[b], (t >> 1) & 1, abort_flag, p.status, 205, kBackoffNs)) return false;
         tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk) {
@@ -263,14 +285,30 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           }
         }
         mma_commit(&bars->pv_done[t % kRing]);
-        return true;
       };
-      // S_b of the set's next step is produced as soon as the softmax threads have pulled the current one into
-      // registers, i.e. while they exponentiate; P V follows when they hand over the probabilities.
-      if (ok && b < steps) ok = issue_qk(b);
-      for (int t = b; t < steps && ok; t += 2) {
-        if (t + 2 < steps) ok = issue_qk(t + 2);
-        if (ok) ok = issue_pv(t);
+      // Two cursors, polled without blocking, so that neither product waits behind the other's operands:
+      //   Q K^T of step tq needs its K tile and S_b drained by the softmax of the set's previous step (tq - 2);
+      //   P V of step tp needs its V tile and the probabilities of step tp.
+      int tq = b, tp = b;
+      IdleGuard guard;
+      while (ok && tp < steps) {
+        bool moved = false;
+        if (mbar_test(&bars->p_full[b], (tp >> 1) & 1) && mbar_test(&bars->v_full[tp % kStages], (tp / kStages) & 1)) {
+          issue_pv(tp);
+          tp += 2;
+          moved = true;
+        }
+        if (tq < steps && mbar_test(&bars->k_full[tq % kStages], (tq / kStages) & 1) &&
+            mbar_test(&bars->s_empty[b], ((tq >> 1) & 1) ^ 1)) {
+          issue_qk(tq);
+          tq += 2;
+          moved = true;
+        }
+        if (moved) {
+          guard.progress();
+        } else {
+          ok = guard.idle(abort_flag, p.status, 202, 0);
+        }
       }
       if (b == 0 && ok && p.k_marg > 0) {
         ok = mbar_wait(&bars->g_full, 0, abort_flag, p.status, 206, kBackoffNs) &&

@@ -36,6 +36,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity, ui
       : "memory");
   return ok != 0;
 }
+// Non-blocking test of a phase: true when the phase with this parity has completed.
+__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 __device__ __forceinline__ uint64_t global_timer_ns() {
   uint64_t t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -70,6 +82,31 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     }
   }
 }
+
+// Bounded idling for a single-thread role that polls several barriers without blocking on any of them: call
+// idle() whenever a round of polls made no progress and progress() whenever one did.  idle() sleeps briefly and
+// returns false once nothing has moved for the wait limit or another role of the CTA (or another CTA) gave up.
+struct IdleGuard {
+  uint64_t since = 0;
+  uint32_t polls = 0;
+  __device__ __forceinline__ void progress() { polls = 0; }
+  __device__ __forceinline__ bool idle(volatile int* abort_flag, int* status, int code, uint32_t backoff_ns) {
+    if (backoff_ns != 0) __nanosleep(backoff_ns);
+    if (polls == 0) since = global_timer_ns();
+    if ((++polls & 0xFu) != 0) return true;
+    if (*abort_flag != 0) return false;
+    if (status != nullptr && *reinterpret_cast<volatile int*>(status) != 0) {
+      *abort_flag = code;
+      return false;
+    }
+    if (global_timer_ns() - since > kWaitLimitNs) {
+      *abort_flag = code;
+      if (status != nullptr) atomicCAS(status, 0, code);
+      return false;
+    }
+    return true;
+  }
+};
 
 // ------------------------------------------------------------------------------------------------ TMA
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
