@@ -1,8 +1,8 @@
 // lite3r_sla_forward_static_scratch: the SLA forward for callers that cannot hand the library any scratch buffer.
 //
 // Some hosts of this library cannot allocate device memory at the point where they call it: a plug-in running inside
-// another runtime's pre-planned arena, code executing while a stream is being captured, a real-time loop that must
-// not touch the allocator, or a process whose memory pool has already been sized to the last byte.  For them the
+// another runtime's pre-planned arena, a real-time loop that must not touch the allocator, or a process whose memory
+// pool has already been sized to the last byte.  For them the
 // forward's scratch (per-key-block summaries and per-query-block aggregates) lives in a fixed array that is part of
 // the loaded library image: every GPU that loads the library reserves LITE3R_STATIC_SCRATCH_BYTES for it until the
 // process exits.  The paper has no counterpart; this is a deployment convenience of the library.
