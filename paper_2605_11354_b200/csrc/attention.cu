@@ -54,6 +54,7 @@ constexpr uint32_t kOffQ = 0;
 constexpr uint32_t kOffK = kOffQ + kQBytes;
 constexpr uint32_t kOffV = kOffK + kStages * kKStage;
 constexpr uint32_t kOffP = kOffV + kStages * kVStage;
+constexpr uint32_t kOffG = kOffK + kKStage;  // aggregated summaries of the linear branch: K stages 1-2 (16 KB)
 constexpr uint32_t kOffBar = kOffP + 2 * kPBuf;
 constexpr uint32_t kSmemBytes = kOffBar + 256;  // two CTAs per SM: 2 * (114944 + 1024 reserved) <= 232448
 
@@ -237,13 +238,14 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
       }
       if (ok && p.k_marg > 0) {
-        // The aggregated summaries reuse V stage 0; it is free once the last two P V products have completed.
-        for (int u = max(0, steps - 2); u < steps && ok; ++u)
-          ok = mbar_wait(&bars->pv_done[u % kRing], (u / kRing) & 1, abort_flag, p.status, 103, kBackoffNs);
+        // The aggregated summaries go to K stages 1 and 2, which are free once the last three Q K^T products have
+        // completed: well before the last P V products, so this load is off the tail's critical path.
+        for (int u = max(0, steps - kStages); u < steps && ok; ++u)
+          ok = mbar_wait(&bars->qk_done[u % kRing], (u / kRing) & 1, abort_flag, p.status, 103, kBackoffNs);
         if (ok) {
           mbar_arrive_expect_tx(&bars->g_full, kHalves * 8192);
           for (int hf = 0; hf < kHalves; ++hf)
-            tma_load_2d(smem + kOffV + hf * 8192, &map_g, &bars->g_full, 0, static_cast<int>((bh_rows + i_q[hf]) * 64));
+            tma_load_2d(smem + kOffG + hf * 8192, &map_g, &bars->g_full, 0, static_cast<int>((bh_rows + i_q[hf]) * 64));
         }
       }
     }
@@ -315,13 +317,13 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
              mbar_wait(&bars->phi_full, 0, abort_flag, p.status, 207, kBackoffNs);
         if (ok) {
           tc_fence_after();
-          const uint32_t phi_addr = smem_u32(smem + kOffP);
+          const uint32_t phi_addr = smem_u32(smem + kOffP), g_addr = smem_u32(smem + kOffG);
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk) {
 #pragma unroll
             for (int hf = 0; hf < kHalves; ++hf) {
               const uint64_t a = smem_desc(phi_addr + (kPair ? hf * 8192 : 0) + kk * 32, 16, 1024, kSwizzle128);
-              const uint64_t bd = smem_desc(v_addr + hf * 8192 + kk * 32, 16, 1024, kSwizzle128);
+              const uint64_t bd = smem_desc(g_addr + hf * 8192 + kk * 32, 16, 1024, kSwizzle128);
               mma_f16(tmem + kColL + ((hf * 16u) << 16), a, bd, idesc_lin, kk);
             }
           }
@@ -460,17 +462,13 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       mbar_arrive(&bars->p_full[b]);
     }
 
-    // both sets' last P V products (the epilogue reads O_0 and O_1)
-    for (int u = max(0, steps - 2); u < steps && ok; ++u)
-      ok = mbar_wait(&bars->pv_done[u % kRing], (u / kRing) & 1, abort_flag, p.status, 304);
-    tc_fence_after();
-
     // linear branch: this thread's 32 columns (set b -> columns 32 b ..) of phi(q) as bf16 A operand, partial
-    // denominator on the side
+    // denominator on the side; computed in registers while the last P V products are still running
     float den = 0.f;
+    uint32_t phi_packed[16];
     if (ok && p.k_marg > 0) {
       const uint4* qsrc = reinterpret_cast<const uint4*>(p.q_codes + (q_tile * BS + row_in_block) * kHeadDim);
-      const float* zeta = p.zeta + q_tile * kHeadDim + b * 32;
+      const float4* zeta = reinterpret_cast<const float4*>(p.zeta + q_tile * kHeadDim + b * 32);
       float e[32];
       float mx = -INFINITY;
 #pragma unroll
@@ -489,28 +487,39 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
       }
       const float cq = sq * kLog2e, shift = mx * cq;  // sq > 0 commutes with max
-      uint32_t packed[16];
 #pragma unroll
-      for (int d = 0; d < 32; d += 2) {
-        float e0, e1;
-        if (p.phi == LITE3R_PHI_SOFTMAX) {  // the softmax normaliser cancels in the ratio
-          e0 = ex2(fmaf(e[d], cq, -shift));
-          e1 = ex2(fmaf(e[d + 1], cq, -shift));
-        } else {
-          e0 = e[d] > 0.f ? fmaf(e[d], sq, 1.f) : ex2(e[d] * cq);
-          e1 = e[d + 1] > 0.f ? fmaf(e[d + 1], sq, 1.f) : ex2(e[d + 1] * cq);
+      for (int d = 0; d < 32; d += 4) {
+        const float4 z = __ldg(zeta + (d >> 2));
+        const float zz[4] = {z.x, z.y, z.z, z.w};
+#pragma unroll
+        for (int y = 0; y < 4; y += 2) {
+          float e0, e1;
+          if (p.phi == LITE3R_PHI_SOFTMAX) {  // the softmax normaliser cancels in the ratio
+            e0 = ex2(fmaf(e[d + y], cq, -shift));
+            e1 = ex2(fmaf(e[d + y + 1], cq, -shift));
+          } else {
+            e0 = e[d + y] > 0.f ? fmaf(e[d + y], sq, 1.f) : ex2(e[d + y] * cq);
+            e1 = e[d + y + 1] > 0.f ? fmaf(e[d + y + 1], sq, 1.f) : ex2(e[d + y + 1] * cq);
+          }
+          const uint32_t pk = pack_bf162(e0, e1);
+          phi_packed[(d + y) >> 1] = pk;
+          // the denominator uses the same rounded values as the MMA's numerator
+          den = fmaf(__uint_as_float(pk << 16), zz[y], den);
+          den = fmaf(__uint_as_float(pk & 0xFFFF0000u), zz[y + 1], den);
         }
-        const uint32_t pk = pack_bf162(e0, e1);
-        packed[d >> 1] = pk;
-        // the denominator uses the same rounded values as the MMA's numerator
-        den = fmaf(__uint_as_float(pk << 16), __ldg(zeta + d), den);
-        den = fmaf(__uint_as_float(pk & 0xFFFF0000u), __ldg(zeta + d + 1), den);
       }
-      uint8_t* const phirow = smem + kOffP + p_row * 128;  // the phi operand reuses P_0 (all P V products are done)
+    }
+
+    // both sets' last P V products (the epilogue reads O_0 and O_1, and the phi operand reuses P_0)
+    for (int u = max(0, steps - 2); u < steps && ok; ++u)
+      ok = mbar_wait(&bars->pv_done[u % kRing], (u / kRing) & 1, abort_flag, p.status, 304);
+    tc_fence_after();
+    if (ok && p.k_marg > 0) {
+      uint8_t* const phirow = smem + kOffP + p_row * 128;
 #pragma unroll
       for (int i = 0; i < 4; ++i)
         *reinterpret_cast<uint4*>(phirow + (((b * 4 + i) ^ swz) << 4)) =
-            make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
+            make_uint4(phi_packed[4 * i], phi_packed[4 * i + 1], phi_packed[4 * i + 2], phi_packed[4 * i + 3]);
       fence_proxy_async_smem();
       mbar_arrive(&bars->phi_full);
     }
