@@ -55,6 +55,7 @@ constexpr uint32_t kOffK = kOffQ + kQBytes;
 constexpr uint32_t kOffV = kOffK + kStages * kKStage;
 constexpr uint32_t kOffP = kOffV + kStages * kVStage;
 constexpr uint32_t kOffG = kOffK + kKStage;  // aggregated summaries of the linear branch: K stages 1-2 (16 KB)
+constexpr uint32_t kOffZeta = kOffX + 4096;  // their denominators zeta_i (256 B per query block): rest of K stage 0
 constexpr uint32_t kOffBar = kOffP + 2 * kPBuf;
 constexpr uint32_t kSmemBytes = kOffBar + 256;  // two CTAs per SM: 2 * (114944 + 1024 reserved) <= 232448
 
@@ -243,9 +244,11 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         for (int u = max(0, steps - kStages); u < steps && ok; ++u)
           ok = mbar_wait(&bars->qk_done[u % kRing], (u / kRing) & 1, abort_flag, p.status, 103, kBackoffNs);
         if (ok) {
-          mbar_arrive_expect_tx(&bars->g_full, kHalves * 8192);
-          for (int hf = 0; hf < kHalves; ++hf)
+          mbar_arrive_expect_tx(&bars->g_full, kHalves * (8192 + 256));
+          for (int hf = 0; hf < kHalves; ++hf) {
             tma_load_2d(smem + kOffG + hf * 8192, &map_g, &bars->g_full, 0, static_cast<int>((bh_rows + i_q[hf]) * 64));
+            bulk_load(smem + kOffZeta + hf * 256, p.zeta + (bh_rows + i_q[hf]) * kHeadDim, 256, &bars->g_full);
+          }
         }
       }
     }
@@ -463,17 +466,21 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     }
 
     // linear branch: this thread's 32 columns (set b -> columns 32 b ..) of phi(q) as bf16 A operand, partial
-    // denominator on the side; computed in registers while the last P V products are still running
+    // denominator on the side; computed in registers while the last P V products are still running.  The query row
+    // comes from the Q tile in shared memory (64-byte rows, 64B swizzle: 16-byte chunk c of row r sits at chunk
+    // c ^ ((r >> 1) & 3)), zeta_i from the copy that arrived with the aggregated summaries.
     float den = 0.f;
     uint32_t phi_packed[16];
     if (ok && p.k_marg > 0) {
-      const uint4* qsrc = reinterpret_cast<const uint4*>(p.q_codes + (q_tile * BS + row_in_block) * kHeadDim);
-      const float4* zeta = reinterpret_cast<const float4*>(p.zeta + q_tile * kHeadDim + b * 32);
+      ok = mbar_wait(&bars->q_full, 0, abort_flag, p.status, 307) && mbar_wait(&bars->g_full, 0, abort_flag, p.status, 308);
+      const uint8_t* qrow = smem + kOffQ + p_row * 64;
+      const float4* zeta = reinterpret_cast<const float4*>(smem + kOffZeta + hf * 256 + b * 128);
+      const int qswz = (p_row >> 1) & 3;
       float e[32];
       float mx = -INFINITY;
 #pragma unroll
       for (int w = 0; w < 4; ++w) {
-        const uint4 raw = __ldg(qsrc + w);
+        const uint4 raw = *reinterpret_cast<const uint4*>(qrow + ((w ^ qswz) << 4));
         const uint32_t words[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
         for (int xw = 0; xw < 4; ++xw) {
@@ -489,7 +496,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       const float cq = sq * kLog2e, shift = mx * cq;  // sq > 0 commutes with max
 #pragma unroll
       for (int d = 0; d < 32; d += 4) {
-        const float4 z = __ldg(zeta + (d >> 2));
+        const float4 z = zeta[d >> 2];
         const float zz[4] = {z.x, z.y, z.z, z.w};
 #pragma unroll
         for (int y = 0; y < 4; y += 2) {
