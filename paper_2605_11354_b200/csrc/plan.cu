@@ -12,7 +12,8 @@
 //     owns one key block and R/4 rows, so every staged value feeds several fp64 FMAs.  Scores are kept in shared
 //     memory as order-preserving 64-bit keys.
 //   Phase B (one warp per row): "the k best of the row" is found by a most-significant-digit-first radix select
-//     over the 64-bit keys (8-bit digits, per-warp histogram in shared memory): it yields a key prefix such that
+//     over the 64-bit keys (8-bit digits placed at the highest bit on which the remaining candidates differ,
+//     per-warp histogram in shared memory): it yields a key prefix such that
 //     every entry above it is selected, and of the entries equal to it the first `take` in index order are.  That
 //     is exactly the total order (score descending, index ascending), at O(Nb) work per row.  Two selections
 //     give the classes: the best k_crit are critical, the best Nb - k_neg are critical-or-marginal.
@@ -24,7 +25,8 @@ namespace lite3r {
 namespace {
 
 constexpr int kChunk = 64;          // key blocks staged per pass (upper bound; the used part is keys_per_warp * R)
-constexpr int kPitch = kHeadDim + 2;  // staged row pitch in doubles: 16-byte aligned rows, conflict-free 16-byte reads
+constexpr int kPitch = kHeadDim + 4;  // staged row pitch in doubles: 16-byte aligned rows; 8-byte reads of four consecutive
+                                      // values from four (eight) rows and 16-byte reads of eight rows fall on different banks
 
 // Maps a double to an unsigned key with the same order (larger double -> larger key).
 __device__ __forceinline__ unsigned long long order_key(double v) {
@@ -54,7 +56,34 @@ __device__ Selection select_top(const unsigned long long* keys, int n, int k, un
   }
   unsigned long long prefix = 0ull, mask = 0ull;
   int remaining = k;
-  for (int shift = 56; shift >= 0; shift -= 8) {
+  while (true) {
+    // Bits on which the candidates (keys matching the prefix so far) still differ: scores of one row share their
+    // sign and leading exponent bits, so fixed digit positions would spend whole passes (and 32-way histogram
+    // conflicts) on digits that are equal for everyone.  Each pass starts at the highest differing bit instead.
+    unsigned long long all_and = ~0ull, all_or = 0ull;
+    for (int j = lane; j < n; j += 32) {
+      const unsigned long long key = keys[j];
+      if ((key & mask) == prefix) {
+        all_and &= key;
+        all_or |= key;
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      all_and &= __shfl_xor_sync(0xFFFFFFFFu, all_and, o);
+      all_or |= __shfl_xor_sync(0xFFFFFFFFu, all_or, o);
+    }
+    const unsigned long long diff = all_and ^ all_or;
+    if (diff == 0ull) {  // all candidates are equal: the first `remaining` of them by index are selected
+      prefix = all_and;
+      mask = ~0ull;
+      break;
+    }
+    const int hb = 63 - __clzll(static_cast<long long>(diff));      // highest differing bit
+    const int shift = hb >= 7 ? hb - 7 : 0;                          // digit = bits shift .. shift+7
+    const unsigned long long above_hb = hb == 63 ? 0ull : ~((2ull << hb) - 1ull);
+    prefix |= all_and & above_hb & ~mask;                            // the common leading bits join the prefix
+    mask |= above_hb;
 #pragma unroll
     for (int b = 0; b < 8; ++b) hist[lane + 32 * b] = 0u;
     __syncwarp();
@@ -96,10 +125,11 @@ __device__ Selection select_top(const unsigned long long* keys, int n, int k, un
     above = __shfl_sync(0xFFFFFFFFu, above, src);
     bin = __shfl_sync(0xFFFFFFFFu, bin, src);
     remaining -= above;
-    prefix |= static_cast<unsigned long long>(digit) << shift;
-    mask |= 0xFFull << shift;
+    const unsigned long long field = 0xFFull << shift;
+    prefix = (prefix & ~field) | (static_cast<unsigned long long>(digit) << shift);
+    mask |= field;
     __syncwarp();
-    if (bin == remaining) break;  // the whole bin is selected: lower digits cannot matter
+    if (bin == remaining || shift == 0) break;  // the whole bin is selected, or every bit has been decided
   }
   s.prefix = prefix;
   s.mask = mask;
@@ -123,8 +153,8 @@ __global__ void __launch_bounds__(R * 32) plan_kernel(const int* __restrict__ q_
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int pitch = (nb + 1) & ~1;  // key-row pitch: keeps everything behind the keys 16-byte aligned
   unsigned long long* s_key = reinterpret_cast<unsigned long long*>(smem_raw);        // [R][pitch]
-  double* s_q = reinterpret_cast<double*>(s_key + static_cast<size_t>(R) * pitch);    // [R][64]
-  double* s_k = s_q + R * kHeadDim;                                                   // [kChunk][kPitch]
+  double* s_q = reinterpret_cast<double*>(s_key + static_cast<size_t>(R) * pitch);    // [R][kPitch]
+  double* s_k = s_q + R * kPitch;                                                     // [kChunk][kPitch]
   unsigned int* s_hist = reinterpret_cast<unsigned int*>(s_k + kChunk * kPitch);      // [R][256]
 
   const int row_tiles = (nb + R - 1) / R;
@@ -135,22 +165,75 @@ __global__ void __launch_bounds__(R * 32) plan_kernel(const int* __restrict__ q_
   const size_t bh_rows = static_cast<size_t>(bh) * nb;
 
   for (int t = threadIdx.x; t < R * kHeadDim; t += kThreads) {
-    const int r = t / kHeadDim;
-    s_q[t] = (i0 + r < nb) ? static_cast<double>(q_colsum[(bh_rows + i0 + r) * kHeadDim + (t % kHeadDim)]) : 0.0;
+    const int r = t / kHeadDim, d = t % kHeadDim;
+    s_q[r * kPitch + d] = (i0 + r < nb) ? static_cast<double>(q_colsum[(bh_rows + i0 + r) * kHeadDim + d]) : 0.0;
   }
 
-  // Phase A
+  // Phase A.  The column sums of the next kStep key blocks are fetched (16-byte loads) into registers before the
+  // current ones are multiplied, so their latency hides behind the fp64 work; both staged arrays use a row pitch
+  // of 66 doubles, which keeps the 16-byte reads of the eight key rows and of the four row groups of a warp on
+  // different banks.
+  constexpr int kLoads = kStep * (kHeadDim / 4) / kThreads;  // int4 loads per thread and pass
   const int kl = lane % kKeysPerWarp, rg = lane / kKeysPerWarp;
   const int jj = warp * kKeysPerWarp + kl;
+  int4 pre[kLoads];
+  auto prefetch = [&](int j0) {
+    const int4* src = reinterpret_cast<const int4*>(k_colsum + (bh_rows + j0) * kHeadDim);
+    const int n4 = min(kStep, nb - j0) * (kHeadDim / 4);
+#pragma unroll
+    for (int q = 0; q < kLoads; ++q) {
+      const int v = threadIdx.x + q * kThreads;
+      pre[q] = v < n4 ? __ldg(src + v) : make_int4(0, 0, 0, 0);
+    }
+  };
+  prefetch(0);
+  double q_frag[R == 8 ? kHeadDim / 4 : 1] = {};
+  if constexpr (R == 8) {
+    __syncthreads();  // s_q is complete
+#pragma unroll
+    for (int st = 0; st < kHeadDim / 4; ++st) q_frag[st] = s_q[(lane >> 2) * kPitch + 4 * st + (lane & 3)];
+  }
   for (int j0 = 0; j0 < nb; j0 += kStep) {
     __syncthreads();
     const int nj = min(kStep, nb - j0);
-    for (int t = threadIdx.x; t < nj * kHeadDim; t += kThreads)
-      s_k[(t / kHeadDim) * kPitch + (t % kHeadDim)] = static_cast<double>(k_colsum[(bh_rows + j0) * kHeadDim + t]);
+#pragma unroll
+    for (int q = 0; q < kLoads; ++q) {
+      const int v = threadIdx.x + q * kThreads;
+      double* dst = s_k + (v / (kHeadDim / 4)) * kPitch + (v % (kHeadDim / 4)) * 4;
+      *reinterpret_cast<double2*>(dst) = make_double2(static_cast<double>(pre[q].x), static_cast<double>(pre[q].y));
+      *reinterpret_cast<double2*>(dst + 2) = make_double2(static_cast<double>(pre[q].z), static_cast<double>(pre[q].w));
+    }
+    if (j0 + kStep < nb) prefetch(j0 + kStep);
     __syncthreads();
-    if (jj < nj) {
+    if constexpr (R == 8) {
+      // 8 rows x 8 key blocks per warp as an fp64 tensor-core product (m8n8k4, 16 steps over the 64 columns): the
+      // integer products and sums stay below 2^53, so the result is the exact dot product whatever the order.  A
+      // lane holds A[g][t] = q row g, column 4 s + t (kept in registers for the whole kernel) and loads
+      // B[t][g] = key block g of the warp's eight, column 4 s + t; it ends with the scores of row g against key
+      // blocks 2 t and 2 t + 1.
+      const int g = lane >> 2, t4 = lane & 3;
+      const double* kr = s_k + (warp * 8 + g) * kPitch + t4;
+      double c0 = 0.0, c1 = 0.0;
+#pragma unroll
+      for (int st = 0; st < kHeadDim / 4; ++st) {
+        const double bv = kr[4 * st];
+        asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+                     : "+d"(c0), "+d"(c1)
+                     : "d"(q_frag[st]), "d"(bv));
+      }
+      const double cc[2] = {c0, c1};
+#pragma unroll
+      for (int x = 0; x < 2; ++x) {
+        const int j = j0 + warp * 8 + 2 * t4 + x;
+        if (j < nb) {
+          const int valid = min(block, tokens - j * block);
+          const double tt = cc[x] * static_cast<double>(k_scales[bh_rows + j]) / static_cast<double>(valid) + 0.0;
+          s_key[static_cast<size_t>(g) * pitch + j] = order_key(tt);
+        }
+      }
+    } else if (jj < nj) {
       const double2* kr = reinterpret_cast<const double2*>(s_k + jj * kPitch);
-      const double2* qr = reinterpret_cast<const double2*>(s_q + rg * kRowsPerLane * kHeadDim);
+      const double2* qr = reinterpret_cast<const double2*>(s_q + rg * kRowsPerLane * kPitch);
       double acc[kRowsPerLane];
 #pragma unroll
       for (int x = 0; x < kRowsPerLane; ++x) acc[x] = 0.0;
@@ -159,7 +242,7 @@ __global__ void __launch_bounds__(R * 32) plan_kernel(const int* __restrict__ q_
         const double2 kv = kr[d2];
 #pragma unroll
         for (int x = 0; x < kRowsPerLane; ++x) {
-          const double2 qv = qr[x * (kHeadDim / 2) + d2];
+          const double2 qv = qr[x * (kPitch / 2) + d2];
           acc[x] = fma(qv.x, kv.x, acc[x]);
           acc[x] = fma(qv.y, kv.y, acc[x]);
         }
@@ -213,7 +296,7 @@ __global__ void __launch_bounds__(R * 32) plan_kernel(const int* __restrict__ q_
 }
 
 size_t plan_smem_bytes(int nb, int rows) {
-  return static_cast<size_t>(rows) * ((nb + 1) & ~1) * 8 + static_cast<size_t>(rows) * kHeadDim * 8 +
+  return static_cast<size_t>(rows) * ((nb + 1) & ~1) * 8 + static_cast<size_t>(rows) * kPitch * 8 +
          static_cast<size_t>(kChunk) * kPitch * 8 + static_cast<size_t>(rows) * 256 * 4;
 }
 
