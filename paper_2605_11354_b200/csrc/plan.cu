@@ -213,15 +213,17 @@ __global__ void __launch_bounds__(R * 32) plan_kernel(const int* __restrict__ q_
       // blocks 2 t and 2 t + 1.
       const int g = lane >> 2, t4 = lane & 3;
       const double* kr = s_k + (warp * 8 + g) * kPitch + t4;
-      double c0 = 0.0, c1 = 0.0;
+      double c[2][2] = {{0.0, 0.0}, {0.0, 0.0}};  // two accumulation chains (even / odd steps) hide the MMA latency
+      double bv[kHeadDim / 4];
+#pragma unroll
+      for (int st = 0; st < kHeadDim / 4; ++st) bv[st] = kr[4 * st];
 #pragma unroll
       for (int st = 0; st < kHeadDim / 4; ++st) {
-        const double bv = kr[4 * st];
         asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
-                     : "+d"(c0), "+d"(c1)
-                     : "d"(q_frag[st]), "d"(bv));
+                     : "+d"(c[st & 1][0]), "+d"(c[st & 1][1])
+                     : "d"(q_frag[st]), "d"(bv[st]));
       }
-      const double cc[2] = {c0, c1};
+      const double cc[2] = {c[0][0] + c[1][0], c[0][1] + c[1][1]};
 #pragma unroll
       for (int x = 0; x < 2; ++x) {
         const int j = j0 + warp * 8 + 2 * t4 + x;
