@@ -29,8 +29,8 @@ constexpr int kThreads = kComputeThreads + 32;
 constexpr int kCtasPerSm = 4;
 constexpr uint32_t kTmemCols = 128;
 constexpr uint32_t kColH = 0, kColZ = 64;
-constexpr uint32_t kOffA = 0;            // phi operand, later H operand (16 KB)
-constexpr uint32_t kOffV = 16384;        // V operand (16 KB)
+constexpr uint32_t kOffA = 0;            // phi operand (16 KB)
+constexpr uint32_t kOffV = 16384;        // V operand, later H operand (16 KB)
 constexpr uint32_t kOffW = 32768;        // W operand (8 KB)
 constexpr uint32_t kOffOnes = 40960;     // ones operand (1 KB)
 constexpr uint32_t kOffBar = 41984;
@@ -139,12 +139,23 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) summary_kernel(const Sum
           for (int kk = 0; kk < kKSteps; ++kk) {
             const uint64_t a = smem_desc(a_addr + tile_off + kk * 2048, 8192, 1024, kSwizzle128);
             const uint64_t b = smem_desc(v_addr + tile_off + kk * 2048, 8192, 1024, kSwizzle128);
-            const uint64_t o = smem_desc(o_addr + (kk & 3) * 32, 16, 1024, kSwizzle128);
             mma_f16(tmem + kColH + lane_off, a, b, idesc_h, kk);
-            mma_f16(tmem + kColZ + lane_off, a, o, idesc_z, kk);
           }
         }
         mma_commit(&bars->h_done);
+        // the row sums are only needed at the end of the round: they follow the commit, and run while the compute
+        // threads already move H (into the V operand's space, which MMA 1 has finished with; phi stays intact)
+#pragma unroll
+        for (int hf = 0; hf < kTilesPerRound; ++hf) {
+          const uint32_t lane_off = (static_cast<uint32_t>(hf) * 16u) << 16;
+          const uint32_t tile_off = kTilesPerRound == 2 ? hf * 8192u : 0u;
+#pragma unroll
+          for (int kk = 0; kk < kKSteps; ++kk) {
+            const uint64_t a = smem_desc(a_addr + tile_off + kk * 2048, 8192, 1024, kSwizzle128);
+            const uint64_t o = smem_desc(o_addr + (kk & 3) * 32, 16, 1024, kSwizzle128);
+            mma_f16(tmem + kColZ + lane_off, a, o, idesc_z, kk);
+          }
+        }
         if (!(ok = mbar_wait(&bars->h_full, ph, abort_flag, p.status, 502))) break;
         tc_fence_after();
 #pragma unroll
@@ -153,7 +164,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) summary_kernel(const Sum
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk) {
             const uint64_t a = smem_desc(w_addr + kk * 2048, 8192, 1024, kSwizzle128);
-            const uint64_t b = smem_desc(a_addr + hf * 8192 + kk * 32, 16, 1024, kSwizzle128);
+            const uint64_t b = smem_desc(v_addr + hf * 8192 + kk * 32, 16, 1024, kSwizzle128);
             mma_f16(tmem + kColH + lane_off, a, b, idesc_w, kk);
           }
         }
@@ -190,6 +201,17 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) summary_kernel(const Sum
           const uint4 v4 = make_uint4(float2_to_half2_bits(x0.x, x0.y), float2_to_half2_bits(x0.z, x0.w),
                                       float2_to_half2_bits(x1.x, x1.y), float2_to_half2_bits(x1.z, x1.w));
           *reinterpret_cast<uint4*>(dst + (((half * 4 + c) ^ (e & 7)) << 4)) = v4;
+        }
+      }
+
+      // ask L2 for the rows this thread will need in the next round
+      if (r + 1 < r_end) {
+        const int nbh = (r + 1) / p.rounds_per_head;
+        const int nj = ((r + 1) % p.rounds_per_head) * kTilesPerRound + tile_tok;
+        if (nj < p.nb && s < min(BS, p.tokens - nj * BS)) {
+          const size_t off = ((static_cast<size_t>(nbh) * p.nb + nj) * BS + s) * kHeadDim;
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(p.k_codes + off));
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(p.v_codes + off));
         }
       }
 
@@ -279,7 +301,6 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) summary_kernel(const Sum
         uint32_t lo[32], hi[32];
         tmem_ld32(lane_addr + kColH, lo);
         tmem_ld32(lane_addr + kColH + 32, hi);
-        const uint32_t zbits = tmem_ld1(lane_addr + kColZ);
         tmem_wait_ld();
         tc_fence_before();
         const int j = j0 + hf;
@@ -292,8 +313,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) summary_kernel(const Sum
             hw[e >> 1] = float2_to_half2_bits(__uint_as_float(lo[e]) * sv, __uint_as_float(lo[e + 1]) * sv);
             hw[16 + (e >> 1)] = float2_to_half2_bits(__uint_as_float(hi[e]) * sv, __uint_as_float(hi[e + 1]) * sv);
           }
-          store_row_swizzled(smem + kOffA + hf * 8192, d_row, hw);
-          p.hws[tile * kSummaryRow + kHeadDim * kHeadDim + d_row] = __float2bfloat16_rn(__uint_as_float(zbits));
+          store_row_swizzled(smem + kOffV + hf * 8192, d_row, hw);
         }
       }
       fence_proxy_async_smem();
@@ -306,10 +326,12 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) summary_kernel(const Sum
         uint32_t lo[32], hi[32];
         tmem_ld32(lane_addr + kColH, lo);
         tmem_ld32(lane_addr + kColH + 32, hi);
+        const uint32_t zbits = tmem_ld1(lane_addr + kColZ);
         tmem_wait_ld();
         tc_fence_before();
         const int j = j0 + hf;
         if (acc_live && j < p.nb) {
+          p.hws[(bh_rows + j) * kSummaryRow + kHeadDim * kHeadDim + d_row] = __float2bfloat16_rn(__uint_as_float(zbits));
           uint4* dst = reinterpret_cast<uint4*>(p.hws + (bh_rows + j) * kSummaryRow + d_row * kHeadDim);
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
