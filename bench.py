@@ -111,8 +111,8 @@ def kernel_work(wl, plan):
     valid_elems = wl.batch * wl.heads * wl.tokens * wl.head_dim
     nb = wl.n_blocks
     return {
-        # three launches: read the source, write codes + scale + 64 column sums per tile
-        "quantize_x3": ("hbm", 3 * (valid_elems * src_bytes + elems + tiles * (4 + 256))),
+        # one launch for Q, K and V: read the sources, write codes + scale + 64 column sums per tile
+        "quantize_qkv": ("hbm", 3 * (valid_elems * src_bytes + elems + tiles * (4 + 256))),
         # fp64 FMAs of the pooled scores (the selection itself is integer work on top)
         "plan": ("alu_fp64", 2.0 * wl.batch * wl.heads * nb * nb * wl.head_dim),
         # read V codes, write fp16 operand
@@ -148,7 +148,7 @@ def build_roofline(wl, plan, stage_ms, peaks, peak_kind):
                        "work_per_launch": amount}
     top = max(table, key=lambda n: table[n]["ms"])
     t = table[top]
-    launches = 3 if top == "quantize_x3" else 1
+    launches = 1
     return {"kernel": top, "bound": t["bound"], "achieved": t["achieved"], "peak": t["peak"], "unit": t["unit"],
             "frac": t["frac"],
             "peak_source": (f"{peak_kind} HBM copy" if t["bound"] == "hbm" else
@@ -319,7 +319,7 @@ def run_ours(args, wl):
     e2e_flops, _ = pdist.aggregate_throughput(flops * args.steps, e2e_total / 1e3, device)
 
     peaks, peak_kind = measured_peaks()
-    stage = {"quantize_x3": quant_ms, "plan": plan_ms,
+    stage = {"quantize_qkv": quant_ms, "plan": plan_ms,
              "prep": statistics.mean(s[0] for s in stages), "summary": statistics.mean(s[1] for s in stages),
              "aggregation": statistics.mean(s[2] for s in stages), "attention": statistics.mean(s[3] for s in stages)}
     roofline = build_roofline(wl, eng.plan, stage, peaks, peak_kind)

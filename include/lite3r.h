@@ -104,6 +104,14 @@ LITE3R_API lite3r_status lite3r_forward_workspace(const lite3r_shape* shape, dou
  * Writes out.codes, out.scales and, when out.colsum is not NULL, out.colsum.  x: DEVICE source tensor. */
 LITE3R_API lite3r_status lite3r_quantize_fp8(const lite3r_tensor* x, const lite3r_shape* shape, lite3r_fp8 out, void* stream);
 
+/* The same quantisation (same passage of the paper) of Q, K and V of one attention call in a single launch: three
+ * lite3r_quantize_fp8 calls cost three launches and three pipeline fill/drain phases, which is a large share of
+ * the time at small sequence lengths.  The three sources must have the same dtype (else LITE3R_ERR_UNSUPPORTED);
+ * strides may differ.  Results are identical to three separate calls. */
+LITE3R_API lite3r_status lite3r_quantize_fp8_qkv(const lite3r_tensor* q, const lite3r_tensor* k, const lite3r_tensor* v,
+                                      const lite3r_shape* shape, lite3r_fp8 q_out, lite3r_fp8 k_out, lite3r_fp8 v_out,
+                                      void* stream);
+
 /* Pooled scores and row-wise top-k classification (Algorithm 1 lines 2-3 on block means):
  *   s_ij = mean_i(q_hat) . mean_j(k_hat) / sqrt(D), means over valid tokens of the dequantised blocks;
  *   row i ranks j by (s_ij descending, j ascending); first k_crit critical, last k_neg negligible.

@@ -45,7 +45,7 @@ class Plan(C.Structure):
 EXPORTS = ("lite3r_fp8_sizes", "lite3r_plan_sizes", "lite3r_forward_workspace", "lite3r_quantize_fp8",
            "lite3r_sla_plan", "lite3r_sla_forward", "lite3r_status_string", "lite3r_last_cuda_error",
            "lite3r_launch_count", "lite3r_profile_enable", "lite3r_profile_stage_ms",
-           "lite3r_sla_forward_static_scratch")
+           "lite3r_sla_forward_static_scratch", "lite3r_quantize_fp8_qkv")
 STATIC_SCRATCH_BYTES = 32 << 20  # LITE3R_STATIC_SCRATCH_BYTES
 
 
@@ -63,6 +63,9 @@ def lib() -> C.CDLL:
     L.lite3r_plan_sizes.argtypes = [C.POINTER(Shape), C.c_double, C.c_double, sz, sz, sz, ip, ip, ip]
     L.lite3r_forward_workspace.argtypes = [C.POINTER(Shape), C.c_double, C.c_double, sz]
     L.lite3r_quantize_fp8.argtypes = [C.POINTER(Tensor), C.POINTER(Shape), Fp8, C.c_void_p]
+    L.lite3r_quantize_fp8_qkv.argtypes = [C.POINTER(Tensor), C.POINTER(Tensor), C.POINTER(Tensor), C.POINTER(Shape), Fp8,
+                                          Fp8, Fp8, C.c_void_p]
+    L.lite3r_quantize_fp8_qkv.restype = C.c_int
     L.lite3r_sla_plan.argtypes = [C.POINTER(Fp8), C.POINTER(Fp8), C.POINTER(Shape), C.c_double, C.c_double,
                                   C.POINTER(Plan), C.c_void_p]
     L.lite3r_sla_forward.argtypes = [C.POINTER(Fp8), C.POINTER(Fp8), C.POINTER(Fp8), C.c_void_p, C.c_longlong,
@@ -191,6 +194,24 @@ def lite3r_quantize_fp8(x: torch.Tensor, shape: Shape, out: Fp8Tensor, stream=No
            "lite3r_quantize_fp8")
 
 
+def _source(x: torch.Tensor, what: str) -> Tensor:
+    if not x.is_cuda or x.dim() != 4 or x.stride(3) != 1:
+        raise Lite3rError(f"{what}: sources must be CUDA tensors [B,H,N,D] with contiguous D")
+    dtype = {torch.float32: F32, torch.bfloat16: BF16}.get(x.dtype)
+    if dtype is None:
+        raise Lite3rError(f"{what}: dtype must be float32 or bfloat16")
+    return Tensor(x.data_ptr(), dtype, x.stride(0), x.stride(1), x.stride(2))
+
+
+def lite3r_quantize_fp8_qkv(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, shape: Shape, q_out: Fp8Tensor,
+                            k_out: Fp8Tensor, v_out: Fp8Tensor, stream=None) -> None:
+    """Q, K and V of one attention call quantised by a single launch (same results as three single calls)."""
+    tq, tk, tv = (_source(x, "lite3r_quantize_fp8_qkv") for x in (q, k, v))
+    _check(lib().lite3r_quantize_fp8_qkv(C.byref(tq), C.byref(tk), C.byref(tv), C.byref(shape), q_out.c_struct(),
+                                         k_out.c_struct(), v_out.c_struct(), _stream_ptr(stream)),
+           "lite3r_quantize_fp8_qkv")
+
+
 def lite3r_sla_plan(q: Fp8Tensor, k: Fp8Tensor, shape: Shape, crit: float, neg: float, plan: PlanBuffers,
                     stream=None) -> None:
     p = plan.c_struct()
@@ -256,9 +277,12 @@ class SlaForward:
         self.status = torch.zeros(1, dtype=torch.int32, device=self.device)
 
     def quantize(self, q, k, v, stream=None):
-        lite3r_quantize_fp8(q, self.shape, self.q8, stream)
-        lite3r_quantize_fp8(k, self.shape, self.k8, stream)
-        lite3r_quantize_fp8(v, self.shape, self.v8, stream)
+        if q.dtype == k.dtype == v.dtype:
+            lite3r_quantize_fp8_qkv(q, k, v, self.shape, self.q8, self.k8, self.v8, stream)
+        else:
+            lite3r_quantize_fp8(q, self.shape, self.q8, stream)
+            lite3r_quantize_fp8(k, self.shape, self.k8, stream)
+            lite3r_quantize_fp8(v, self.shape, self.v8, stream)
 
     def make_plan(self, stream=None):
         lite3r_sla_plan(self.q8, self.k8, self.shape, self.crit, self.neg, self.plan, stream)

@@ -158,16 +158,36 @@ lite3r_status lite3r_forward_workspace(const lite3r_shape* shape, double crit, d
   return LITE3R_OK;
 }
 
-lite3r_status lite3r_quantize_fp8(const lite3r_tensor* x, const lite3r_shape* shape, lite3r_fp8 out, void* stream) {
-  lite3r_status st = check_shape(shape);
-  if (st != LITE3R_OK) return st;
+static lite3r_status check_source(const lite3r_tensor* x) {
   if (x == nullptr || x->ptr == nullptr || !aligned(x->ptr, 16)) return LITE3R_ERR_INVALID_ARG;
   if (x->dtype != LITE3R_F32 && x->dtype != LITE3R_BF16) return LITE3R_ERR_UNSUPPORTED;
   if (x->stride_n < kHeadDim || x->stride_b < 0 || x->stride_h < 0) return LITE3R_ERR_INVALID_ARG;
   if ((x->stride_b % 8) || (x->stride_h % 8) || (x->stride_n % 8)) return LITE3R_ERR_INVALID_ARG;
+  return LITE3R_OK;
+}
+
+lite3r_status lite3r_quantize_fp8(const lite3r_tensor* x, const lite3r_shape* shape, lite3r_fp8 out, void* stream) {
+  lite3r_status st = check_shape(shape);
+  if (st != LITE3R_OK) return st;
+  if ((st = check_source(x)) != LITE3R_OK) return st;
   st = check_fp8(&out, true, false);
   if (st != LITE3R_OK) return st;
-  return launch_quantize(*x, *shape, out, static_cast<cudaStream_t>(stream));
+  return launch_quantize(&x, &out, 1, *shape, static_cast<cudaStream_t>(stream));
+}
+
+lite3r_status lite3r_quantize_fp8_qkv(const lite3r_tensor* q, const lite3r_tensor* k, const lite3r_tensor* v,
+                                      const lite3r_shape* shape, lite3r_fp8 q_out, lite3r_fp8 k_out, lite3r_fp8 v_out,
+                                      void* stream) {
+  lite3r_status st = check_shape(shape);
+  if (st != LITE3R_OK) return st;
+  const lite3r_tensor* x[3] = {q, k, v};
+  const lite3r_fp8 out[3] = {q_out, k_out, v_out};
+  for (int n = 0; n < 3; ++n) {
+    if ((st = check_source(x[n])) != LITE3R_OK) return st;
+    if ((st = check_fp8(&out[n], true, false)) != LITE3R_OK) return st;
+    if (x[n]->dtype != x[0]->dtype) return LITE3R_ERR_UNSUPPORTED;
+  }
+  return launch_quantize(x, out, 3, *shape, static_cast<cudaStream_t>(stream));
 }
 
 lite3r_status lite3r_sla_plan(const lite3r_fp8* q, const lite3r_fp8* k, const lite3r_shape* shape, double crit,

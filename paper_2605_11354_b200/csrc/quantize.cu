@@ -51,11 +51,19 @@ __device__ __forceinline__ void unpack8(const float* p, float v[8]) {
 // asynchronous copies, kDepth tiles ahead of the one being processed, so the bytes a CTA keeps in flight are set by
 // its shared-memory ring and not by its registers: that, not the arithmetic, is what the HBM rate depends on.  Every
 // thread copies and later reads only its own 8-value segments, so the ring needs no barrier.
+// Up to three tensors of one shape (Q, K, V) quantised by one launch: the tiles of all of them form one walk.
+struct QuantBatch {
+  const void* x[3];
+  long long stride_b[3], stride_h[3], stride_n[3];
+  uint8_t* codes[3];
+  float* scales[3];
+  int* colsum[3];
+  int count;
+};
+
 template <int BS, typename SrcT>
-__global__ void __launch_bounds__(kThreads) quantize_kernel(const SrcT* __restrict__ x, long long stride_b,
-                                                            long long stride_h, long long stride_n, int heads,
-                                                            int tokens, int nb, int tiles, uint8_t* __restrict__ codes,
-                                                            float* __restrict__ scales, int* __restrict__ colsum) {
+__global__ void __launch_bounds__(kThreads) quantize_kernel(const __grid_constant__ QuantBatch batch, int heads, int tokens,
+                                                            int nb, int tiles) {
   constexpr int kPasses = BS / kRowsPerPass;
   constexpr int kSegBytes = 8 * sizeof(SrcT);                 // one thread's 8 values of one row
   constexpr int kTileBytes = kPasses * kThreads * kSegBytes;  // = BS * 64 * sizeof(SrcT)
@@ -69,15 +77,20 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const SrcT* __restri
   const int stride = static_cast<int>(gridDim.x);
 
   // Copies this thread's segments of the next tile of the walk into ring slot `slot` (nothing once the walk has
-  // ended).  The walk's position (batch*head index and block index) advances by additions only.
-  int f_tile = blockIdx.x, f_bh = f_tile / nb, f_i = f_tile % nb;
-  const int step_bh = stride / nb, step_i = stride % nb;
+  // ended).  A position of the walk is (tensor, tile); it advances by the grid size.
+  int f_which = 0, f_tile = blockIdx.x;
+  while (f_tile >= tiles && f_which < batch.count) {
+    f_tile -= tiles;
+    ++f_which;
+  }
   auto fetch = [&](int slot) {
-    if (f_tile < tiles) {
+    if (f_which < batch.count) {
+      const int f_bh = f_tile / nb, f_i = f_tile - f_bh * nb;
       const int valid = min(BS, tokens - f_i * BS);
       const int b = f_bh / heads;
-      const SrcT* src = x + b * stride_b + (f_bh - b * heads) * stride_h + static_cast<long long>(f_i) * BS * stride_n +
-                        seg * 8;
+      const long long stride_n = batch.stride_n[f_which];
+      const SrcT* src = static_cast<const SrcT*>(batch.x[f_which]) + b * batch.stride_b[f_which] +
+                        (f_bh - b * heads) * batch.stride_h[f_which] + static_cast<long long>(f_i) * BS * stride_n + seg * 8;
 #pragma unroll
       for (int p = 0; p < kPasses; ++p) {
         const int r = row0 + p * kRowsPerPass;
@@ -90,11 +103,9 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const SrcT* __restri
     }
     cp_async_commit();
     f_tile += stride;
-    f_bh += step_bh;
-    f_i += step_i;
-    if (f_i >= nb) {
-      f_i -= nb;
-      ++f_bh;
+    while (f_tile >= tiles && f_which < batch.count) {
+      f_tile -= tiles;
+      ++f_which;
     }
   };
 
@@ -102,7 +113,15 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const SrcT* __restri
   for (int d = 0; d < kDepth - 1; ++d) fetch(d);
 
   int slot = 0;
-  for (int tile = blockIdx.x; tile < tiles; tile += stride) {
+  int which = 0, tile = blockIdx.x;
+  while (tile >= tiles && which < batch.count) {
+    tile -= tiles;
+    ++which;
+  }
+  for (; which < batch.count;) {
+    uint8_t* const codes = batch.codes[which];
+    float* const scales = batch.scales[which];
+    int* const colsum = batch.colsum[which];
     fetch(slot == 0 ? kDepth - 1 : slot - 1);
     cp_async_wait<kDepth - 1>();  // all but the kDepth-1 newest groups are complete: this tile has landed
     float v[kPasses][8];
@@ -190,11 +209,16 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const SrcT* __restri
       if (threadIdx.x < kHeadDim) colsum[static_cast<size_t>(tile) * kHeadDim + threadIdx.x] = s_col[threadIdx.x];
     }
     __syncthreads();  // s_max and s_col are reused by the next tile
+    tile += stride;
+    while (tile >= tiles && which < batch.count) {
+      tile -= tiles;
+      ++which;
+    }
   }
 }
 
 template <int BS, typename SrcT>
-lite3r_status launch(const lite3r_tensor& x, const lite3r_shape& s, const lite3r_fp8& out, cudaStream_t stream) {
+lite3r_status launch(const QuantBatch& batch, const lite3r_shape& s, cudaStream_t stream) {
   const int nb = ceil_div(s.tokens, BS);
   const int tiles = s.batch * s.heads * nb;
   constexpr int kTileBytes = BS * kHeadDim * static_cast<int>(sizeof(SrcT));
@@ -208,21 +232,31 @@ lite3r_status launch(const lite3r_tensor& x, const lite3r_shape& s, const lite3r
   st = record_cuda(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, quantize_kernel<BS, SrcT>, kThreads, kSmem));
   if (st != LITE3R_OK) return st;
   if (per_sm < 1) per_sm = 1;
-  const int grid = tiles < sms * per_sm ? tiles : sms * per_sm;
-  quantize_kernel<BS, SrcT><<<grid, kThreads, kSmem, stream>>>(static_cast<const SrcT*>(x.ptr), x.stride_b, x.stride_h,
-                                                                x.stride_n, s.heads, s.tokens, nb, tiles, out.codes,
-                                                                out.scales, out.colsum);
+  const long long all = static_cast<long long>(tiles) * batch.count;
+  const int grid = static_cast<int>(all < static_cast<long long>(sms) * per_sm ? all : static_cast<long long>(sms) * per_sm);
+  quantize_kernel<BS, SrcT><<<grid, kThreads, kSmem, stream>>>(batch, s.heads, s.tokens, nb, tiles);
   return after_launch();
 }
 
 }  // namespace
 
-lite3r_status launch_quantize(const lite3r_tensor& x, const lite3r_shape& s, const lite3r_fp8& out,
+lite3r_status launch_quantize(const lite3r_tensor* const* x, const lite3r_fp8* out, int count, const lite3r_shape& s,
                               cudaStream_t stream) {
-  if (x.dtype == LITE3R_BF16) {
-    return s.block == 64 ? launch<64, __nv_bfloat16>(x, s, out, stream) : launch<128, __nv_bfloat16>(x, s, out, stream);
+  QuantBatch batch = {};
+  batch.count = count;
+  for (int n = 0; n < count; ++n) {
+    batch.x[n] = x[n]->ptr;
+    batch.stride_b[n] = x[n]->stride_b;
+    batch.stride_h[n] = x[n]->stride_h;
+    batch.stride_n[n] = x[n]->stride_n;
+    batch.codes[n] = out[n].codes;
+    batch.scales[n] = out[n].scales;
+    batch.colsum[n] = out[n].colsum;
   }
-  return s.block == 64 ? launch<64, float>(x, s, out, stream) : launch<128, float>(x, s, out, stream);
+  if (x[0]->dtype == LITE3R_BF16) {
+    return s.block == 64 ? launch<64, __nv_bfloat16>(batch, s, stream) : launch<128, __nv_bfloat16>(batch, s, stream);
+  }
+  return s.block == 64 ? launch<64, float>(batch, s, stream) : launch<128, float>(batch, s, stream);
 }
 
 }  // namespace lite3r

@@ -96,6 +96,26 @@ def test_fp32_source_and_strided_layout():
     assert np.array_equal(alt.scales.cpu().numpy(), scales)
 
 
+def test_qkv_launch_matches_single_launches():
+    """lite3r_quantize_fp8_qkv (one launch for Q, K, V, different strides) is bit-identical to three single calls."""
+    wl = small_workload("qkv", tokens=1111, batch=2, heads=3)
+    inputs = wk.make_inputs(wl)
+    shape = lt.Shape(wl.batch, wl.heads, wl.tokens, 64, wl.block)
+    q, k, v = (pu.to_device(inputs[n], wl.src_dtype) for n in ("q", "k", "v"))
+    k = k.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)  # token-major strides for one of the three
+    single = [lt.alloc_fp8(shape, "cuda:0") for _ in range(3)]
+    for x, out in zip((q, k, v), single):
+        lt.lite3r_quantize_fp8(x, shape, out)
+    fused = [lt.alloc_fp8(shape, "cuda:0") for _ in range(3)]
+    lt.lite3r_quantize_fp8_qkv(q, k, v, shape, *fused)
+    torch.cuda.synchronize()
+    for a, b in zip(single, fused):
+        assert torch.equal(a.codes, b.codes) and torch.equal(a.scales, b.scales) and torch.equal(a.colsum, b.colsum)
+    codes, scales = orc.quantize_fp8_blocks(inputs["v"], wl.block)
+    assert np.array_equal(fused[2].codes.cpu().numpy(), codes)
+    assert np.array_equal(fused[2].scales.cpu().numpy().view(np.uint32), scales.view(np.uint32))
+
+
 def test_quantizer_extremes():
     """All-zero tile, a single huge outlier, tiny magnitudes, negative zero: codes and scales bit-exact."""
     g = np.random.default_rng(5)
