@@ -195,3 +195,26 @@ def test_stress_sweep_on_sampled_blocks(crit, neg):
     inputs = wk.make_inputs(wl)
     qb = pu.sample_blocks(wl, [0], 12, seed=17)
     full_parity(wl, inputs, heads=[9], crit=crit, neg=neg, query_blocks=qb)
+
+
+def test_stress_dense_equivalent_point():
+    """Critical fraction 1.0 at 137 400 tokens: every key block is critical, the sparse branch is dense attention
+    (2147 key steps per query tile) and the linear branch vanishes."""
+    wl = wk.WORKLOADS["stress100"]
+    inputs = wk.make_inputs(wl)
+    qb = pu.sample_blocks(wl, [0], 4, seed=23)
+    full_parity(wl, inputs, heads=[4], crit=1.0, neg=0.0, query_blocks=qb)
+
+
+def test_token_major_output_layout():
+    """The output may be a [B, N, H, D] buffer viewed as [B, H, N, D]: only the strides change."""
+    wl = small_workload("out-strides", tokens=450, batch=2, heads=3)
+    inputs = wk.make_inputs(wl)
+    eng, out = pu.run_gpu(inputs, wl)
+    proj = torch.from_numpy(inputs["proj"]).cuda()
+    buf = torch.full((wl.batch, wl.tokens, wl.heads, 64), float("nan"), device="cuda")
+    view = buf.permute(0, 2, 1, 3)
+    lt.lite3r_sla_forward(eng.q8, eng.k8, eng.v8, proj, eng.shape, eng.phi, eng.plan, view, eng.workspace, eng.status)
+    torch.cuda.synchronize()
+    assert int(eng.status.item()) == 0
+    assert torch.equal(view, out)
