@@ -167,6 +167,13 @@ LITE3R_API lite3r_status lite3r_sla_forward_static_scratch(const lite3r_fp8* q, 
                                                 float* out, long long out_stride_b, long long out_stride_h,
                                                 long long out_stride_n, int* device_status, void* stream);
 
+/* Self-test of the device-side wait bound.  Every wait inside the kernels (on an mbarrier, or a polling loop of a
+ * single-thread role) gives up after one second, records a non-zero code in device_status and lets the kernel end, so a
+ * lost signal can never hang the GPU.  This call runs that mechanism on purpose and harmlessly: a one-thread kernel
+ * waits, with the given limit (nanoseconds, at most 1e9), on a barrier that nothing arrives on.  After synchronising,
+ * *device_status (DEVICE int) must be non-zero (999) and the context must still be usable. */
+LITE3R_API lite3r_status lite3r_selftest_wait_expiry(int* device_status, unsigned long long limit_ns, void* stream);
+
 /* Text for a status code; the last CUDA error code (cudaError_t as int) recorded by this thread. */
 LITE3R_API const char* lite3r_status_string(lite3r_status status);
 LITE3R_API int lite3r_last_cuda_error(void);

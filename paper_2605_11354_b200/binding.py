@@ -45,7 +45,7 @@ class Plan(C.Structure):
 EXPORTS = ("lite3r_fp8_sizes", "lite3r_plan_sizes", "lite3r_forward_workspace", "lite3r_quantize_fp8",
            "lite3r_sla_plan", "lite3r_sla_forward", "lite3r_status_string", "lite3r_last_cuda_error",
            "lite3r_launch_count", "lite3r_profile_enable", "lite3r_profile_stage_ms",
-           "lite3r_sla_forward_static_scratch", "lite3r_quantize_fp8_qkv")
+           "lite3r_sla_forward_static_scratch", "lite3r_quantize_fp8_qkv", "lite3r_selftest_wait_expiry")
 STATIC_SCRATCH_BYTES = 32 << 20  # LITE3R_STATIC_SCRATCH_BYTES
 
 
@@ -76,6 +76,8 @@ def lib() -> C.CDLL:
                                                     C.c_void_p, C.c_longlong, C.c_longlong, C.c_longlong, C.c_void_p,
                                                     C.c_void_p]
     L.lite3r_sla_forward_static_scratch.restype = C.c_int
+    L.lite3r_selftest_wait_expiry.argtypes = [C.c_void_p, C.c_ulonglong, C.c_void_p]
+    L.lite3r_selftest_wait_expiry.restype = C.c_int
     L.lite3r_status_string.argtypes = [C.c_int]
     L.lite3r_status_string.restype = C.c_char_p
     L.lite3r_last_cuda_error.restype = C.c_int
@@ -101,6 +103,12 @@ def _check(status: int, what: str) -> None:
 def _stream_ptr(stream) -> int:
     s = stream if stream is not None else torch.cuda.current_stream()
     return int(s.cuda_stream)
+
+
+def selftest_wait_expiry(status: torch.Tensor, limit_ns: int, stream=None) -> None:
+    """Runs the bounded-wait self-test kernel; `status` (CUDA int32 [1]) is non-zero afterwards."""
+    _check(lib().lite3r_selftest_wait_expiry(status.data_ptr(), limit_ns, _stream_ptr(stream)),
+           "lite3r_selftest_wait_expiry")
 
 
 def launch_count() -> int:

@@ -249,6 +249,11 @@ lite3r_status lite3r_sla_forward(const lite3r_fp8* q, const lite3r_fp8* k, const
   return launch_forward(a, static_cast<cudaStream_t>(stream));
 }
 
+lite3r_status lite3r_selftest_wait_expiry(int* device_status, unsigned long long limit_ns, void* stream) {
+  if (device_status == nullptr || limit_ns == 0 || limit_ns > 1000000000ull) return LITE3R_ERR_INVALID_ARG;
+  return launch_wait_expiry_probe(device_status, limit_ns, static_cast<cudaStream_t>(stream));
+}
+
 lite3r_status lite3r_profile_enable(int enable) {
   if (enable && !g_profile) {
     for (cudaEvent_t& e : g_events) {

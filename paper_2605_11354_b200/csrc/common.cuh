@@ -119,6 +119,7 @@ lite3r_status make_tensor_map_2d(CUtensorMap* map, CUtensorMapDataType type, int
                                  uint64_t inner, uint64_t rows, uint32_t box_inner, uint32_t box_rows,
                                  CUtensorMapSwizzle swizzle);
 
+lite3r_status launch_wait_expiry_probe(int* status, unsigned long long limit_ns, cudaStream_t stream);
 size_t forward_workspace_bytes(const lite3r_shape& s, const Counts& c);
 lite3r_status launch_forward(const ForwardArgs& a, cudaStream_t stream);
 

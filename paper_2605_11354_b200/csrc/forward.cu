@@ -10,6 +10,7 @@
 #include <algorithm>
 
 #include "common.cuh"
+#include "sm100.cuh"
 
 namespace lite3r {
 
@@ -36,6 +37,19 @@ __global__ void __launch_bounds__(256) prep_kernel(const uint8_t* __restrict__ v
     uint4* dst = reinterpret_cast<uint4*>(v16) + 2 * w;
     dst[0] = make_uint4(out[0], out[1], out[2], out[3]);
     dst[1] = make_uint4(out[4], out[5], out[6], out[7]);
+  }
+}
+
+// Self-test of the bounded waits: one thread waits on a barrier that nothing ever arrives on.  The wait must give up
+// after limit_ns, write its code to *status and let the kernel end normally.
+__global__ void wait_expiry_probe_kernel(int* status, unsigned long long limit_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    sm100::mbar_init(&bar, 1);
+    abort_flag = 0;
+    sm100::mbar_fence_init();
+    sm100::mbar_wait(&bar, 0, &abort_flag, status, 999, 0, limit_ns);
   }
 }
 
@@ -119,6 +133,13 @@ lite3r_status run_forward(const ForwardArgs& a, cudaStream_t stream) {
 }
 
 }  // namespace
+
+lite3r_status launch_wait_expiry_probe(int* status, unsigned long long limit_ns, cudaStream_t stream) {
+  lite3r_status st = record_cuda(cudaMemsetAsync(status, 0, sizeof(int), stream));
+  if (st != LITE3R_OK) return st;
+  wait_expiry_probe_kernel<<<1, 32, 0, stream>>>(status, limit_ns);
+  return after_launch();
+}
 
 size_t forward_workspace_bytes(const lite3r_shape& s, const Counts& c) {
   (void)c;

@@ -61,7 +61,7 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 // polling does not take issue slots from the working warps.
 constexpr uint64_t kWaitLimitNs = 1000000000ull;  // 1 s
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                          int code, uint32_t backoff_ns = 0) {
+                                          int code, uint32_t backoff_ns = 0, uint64_t limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   uint32_t polls = 0;
@@ -74,7 +74,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
         *abort_flag = code;
         return false;
       }
-      if (global_timer_ns() - t0 > kWaitLimitNs) {
+      if (global_timer_ns() - t0 > limit_ns) {
         *abort_flag = code;
         if (status != nullptr) atomicCAS(status, 0, code);
         return false;

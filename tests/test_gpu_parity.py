@@ -218,3 +218,19 @@ def test_token_major_output_layout():
     torch.cuda.synchronize()
     assert int(eng.status.item()) == 0
     assert torch.equal(view, out)
+
+
+def test_device_waits_are_bounded():
+    """A wait that can never be satisfied gives up after its limit, reports through device_status and leaves the
+    context usable (the forward still runs and matches afterwards)."""
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    lt.selftest_wait_expiry(status, 2_000_000)  # 2 ms
+    t1.record()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 999
+    assert 1.0 <= t0.elapsed_time(t1) < 200.0
+    wl = wk.WORKLOADS["tiny"]
+    full_parity(wl, wk.make_inputs(wl))
