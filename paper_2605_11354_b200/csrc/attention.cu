@@ -345,7 +345,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const size_t q_tile = bh_rows + iq;
     const uint32_t lane_addr = tmem + ((static_cast<uint32_t>(quarter) * 32u) << 16);
     const uint32_t s_addr = lane_addr + kColS + b * 64, o_addr = lane_addr + kColO + b * 64;
-    const int token = iq * BS + row_in_block;
     const float sq = __ldg(p.q_scales + q_tile);
     const float qk_scale = sq * (kLog2e * 0.125f);
     const int* list = p.crit_idx + q_tile * p.k_crit;
@@ -554,11 +553,9 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       tc_fence_after();
     }
 
+    ok = __all_sync(0xFFFFFFFFu, ok);  // the store below synchronises the warp
     if (ok) {
-      const bool live = token < p.tokens && (!kPair || hf == 0 || i_q[1] != i_q[0]);
       const int bb = bh / p.heads, h = bh % p.heads;
-      float* dst = p.out + bb * p.out_stride_b + h * p.out_stride_h + static_cast<long long>(token) * p.out_stride_n +
-                   b * 32;
       // accumulators of a set that ran no step hold no data: they are not read
       const bool has_mine = steps > b, has_other = steps > (b ^ 1);
       const float l_scale = p.k_marg > 0 ? 1.f / den : 0.f;
@@ -585,10 +582,27 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 #pragma unroll
         for (int k = 0; k < 32; ++k) acc[k] = fmaf(__uint_as_float(v[k]), l_scale, acc[k]);
       }
-      if (live) {
+      // A thread owns 128 bytes of one output row, so a direct store would touch 32 different lines per instruction.
+      // The warp's 32 x 128-byte block is turned around in its own rows of P_b (free: P V products and the linear
+      // product have completed) so that every store instruction writes four whole 128-byte row segments.
 #pragma unroll
-        for (int k = 0; k < 32; k += 4)
-          *reinterpret_cast<float4*>(dst + k) = make_float4(acc[k], acc[k + 1], acc[k + 2], acc[k + 3]);
+      for (int ch = 0; ch < 8; ++ch)
+        *reinterpret_cast<float4*>(prow + ((ch ^ swz) << 4)) =
+            make_float4(acc[4 * ch], acc[4 * ch + 1], acc[4 * ch + 2], acc[4 * ch + 3]);
+      __syncwarp();
+      const int ch = lane & 7;
+      float* const out_bh = p.out + bb * p.out_stride_b + h * p.out_stride_h + b * 32 + ch * 4;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int r = 4 * k + (lane >> 3);  // row of this warp's block: the one thread `r` of the warp computed
+        const int r_hf = kPair ? (r >> 4) : 0;
+        const int r_in_block = kPair ? quarter * 16 + (r & 15) : quarter * 32 + r;
+        const int r_p = kPair ? r_hf * 64 + r_in_block : r_in_block;
+        const int r_token = i_q[r_hf] * BS + r_in_block;
+        const float4 val =
+            *reinterpret_cast<const float4*>(smem + kOffP + b * kPBuf + r_p * 128 + ((ch ^ (r_p & 7)) << 4));
+        if (r_token < p.tokens && (!kPair || r_hf == 0 || i_q[1] != i_q[0]))
+          *reinterpret_cast<float4*>(out_bh + static_cast<long long>(r_token) * p.out_stride_n) = val;
       }
     }
   }
