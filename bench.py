@@ -118,8 +118,8 @@ def kernel_work(wl, plan):
     valid_elems = wl.batch * wl.heads * wl.tokens * wl.head_dim
     nb = wl.n_blocks
     return {
-        # one launch for Q, K and V: read the sources, write codes + scale + 64 column sums per tile
-        "quantize_qkv": ("hbm", 3 * (valid_elems * src_bytes + elems + tiles * (4 + 256))),
+        # one launch for Q, K and V: read the sources, write codes + scale per tile, 64 column sums per Q and K tile
+        "quantize_qkv": ("hbm", 3 * (valid_elems * src_bytes + elems + tiles * 4) + 2 * tiles * 256),
         # fp64 FMAs of the pooled scores (the selection itself is integer work on top)
         "plan": ("alu_fp64", 2.0 * wl.batch * wl.heads * nb * nb * wl.head_dim),
         # read V codes, write fp16 operand

@@ -152,10 +152,11 @@ def lite3r_forward_workspace(shape: Shape, crit: float, neg: float) -> int:
 class Fp8Tensor:
     codes: torch.Tensor  # uint8 [B,H,Nb*Bs,D]
     scales: torch.Tensor  # fp32 [B,H,Nb]
-    colsum: torch.Tensor  # int32 [B,H,Nb,D]
+    colsum: torch.Tensor | None  # int32 [B,H,Nb,D]; None: the quantiser skips the column sums (only Q and K need them)
 
     def c_struct(self) -> Fp8:
-        return Fp8(self.codes.data_ptr(), self.scales.data_ptr(), self.colsum.data_ptr())
+        return Fp8(self.codes.data_ptr(), self.scales.data_ptr(),
+                   self.colsum.data_ptr() if self.colsum is not None else None)
 
 
 @dataclass
@@ -172,12 +173,12 @@ class PlanBuffers:
                     self.marg_idx.data_ptr() if self.k_marg else None, self.k_crit, self.k_marg, self.k_neg)
 
 
-def alloc_fp8(shape: Shape, device) -> Fp8Tensor:
+def alloc_fp8(shape: Shape, device, colsum: bool = True) -> Fp8Tensor:
     nb = -(-shape.tokens // shape.block)
     B, H, D = shape.batch, shape.heads, shape.head_dim
     return Fp8Tensor(torch.empty((B, H, nb * shape.block, D), dtype=torch.uint8, device=device),
                      torch.empty((B, H, nb), dtype=torch.float32, device=device),
-                     torch.empty((B, H, nb, D), dtype=torch.int32, device=device))
+                     torch.empty((B, H, nb, D), dtype=torch.int32, device=device) if colsum else None)
 
 
 def alloc_plan(shape: Shape, crit: float, neg: float, device) -> PlanBuffers:
@@ -275,7 +276,8 @@ class SlaForward:
         self.shape = Shape(batch, heads, tokens, head_dim, block)
         self.crit, self.neg, self.phi = float(crit), float(neg), PHI_CODES[phi]
         self.device = torch.device(device)
-        self.q8, self.k8, self.v8 = (alloc_fp8(self.shape, self.device) for _ in range(3))
+        self.q8, self.k8 = (alloc_fp8(self.shape, self.device) for _ in range(2))
+        self.v8 = alloc_fp8(self.shape, self.device, colsum=False)  # the block plan pools Q and K only
         self.plan = alloc_plan(self.shape, self.crit, self.neg, self.device)
         nbytes = lite3r_forward_workspace(self.shape, self.crit, self.neg)
         self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)

@@ -1,23 +1,41 @@
 // K1: scaled FP8 (e4m3) quantisation, one scale per (b, h, token-block) tile of Bs x 64
 // (paper appendix "Scaled FP8 Quantization"; epsilon from "Implementation Details").
 //
-// One CTA per tile at a time (persistent CTAs).  The tile (8-32 KB) is read once into registers with 16-byte loads,
-// one tile ahead of the tile being processed; the tile maximum is
+// One CTA per tile at a time (persistent CTAs of 64 or 128 threads, 64 values per thread).  Tiles travel global ->
+// shared memory by asynchronous 16-byte copies, a few tiles ahead of the one being processed; the tile maximum is
 // reduced through shuffles and shared memory, then every value is divided by the scale (with the result of an
 // IEEE fp32 division, so the codes equal a plain fp32 program's bit for bit), clamped, cast to e4m3 with
-// round-to-nearest-even and written with 8-byte stores.  The same pass emits the per-tile column sums of the code values as exact
-// integers (units of 2^-9), which is all the block plan needs.  HBM-bound: 2 (bf16) or 4 (fp32) bytes read
-// and 1 byte written per element.
+// round-to-nearest-even and written with 8-byte stores.  The same pass emits, where asked for, the per-tile column
+// sums of the code values as exact integers (units of 2^-9), which is all the block plan needs.  HBM traffic: 2
+// (bf16) or 4 (fp32) bytes read and 1 byte written per element; the instruction count per element decides how
+// close the kernel gets to that, hence the packed fp32x2 arithmetic and the bf16 maximum taken on bit patterns.
+// Sources are expected to be finite (a NaN would become the tile maximum).
 #include "common.cuh"
+#include "sm100.cuh"
 
 namespace lite3r {
 
 namespace {
 
-constexpr int kThreads = 128;  // a thread then owns 32-64 values of a tile: the per-tile reductions cost less per value
-// Ring depth for a tile size: about 32 KB of shared memory per CTA, at least two tiles.
-__host__ __device__ constexpr int ring_depth(int tile_bytes) { return 32768 / tile_bytes >= 2 ? 32768 / tile_bytes : 2; }
-constexpr int kRowsPerPass = kThreads / 8;  // a thread owns one 8-column segment of one row per pass
+using sm100::add_f32x2;
+using sm100::fma_f32x2;
+using sm100::pack_f32x2;
+using sm100::unpack_f32x2;
+
+#ifndef LITE3R_QUANT_THREADS_SMALL
+#define LITE3R_QUANT_THREADS_SMALL 64
+#endif
+constexpr int kQuantThreadsSmall = LITE3R_QUANT_THREADS_SMALL;  // CTA size for 8 KB tiles
+
+// Threads per CTA (= per tile).  The per-tile work that does not shrink with the tile (address arithmetic, the two
+// reductions, barriers) is paid per thread, so few threads with many values each keep the instruction count per
+// value low: the kernel is otherwise bound by instruction issue, not by HBM.
+__host__ __device__ constexpr int cta_threads(int tile_bytes) { return tile_bytes <= 8192 ? kQuantThreadsSmall : 128; }
+// Ring depth for a tile size and CTA size: enough CTAs per SM to cover the arithmetic, at least two tiles each.
+__host__ __device__ constexpr int ring_depth(int tile_bytes, int threads) {
+  const int budget = threads * 256;
+  return budget / tile_bytes >= 2 ? budget / tile_bytes : 2;
+}
 
 // Asynchronous 16-byte copy global -> shared; with src_bytes = 0 the destination is zero-filled.
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc, uint32_t src_bytes) {
@@ -47,6 +65,16 @@ __device__ __forceinline__ void unpack8(const float* p, float v[8]) {
   v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
 }
 
+// Largest magnitude of eight values as a float.  bf16 magnitudes are ordered like their bit patterns, so two of them
+// are compared per 16-bit-pair instruction before anything is unpacked.
+__device__ __forceinline__ uint32_t amax8_bits(const __nv_bfloat16* p, uint32_t acc) {
+  const uint4 w = *reinterpret_cast<const uint4*>(p);
+  acc = __vmaxu2(acc, __vmaxu2(w.x & 0x7FFF7FFFu, w.y & 0x7FFF7FFFu));
+  return __vmaxu2(acc, __vmaxu2(w.z & 0x7FFF7FFFu, w.w & 0x7FFF7FFFu));
+}
+__device__ __forceinline__ uint32_t amax8_bits(const float*, uint32_t acc) { return acc; }  // fp32 sources compare as floats
+__device__ __forceinline__ float amax_finish(uint32_t acc) { return __uint_as_float(max(acc << 16, acc & 0xFFFF0000u)); }
+
 // Persistent CTAs walk the tiles with a stride of the grid size.  Tiles travel global -> shared memory through
 // asynchronous copies, kDepth tiles ahead of the one being processed, so the bytes a CTA keeps in flight are set by
 // its shared-memory ring and not by its registers: that, not the arithmetic, is what the HBM rate depends on.  Every
@@ -61,15 +89,17 @@ struct QuantBatch {
   int count;
 };
 
-template <int BS, typename SrcT>
+template <int BS, typename SrcT, int kThreads>
 __global__ void __launch_bounds__(kThreads) quantize_kernel(const __grid_constant__ QuantBatch batch, int heads, int tokens,
                                                             int nb, int tiles) {
+  constexpr int kRowsPerPass = kThreads / 8;  // a thread owns one 8-column segment of one row per pass
   constexpr int kPasses = BS / kRowsPerPass;
+  constexpr bool kKeep = kPasses <= 8;  // the tile stays in registers between the two sweeps, else it is re-read
   constexpr int kSegBytes = 8 * sizeof(SrcT);                 // one thread's 8 values of one row
   constexpr int kTileBytes = kPasses * kThreads * kSegBytes;  // = BS * 64 * sizeof(SrcT)
-  constexpr int kDepth = ring_depth(kTileBytes);
+  constexpr int kDepth = ring_depth(kTileBytes, kThreads);
   extern __shared__ __align__(16) uint8_t ring[];
-  __shared__ float s_max[kThreads / 32];
+  __shared__ float s_max[(kThreads + 31) / 32];
   __shared__ int s_col[kHeadDim];
 
   const int seg = threadIdx.x & 7;
@@ -124,23 +154,40 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const __grid_constan
     int* const colsum = batch.colsum[which];
     fetch(slot == 0 ? kDepth - 1 : slot - 1);
     cp_async_wait<kDepth - 1>();  // all but the kDepth-1 newest groups are complete: this tile has landed
-    float v[kPasses][8];
+    float v[kKeep ? kPasses : 1][8];
+    const uint8_t* const mine = ring + slot * kTileBytes + threadIdx.x * kSegBytes;
     float amax = 0.f;
+    if (sizeof(SrcT) == 2) {
+      uint32_t acc = 0;
 #pragma unroll
-    for (int p = 0; p < kPasses; ++p) {
-      unpack8(reinterpret_cast<const SrcT*>(ring + slot * kTileBytes + (p * kThreads + threadIdx.x) * kSegBytes), v[p]);
+      for (int p = 0; p < kPasses; ++p) {
+        const SrcT* const src = reinterpret_cast<const SrcT*>(mine + p * kThreads * kSegBytes);
+        acc = amax8_bits(src, acc);
+        if (kKeep) unpack8(src, v[kKeep ? p : 0]);
+      }
+      amax = amax_finish(acc);
+    } else {
 #pragma unroll
-      for (int c = 0; c < 8; ++c) amax = fmaxf(amax, fabsf(v[p][c]));
+      for (int p = 0; p < kPasses; ++p) {
+        float* const vp = v[kKeep ? p : 0];
+        unpack8(reinterpret_cast<const SrcT*>(mine + p * kThreads * kSegBytes), vp);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) amax = fmaxf(amax, fabsf(vp[c]));
+      }
     }
     slot = slot + 1 == kDepth ? 0 : slot + 1;
 
     amax = warp_max(amax);
-    if (threadIdx.x < kHeadDim) s_col[threadIdx.x] = 0;
-    if ((threadIdx.x & 31) == 0) s_max[threadIdx.x >> 5] = amax;
-    __syncthreads();
-    amax = s_max[0];
+    for (int c = threadIdx.x; c < kHeadDim; c += kThreads) s_col[c] = 0;
+    if (kThreads > 32) {
+      if ((threadIdx.x & 31) == 0) s_max[threadIdx.x >> 5] = amax;
+      __syncthreads();
+      amax = s_max[0];
 #pragma unroll
-    for (int w = 1; w < kThreads / 32; ++w) amax = fmaxf(amax, s_max[w]);
+      for (int w = 1; w < kThreads / 32; ++w) amax = fmaxf(amax, s_max[w]);
+    } else {
+      __syncwarp();
+    }
 
     const float scale = __fdiv_rn(__fadd_rn(amax, 1e-8f), 448.0f);
     if (threadIdx.x == 0) scales[tile] = scale;
@@ -152,32 +199,41 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const __grid_constan
     const float r = __frcp_rn(scale);
     const float r_lo = r * (1.0f - 0x1p-20f), r_hi = r * (1.0f + 0x1p-20f);
 
-    float sums[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};  // exact: at most four code values per column
+    // fp32 sums of code values are exact (at most 16 values of at most 448 in units of 2^-9: 22 bits); two columns
+    // per packed-pair instruction, like the two products
+    uint64_t sums2[4] = {0ull, 0ull, 0ull, 0ull};
+    const uint64_t r_lo2 = pack_f32x2(r_lo, r_lo), r_hi2 = pack_f32x2(r_hi, r_hi), neg0 = pack_f32x2(-0.f, -0.f);
     uint8_t* dst = codes + (static_cast<size_t>(tile) * BS) * kHeadDim + seg * 8;
 #pragma unroll
     for (int p = 0; p < kPasses; ++p) {
       const int row = row0 + p * kRowsPerPass;
+      float* const vp = v[kKeep ? p : 0];
+      if (!kKeep) unpack8(reinterpret_cast<const SrcT*>(mine + p * kThreads * kSegBytes), vp);
       uint32_t two[4];
       bool same = true;
 #pragma unroll
       for (int c = 0; c < 8; c += 2) {
         // the saturating conversion clamps to +-448 exactly like clamp-then-cast
-        const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(v[p][c] * r_lo, v[p][c + 1] * r_lo), __NV_SATFINITE, __NV_E4M3);
-        two[c >> 1] = __nv_cvt_float2_to_fp8x2(make_float2(v[p][c] * r_hi, v[p][c + 1] * r_hi), __NV_SATFINITE, __NV_E4M3);
+        // x * r + (-0) is x * r, signed zeros included
+        const uint64_t x2 = pack_f32x2(vp[c], vp[c + 1]);
+        float2 y_lo, y_hi;
+        unpack_f32x2(fma_f32x2(x2, r_lo2, neg0), y_lo.x, y_lo.y);
+        unpack_f32x2(fma_f32x2(x2, r_hi2, neg0), y_hi.x, y_hi.y);
+        const uint32_t lo = __nv_cvt_float2_to_fp8x2(y_lo, __NV_SATFINITE, __NV_E4M3);
+        two[c >> 1] = __nv_cvt_float2_to_fp8x2(y_hi, __NV_SATFINITE, __NV_E4M3);
         same &= lo == two[c >> 1];
       }
       if (!same) {
 #pragma unroll
         for (int c = 0; c < 8; c += 2)
-          two[c >> 1] = __nv_cvt_float2_to_fp8x2(make_float2(__fdiv_rn(v[p][c], scale), __fdiv_rn(v[p][c + 1], scale)),
+          two[c >> 1] = __nv_cvt_float2_to_fp8x2(make_float2(__fdiv_rn(vp[c], scale), __fdiv_rn(vp[c + 1], scale)),
                                                  __NV_SATFINITE, __NV_E4M3);
       }
 #pragma unroll
       for (int c = 0; c < 8; c += 2) {
         const __half2_raw back = __nv_cvt_fp8x2_to_halfraw2(static_cast<__nv_fp8x2_storage_t>(two[c >> 1]), __NV_E4M3);
         const float2 f = __half22float2(__half2(back));
-        sums[c] += f.x;
-        sums[c + 1] += f.y;
+        sums2[c >> 1] = add_f32x2(sums2[c >> 1], pack_f32x2(f.x, f.y));
       }
       *reinterpret_cast<uint2*>(dst + static_cast<size_t>(row) * kHeadDim) =
           make_uint2(two[0] | (two[1] << 16), two[2] | (two[3] << 16));
@@ -187,7 +243,12 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const __grid_constan
       // the number of columns a lane still carries, so eight columns take six shuffles instead of sixteen.
       int s8[8];
 #pragma unroll
-      for (int c = 0; c < 8; ++c) s8[c] = __float2int_rn(sums[c] * 512.0f);  // exact integer, units of 2^-9
+      for (int c = 0; c < 8; c += 2) {  // exact integers, units of 2^-9
+        float lo, hi;
+        unpack_f32x2(sums2[c >> 1], lo, hi);
+        s8[c] = __float2int_rn(lo * 512.0f);
+        s8[c + 1] = __float2int_rn(hi * 512.0f);
+      }
       const bool up16 = (threadIdx.x & 16) != 0, up8 = (threadIdx.x & 8) != 0;
       int s4[4], s2[2];
 #pragma unroll
@@ -206,7 +267,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const __grid_constan
       atomicAdd(&s_col[col], s2[0]);
       atomicAdd(&s_col[col + 1], s2[1]);
       __syncthreads();
-      if (threadIdx.x < kHeadDim) colsum[static_cast<size_t>(tile) * kHeadDim + threadIdx.x] = s_col[threadIdx.x];
+      for (int c = threadIdx.x; c < kHeadDim; c += kThreads) colsum[static_cast<size_t>(tile) * kHeadDim + c] = s_col[c];
     }
     __syncthreads();  // s_max and s_col are reused by the next tile
     tile += stride;
@@ -222,19 +283,20 @@ lite3r_status launch(const QuantBatch& batch, const lite3r_shape& s, cudaStream_
   const int nb = ceil_div(s.tokens, BS);
   const int tiles = s.batch * s.heads * nb;
   constexpr int kTileBytes = BS * kHeadDim * static_cast<int>(sizeof(SrcT));
-  constexpr int kSmem = ring_depth(kTileBytes) * kTileBytes;
+  constexpr int kThreads = cta_threads(kTileBytes);
+  constexpr int kSmem = ring_depth(kTileBytes, kThreads) * kTileBytes;
   int sms = 0;
   lite3r_status st = sm_count(&sms);
   if (st != LITE3R_OK) return st;
-  st = record_cuda(cudaFuncSetAttribute(quantize_kernel<BS, SrcT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem));
+  st = record_cuda(cudaFuncSetAttribute(quantize_kernel<BS, SrcT, kThreads>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem));
   if (st != LITE3R_OK) return st;
   int per_sm = 0;
-  st = record_cuda(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, quantize_kernel<BS, SrcT>, kThreads, kSmem));
+  st = record_cuda(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, quantize_kernel<BS, SrcT, kThreads>, kThreads, kSmem));
   if (st != LITE3R_OK) return st;
   if (per_sm < 1) per_sm = 1;
   const long long all = static_cast<long long>(tiles) * batch.count;
   const int grid = static_cast<int>(all < static_cast<long long>(sms) * per_sm ? all : static_cast<long long>(sms) * per_sm);
-  quantize_kernel<BS, SrcT><<<grid, kThreads, kSmem, stream>>>(batch, s.heads, s.tokens, nb, tiles);
+  quantize_kernel<BS, SrcT, kThreads><<<grid, kThreads, kSmem, stream>>>(batch, s.heads, s.tokens, nb, tiles);
   return after_launch();
 }
 
