@@ -35,35 +35,69 @@ __device__ __forceinline__ unsigned long long order_key(double v) {
 }
 
 struct Selection {
-  unsigned long long prefix, mask;  // (key & mask) > prefix: selected; == prefix: the first `take` by index are
-  int take;
+  // An entry is selected when its bucket is above `bucket`; inside that bucket when (key & mask) > prefix, and of the
+  // entries with (key & mask) == prefix the first `take` in index order.
+  unsigned long long prefix, mask;
+  int take, bucket;
 };
 
-// The k best (largest key, then lowest index) of keys[0..n): warp-collective, hist is this warp's 256 counters.
-__device__ Selection select_top(const unsigned long long* keys, int n, int k, unsigned int* hist, int lane) {
-  Selection s;
-  if (k <= 0) {  // nothing selected: no masked key exceeds or equals the all-ones prefix with take 0
-    s.prefix = ~0ull;
-    s.mask = ~0ull;
-    s.take = 0;
-    return s;
+constexpr int kBuckets = 256;
+constexpr int kMaxListed = 128;  // candidates of a threshold bucket kept as an index list; fuller buckets are re-scanned
+
+// Position of rank `remaining` (1-based, counted from the top bin down) in a 256-bin histogram: the bin holding it, the
+// entries in the bins above and the size of that bin.  Warp-collective; lane L owns bins 255-8L .. 248-8L.
+struct Located {
+  int bin, above, size;
+};
+__device__ __forceinline__ Located locate(const unsigned int* hist, int remaining, int lane) {
+  int cnt[8], tot = 0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    cnt[i] = static_cast<int>(hist[255 - 8 * lane - i]);
+    tot += cnt[i];
   }
-  if (k >= n) {  // everything selected
-    s.prefix = 0ull;
-    s.mask = 0ull;
-    s.take = n;
-    return s;
+  int incl = tot;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+    if (lane >= o) incl += up;
   }
+  const int excl = incl - tot;
+  const bool mine = excl < remaining && remaining <= incl;
+  Located r = {0, 0, 0};
+  if (mine) {
+    int run = excl;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      if (r.size == 0 && run + cnt[i] >= remaining) {
+        r.bin = 255 - 8 * lane - i;
+        r.above = run;
+        r.size = cnt[i];
+      }
+      run += cnt[i];
+    }
+  }
+  const int src = __ffs(__ballot_sync(0xFFFFFFFFu, mine)) - 1;
+  r.bin = __shfl_sync(0xFFFFFFFFu, r.bin, src);
+  r.above = __shfl_sync(0xFFFFFFFFu, r.above, src);
+  r.size = __shfl_sync(0xFFFFFFFFu, r.size, src);
+  return r;
+}
+
+// The k best (largest key, then lowest position) of the m candidates cand(0) .. cand(m - 1), 0 < k < m as far as the
+// valid ones go: cand(c, key) says whether candidate c takes part and gives its key.  Most-significant-digit-first
+// radix select over the 64-bit keys, 8-bit digits placed at the highest bit on which the remaining candidates still
+// differ (keys of one row share their sign and leading exponent bits, so fixed digit positions would spend whole
+// passes on digits that are equal for everyone).  Warp-collective; hist is this warp's 256 counters.
+template <class Cand>
+__device__ void radix_select(Cand cand, int m, int k, unsigned int* hist, int lane, Selection& s) {
   unsigned long long prefix = 0ull, mask = 0ull;
   int remaining = k;
   while (true) {
-    // Bits on which the candidates (keys matching the prefix so far) still differ: scores of one row share their
-    // sign and leading exponent bits, so fixed digit positions would spend whole passes (and 32-way histogram
-    // conflicts) on digits that are equal for everyone.  Each pass starts at the highest differing bit instead.
     unsigned long long all_and = ~0ull, all_or = 0ull;
-    for (int j = lane; j < n; j += 32) {
-      const unsigned long long key = keys[j];
-      if ((key & mask) == prefix) {
+    for (int c = lane; c < m; c += 32) {
+      unsigned long long key;
+      if (cand(c, key) && (key & mask) == prefix) {
         all_and &= key;
         all_or |= key;
       }
@@ -87,53 +121,71 @@ __device__ Selection select_top(const unsigned long long* keys, int n, int k, un
 #pragma unroll
     for (int b = 0; b < 8; ++b) hist[lane + 32 * b] = 0u;
     __syncwarp();
-    for (int j = lane; j < n; j += 32) {
-      const unsigned long long key = keys[j];
-      if ((key & mask) == prefix) atomicAdd(&hist[static_cast<unsigned int>(key >> shift) & 255u], 1u);
+    for (int c = lane; c < m; c += 32) {
+      unsigned long long key;
+      if (cand(c, key) && (key & mask) == prefix) atomicAdd(&hist[static_cast<unsigned int>(key >> shift) & 255u], 1u);
     }
     __syncwarp();
-    // lane L owns the digits 255-8L .. 248-8L, visited in descending order
-    int cnt[8], tot = 0;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      cnt[i] = static_cast<int>(hist[255 - 8 * lane - i]);
-      tot += cnt[i];
-    }
-    int incl = tot;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-      if (lane >= o) incl += up;
-    }
-    const int excl = incl - tot;
-    const bool mine = excl < remaining && remaining <= incl;
-    int digit = 0, above = 0, bin = 0;
-    if (mine) {
-      int run = excl;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        if (bin == 0 && run + cnt[i] >= remaining) {
-          digit = 255 - 8 * lane - i;
-          above = run;
-          bin = cnt[i];
-        }
-        run += cnt[i];
-      }
-    }
-    const int src = __ffs(__ballot_sync(0xFFFFFFFFu, mine)) - 1;
-    digit = __shfl_sync(0xFFFFFFFFu, digit, src);
-    above = __shfl_sync(0xFFFFFFFFu, above, src);
-    bin = __shfl_sync(0xFFFFFFFFu, bin, src);
-    remaining -= above;
+    const Located at = locate(hist, remaining, lane);
+    remaining -= at.above;
     const unsigned long long field = 0xFFull << shift;
-    prefix = (prefix & ~field) | (static_cast<unsigned long long>(digit) << shift);
+    prefix = (prefix & ~field) | (static_cast<unsigned long long>(at.bin) << shift);
     mask |= field;
     __syncwarp();
-    if (bin == remaining || shift == 0) break;  // the whole bin is selected, or every bit has been decided
+    if (at.size == remaining || shift == 0) break;  // the whole bin is selected, or every bit has been decided
   }
   s.prefix = prefix;
   s.mask = mask;
   s.take = remaining;
+}
+
+// The k best (largest key, then lowest index) of keys[0..n).  First a histogram over 256 buckets that are linear in
+// the score (bucket(j), any monotone map of the score to 0..255, computed from a single-precision copy): it places
+// the k-th best in one bucket with usually a handful of entries, listed by index (idx, at most kMaxListed) for the
+// radix select that decides between them.  hist must hold the bucket counts of the row on entry.  Warp-collective.
+template <class Bucket>
+__device__ Selection select_top(const unsigned long long* keys, Bucket bucket, int n, int k, unsigned int* hist,
+                                const unsigned int* bucket_hist, unsigned short* idx, int lane) {
+  Selection s;
+  s.prefix = 0ull;
+  s.mask = 0ull;
+  s.take = 0;
+  if (k <= 0) {  // nothing selected
+    s.bucket = kBuckets;
+    return s;
+  }
+  if (k >= n) {  // everything selected
+    s.bucket = -1;
+    return s;
+  }
+  const Located at = locate(bucket_hist, k, lane);
+  s.bucket = at.bin;
+  const int remaining = k - at.above;
+  if (remaining == at.size) {  // the whole bucket is selected
+    s.take = at.size;
+    return s;
+  }
+  if (at.size <= kMaxListed) {
+    const unsigned below = (1u << lane) - 1u;
+    int listed = 0;
+    for (int j0 = 0; j0 < n; j0 += 32) {
+      const int j = j0 + lane;
+      const bool is = j < n && bucket(j) == at.bin;
+      const unsigned b = __ballot_sync(0xFFFFFFFFu, is);
+      if (is) idx[listed + __popc(b & below)] = static_cast<unsigned short>(j);
+      listed += __popc(b);
+    }
+    __syncwarp();
+    radix_select([&](int c, unsigned long long& key) {
+      key = keys[idx[c]];
+      return true;
+    }, at.size, remaining, hist, lane, s);
+  } else {
+    radix_select([&](int c, unsigned long long& key) {
+      key = keys[c];
+      return bucket(c) == at.bin;
+    }, n, remaining, hist, lane, s);
+  }
   return s;
 }
 
@@ -153,9 +205,10 @@ __global__ void __launch_bounds__(R * 32) plan_kernel(const int* __restrict__ q_
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int pitch = (nb + 1) & ~1;  // key-row pitch: keeps everything behind the keys 16-byte aligned
   unsigned long long* s_key = reinterpret_cast<unsigned long long*>(smem_raw);        // [R][pitch]
-  double* s_q = reinterpret_cast<double*>(s_key + static_cast<size_t>(R) * pitch);    // [R][kPitch]
-  double* s_k = s_q + R * kPitch;                                                     // [kChunk][kPitch]
-  unsigned int* s_hist = reinterpret_cast<unsigned int*>(s_k + kChunk * kPitch);      // [R][256]
+  unsigned int* s_hist = reinterpret_cast<unsigned int*>(s_key + static_cast<size_t>(R) * pitch);  // [R][2][256]
+  unsigned short* s_idx = reinterpret_cast<unsigned short*>(s_hist + R * 2 * kBuckets);            // [R][2][kMaxListed]
+  float2* s_range = reinterpret_cast<float2*>(s_idx + R * 2 * kMaxListed);                         // [8][R]     (R == 8)
+  unsigned char* s_bkt = reinterpret_cast<unsigned char*>(s_range + 8 * R);                        // [R][pitch] (R == 8)
 
   const int row_tiles = (nb + R - 1) / R;
   const int bh = blockIdx.x / row_tiles;
@@ -164,99 +217,144 @@ __global__ void __launch_bounds__(R * 32) plan_kernel(const int* __restrict__ q_
   const int lane = threadIdx.x & 31;
   const size_t bh_rows = static_cast<size_t>(bh) * nb;
 
-  for (int t = threadIdx.x; t < R * kHeadDim; t += kThreads) {
-    const int r = t / kHeadDim, d = t % kHeadDim;
-    s_q[r * kPitch + d] = (i0 + r < nb) ? static_cast<double>(q_colsum[(bh_rows + i0 + r) * kHeadDim + d]) : 0.0;
-  }
-
-  // Phase A.  The column sums of the next kStep key blocks are fetched (16-byte loads) into registers before the
-  // current ones are multiplied, so their latency hides behind the fp64 work; both staged arrays use a row pitch
-  // of 66 doubles, which keeps the 16-byte reads of the eight key rows and of the four row groups of a warp on
-  // different banks.
-  constexpr int kLoads = kStep * (kHeadDim / 4) / kThreads;  // int4 loads per thread and pass
-  const int kl = lane % kKeysPerWarp, rg = lane / kKeysPerWarp;
-  const int jj = warp * kKeysPerWarp + kl;
-  int4 pre[kLoads];
-  auto prefetch = [&](int j0) {
-    const int4* src = reinterpret_cast<const int4*>(k_colsum + (bh_rows + j0) * kHeadDim);
-    const int n4 = min(kStep, nb - j0) * (kHeadDim / 4);
-#pragma unroll
-    for (int q = 0; q < kLoads; ++q) {
-      const int v = threadIdx.x + q * kThreads;
-      pre[q] = v < n4 ? __ldg(src + v) : make_int4(0, 0, 0, 0);
-    }
-  };
-  prefetch(0);
-  double q_frag[R == 8 ? kHeadDim / 4 : 1] = {};
   if constexpr (R == 8) {
-    __syncthreads();  // s_q is complete
+    // Phase A, 8 rows x 8 key blocks per warp and step as an fp64 tensor-core product (m8n8k4, 16 k-steps over the
+    // 64 columns): the integer products and sums stay below 2^53, so the result is the exact dot product whatever
+    // the order.  The product does not care which column sits at which k index as long as A and B agree, so lane
+    // (g, t) supplies columns 16 t .. 16 t + 15 of its row (q row g for A, key block g of the warp's eight for B):
+    // 64 contiguous bytes of the int32 column sums, read straight from global memory (L2) one step ahead, with no
+    // staging and no barrier.  int32 -> fp64 is exact and takes one xor and one subtraction: the double with high
+    // word 0x43300000 and low word v ^ 2^31 is 2^52 + 2^31 + v.
+    const int g = lane >> 2, t4 = lane & 3;
+    auto widen = [](int v) {
+      return __hiloint2double(0x43300000, v ^ static_cast<int>(0x80000000u)) - 4503601774854144.0;
+    };
+    auto load16 = [&](const int* base, size_t row, bool in, int4 dst[4]) {
+      const int4* src = reinterpret_cast<const int4*>(base + row * kHeadDim + 16 * t4);
 #pragma unroll
-    for (int st = 0; st < kHeadDim / 4; ++st) q_frag[st] = s_q[(lane >> 2) * kPitch + 4 * st + (lane & 3)];
-  }
-  for (int j0 = 0; j0 < nb; j0 += kStep) {
-    __syncthreads();
-    const int nj = min(kStep, nb - j0);
+      for (int q = 0; q < 4; ++q) dst[q] = in ? __ldg(src + q) : make_int4(0, 0, 0, 0);
+    };
+    double q_frag[16];
+    {
+      int4 qv[4];
+      load16(q_colsum, bh_rows + i0 + g, i0 + g < nb, qv);
 #pragma unroll
-    for (int q = 0; q < kLoads; ++q) {
-      const int v = threadIdx.x + q * kThreads;
-      double* dst = s_k + (v / (kHeadDim / 4)) * kPitch + (v % (kHeadDim / 4)) * 4;
-      *reinterpret_cast<double2*>(dst) = make_double2(static_cast<double>(pre[q].x), static_cast<double>(pre[q].y));
-      *reinterpret_cast<double2*>(dst + 2) = make_double2(static_cast<double>(pre[q].z), static_cast<double>(pre[q].w));
-    }
-    if (j0 + kStep < nb) prefetch(j0 + kStep);
-    __syncthreads();
-    if constexpr (R == 8) {
-      // 8 rows x 8 key blocks per warp as an fp64 tensor-core product (m8n8k4, 16 steps over the 64 columns): the
-      // integer products and sums stay below 2^53, so the result is the exact dot product whatever the order.  A
-      // lane holds A[g][t] = q row g, column 4 s + t (kept in registers for the whole kernel) and loads
-      // B[t][g] = key block g of the warp's eight, column 4 s + t; it ends with the scores of row g against key
-      // blocks 2 t and 2 t + 1.
-      const int g = lane >> 2, t4 = lane & 3;
-      const double* kr = s_k + (warp * 8 + g) * kPitch + t4;
-      double c[2][2] = {{0.0, 0.0}, {0.0, 0.0}};  // two accumulation chains (even / odd steps) hide the MMA latency
-      double bv[kHeadDim / 4];
-#pragma unroll
-      for (int st = 0; st < kHeadDim / 4; ++st) bv[st] = kr[4 * st];
-#pragma unroll
-      for (int st = 0; st < kHeadDim / 4; ++st) {
-        asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
-                     : "+d"(c[st & 1][0]), "+d"(c[st & 1][1])
-                     : "d"(q_frag[st]), "d"(bv[st]));
+      for (int q = 0; q < 4; ++q) {
+        q_frag[4 * q] = widen(qv[q].x);
+        q_frag[4 * q + 1] = widen(qv[q].y);
+        q_frag[4 * q + 2] = widen(qv[q].z);
+        q_frag[4 * q + 3] = widen(qv[q].w);
       }
+    }
+    int4 nxt[4];
+    load16(k_colsum, bh_rows + warp * 8 + g, warp * 8 + g < nb, nxt);
+    float lo = INFINITY, hi = -INFINITY;  // range of row g's scores, as far as this lane sees them
+    const bool block_pow2 = (block & (block - 1)) == 0;
+    const double inv_block = 1.0 / static_cast<double>(block);
+    for (int j0 = warp * 8; j0 < nb; j0 += 64) {
+      int4 cur[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) cur[q] = nxt[q];
+      if (j0 + 64 < nb) load16(k_colsum, bh_rows + j0 + 64 + g, j0 + 64 + g < nb, nxt);
+      double c[2][2] = {{0.0, 0.0}, {0.0, 0.0}};  // two accumulation chains (even / odd steps) hide the MMA latency
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int vals[4] = {cur[q].x, cur[q].y, cur[q].z, cur[q].w};
+#pragma unroll
+        for (int y = 0; y < 4; ++y) {
+          const int st = 4 * q + y;
+          const double bv = widen(vals[y]);
+          asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+                       : "+d"(c[st & 1][0]), "+d"(c[st & 1][1])
+                       : "d"(q_frag[st]), "d"(bv));
+        }
+      }
+      // the lane ends with the scores of row g against key blocks 2 t and 2 t + 1 of the warp's eight
       const double cc[2] = {c[0][0] + c[1][0], c[0][1] + c[1][1]};
 #pragma unroll
       for (int x = 0; x < 2; ++x) {
-        const int j = j0 + warp * 8 + 2 * t4 + x;
+        const int j = j0 + 2 * t4 + x;
         if (j < nb) {
           const int valid = min(block, tokens - j * block);
-          const double tt = cc[x] * static_cast<double>(k_scales[bh_rows + j]) / static_cast<double>(valid) + 0.0;
+          // a full block of 2^n tokens divides exactly by a multiplication; only the last block can be shorter
+          const double num = cc[x] * static_cast<double>(k_scales[bh_rows + j]);
+          const double tt = (valid == block && block_pow2 ? num * inv_block : num / static_cast<double>(valid)) + 0.0;
           s_key[static_cast<size_t>(g) * pitch + j] = order_key(tt);
+          // range of the row in single precision, for the bucket histogram of the selection
+          const float tf = static_cast<float>(tt);
+          lo = fminf(lo, tf);
+          hi = fmaxf(hi, tf);
         }
       }
-    } else if (jj < nj) {
-      const double2* kr = reinterpret_cast<const double2*>(s_k + jj * kPitch);
-      const double2* qr = reinterpret_cast<const double2*>(s_q + rg * kRowsPerLane * kPitch);
-      double acc[kRowsPerLane];
+    }
 #pragma unroll
-      for (int x = 0; x < kRowsPerLane; ++x) acc[x] = 0.0;
+    for (int o = 1; o <= 2; o <<= 1) {
+      lo = fminf(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, o));
+      hi = fmaxf(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, o));
+    }
+    if (t4 == 0) s_range[warp * R + g] = make_float2(lo, hi);
+  } else {
+    // Phase A for sequences too long for eight rows of keys per CTA: the column sums of kStep key blocks at a time
+    // are staged in shared memory as doubles (fetched with 16-byte loads one pass ahead); a lane owns one key block
+    // and R / 4 rows, so every staged value feeds several fp64 FMAs.  Both staged arrays use a row pitch of 68
+    // doubles, which keeps the 16-byte reads of the key rows and of the row groups of a warp on different banks.
+    double* s_q = reinterpret_cast<double*>(s_idx + R * 2 * kMaxListed);  // [R][kPitch]
+    double* s_k = s_q + R * kPitch;                             // [kChunk][kPitch]
+    for (int t = threadIdx.x; t < R * kHeadDim; t += kThreads) {
+      const int r = t / kHeadDim, d = t % kHeadDim;
+      s_q[r * kPitch + d] = (i0 + r < nb) ? static_cast<double>(q_colsum[(bh_rows + i0 + r) * kHeadDim + d]) : 0.0;
+    }
+    constexpr int kLoads = kStep * (kHeadDim / 4) / kThreads;  // int4 loads per thread and pass
+    const int kl = lane % kKeysPerWarp, rg = lane / kKeysPerWarp;
+    const int jj = warp * kKeysPerWarp + kl;
+    int4 pre[kLoads];
+    auto prefetch = [&](int j0) {
+      const int4* src = reinterpret_cast<const int4*>(k_colsum + (bh_rows + j0) * kHeadDim);
+      const int n4 = min(kStep, nb - j0) * (kHeadDim / 4);
+#pragma unroll
+      for (int q = 0; q < kLoads; ++q) {
+        const int v = threadIdx.x + q * kThreads;
+        pre[q] = v < n4 ? __ldg(src + v) : make_int4(0, 0, 0, 0);
+      }
+    };
+    prefetch(0);
+    for (int j0 = 0; j0 < nb; j0 += kStep) {
+      __syncthreads();
+      const int nj = min(kStep, nb - j0);
+#pragma unroll
+      for (int q = 0; q < kLoads; ++q) {
+        const int v = threadIdx.x + q * kThreads;
+        double* dst = s_k + (v / (kHeadDim / 4)) * kPitch + (v % (kHeadDim / 4)) * 4;
+        *reinterpret_cast<double2*>(dst) = make_double2(static_cast<double>(pre[q].x), static_cast<double>(pre[q].y));
+        *reinterpret_cast<double2*>(dst + 2) = make_double2(static_cast<double>(pre[q].z), static_cast<double>(pre[q].w));
+      }
+      if (j0 + kStep < nb) prefetch(j0 + kStep);
+      __syncthreads();
+      if (jj < nj) {
+        const double2* kr = reinterpret_cast<const double2*>(s_k + jj * kPitch);
+        const double2* qr = reinterpret_cast<const double2*>(s_q + rg * kRowsPerLane * kPitch);
+        double acc[kRowsPerLane];
+#pragma unroll
+        for (int x = 0; x < kRowsPerLane; ++x) acc[x] = 0.0;
 #pragma unroll 8
-      for (int d2 = 0; d2 < kHeadDim / 2; ++d2) {
-        const double2 kv = kr[d2];
+        for (int d2 = 0; d2 < kHeadDim / 2; ++d2) {
+          const double2 kv = kr[d2];
+#pragma unroll
+          for (int x = 0; x < kRowsPerLane; ++x) {
+            const double2 qv = qr[x * (kPitch / 2) + d2];
+            acc[x] = fma(qv.x, kv.x, acc[x]);
+            acc[x] = fma(qv.y, kv.y, acc[x]);
+          }
+        }
+        const int j = j0 + jj;
+        const int valid = min(block, tokens - j * block);
+        const double ks = static_cast<double>(k_scales[bh_rows + j]);
+        const double n_valid = static_cast<double>(valid);
 #pragma unroll
         for (int x = 0; x < kRowsPerLane; ++x) {
-          const double2 qv = qr[x * (kPitch / 2) + d2];
-          acc[x] = fma(qv.x, kv.x, acc[x]);
-          acc[x] = fma(qv.y, kv.y, acc[x]);
+          const double t = acc[x] * ks / n_valid + 0.0;
+          s_key[static_cast<size_t>(rg * kRowsPerLane + x) * pitch + j] = order_key(t);
         }
-      }
-      const int j = j0 + jj;
-      const int valid = min(block, tokens - j * block);
-      const double ks = static_cast<double>(k_scales[bh_rows + j]);
-      const double n_valid = static_cast<double>(valid);
-#pragma unroll
-      for (int x = 0; x < kRowsPerLane; ++x) {
-        const double t = acc[x] * ks / n_valid + 0.0;
-        s_key[static_cast<size_t>(rg * kRowsPerLane + x) * pitch + j] = order_key(t);
       }
     }
   }
@@ -266,24 +364,67 @@ __global__ void __launch_bounds__(R * 32) plan_kernel(const int* __restrict__ q_
 
   // Phase B
   const unsigned long long* keys = s_key + static_cast<size_t>(warp) * pitch;
-  unsigned int* hist = s_hist + warp * 256;
-  const Selection sc = select_top(keys, nb, k_crit, hist, lane);
-  const Selection sm = select_top(keys, nb, nb - k_neg, hist, lane);
+  unsigned int* hist = s_hist + warp * 2 * kBuckets;  // radix digits; the second half holds the bucket counts
+  unsigned int* bucket_hist = hist + kBuckets;
+  // Buckets linear in the score between the row's extremes; with fewer than eight rows per CTA (very long
+  // sequences) there is no single-precision copy and every key falls into bucket 0, which leaves the whole
+  // selection to the radix select.
+  float lo = 0.f, scale = 0.f;
+  unsigned char* bkt = s_bkt + static_cast<size_t>(warp) * pitch;
+  if constexpr (R == 8) {
+    float2 range = lane < 8 ? s_range[lane * R + warp] : make_float2(INFINITY, -INFINITY);
+#pragma unroll
+    for (int o = 1; o <= 4; o <<= 1) {
+      range.x = fminf(range.x, __shfl_xor_sync(0xFFFFFFFFu, range.x, o));
+      range.y = fmaxf(range.y, __shfl_xor_sync(0xFFFFFFFFu, range.y, o));
+    }
+    range.x = __shfl_sync(0xFFFFFFFFu, range.x, 0);
+    range.y = __shfl_sync(0xFFFFFFFFu, range.y, 0);
+    lo = range.x;
+    scale = range.y > range.x ? 255.5f / (range.y - range.x) : 0.f;
+  }
+  auto bucket = [&](int j) -> int {
+    if constexpr (R != 8) return 0;
+    return bkt[j];
+  };
+#pragma unroll
+  for (int b = 0; b < 8; ++b) bucket_hist[lane + 32 * b] = 0u;
+  __syncwarp();
+  for (int j = lane; j < nb; j += 32) {
+    int b = 0;
+    if constexpr (R == 8) {
+      // key -> double -> float: every step keeps the order (weakly), which is all the buckets need
+      const unsigned long long key = keys[j];
+      const unsigned long long u = (key >> 63) ? (key & 0x7FFFFFFFFFFFFFFFull) : ~key;
+      const float tf = static_cast<float>(__longlong_as_double(static_cast<long long>(u)));
+      b = min(kBuckets - 1, max(0, __float2int_rz((tf - lo) * scale)));
+      bkt[j] = static_cast<unsigned char>(b);
+    }
+    atomicAdd(&bucket_hist[b], 1u);
+  }
+  __syncwarp();
+  unsigned short* idx = s_idx + warp * 2 * kMaxListed;
+  const Selection sc = select_top(keys, bucket, nb, k_crit, hist, bucket_hist, idx, lane);
+  const Selection sm = select_top(keys, bucket, nb, nb - k_neg, hist, bucket_hist, idx + kMaxListed, lane);
 
   // Phase C
   const size_t row = bh_rows + i;
   signed char* out_cls = cls + row * nb;
   int n_crit = 0, n_marg = 0, tie_c = 0, tie_m = 0;
   const unsigned below = (1u << lane) - 1u;
+#pragma unroll 2
   for (int j0 = 0; j0 < nb; j0 += 32) {
     const int j = j0 + lane;
     const bool in = j < nb;
     const unsigned long long key = in ? keys[j] : 0ull;
+    const int bk = in ? bucket(j) : -2;
     const unsigned long long kc = key & sc.mask, km = key & sm.mask;
-    const bool eq_c = in && kc == sc.prefix, eq_m = in && km == sm.prefix;
+    const bool eq_c = bk == sc.bucket && kc == sc.prefix, eq_m = bk == sm.bucket && km == sm.prefix;
     const unsigned b_eq_c = __ballot_sync(0xFFFFFFFFu, eq_c), b_eq_m = __ballot_sync(0xFFFFFFFFu, eq_m);
-    const bool sel_c = in && (kc > sc.prefix || (eq_c && tie_c + __popc(b_eq_c & below) < sc.take));
-    const bool sel_m = in && (km > sm.prefix || (eq_m && tie_m + __popc(b_eq_m & below) < sm.take));
+    const bool sel_c = in && (bk > sc.bucket || (bk == sc.bucket && kc > sc.prefix) ||
+                              (eq_c && tie_c + __popc(b_eq_c & below) < sc.take));
+    const bool sel_m = in && (bk > sm.bucket || (bk == sm.bucket && km > sm.prefix) ||
+                              (eq_m && tie_m + __popc(b_eq_m & below) < sm.take));
     tie_c += __popc(b_eq_c);
     tie_m += __popc(b_eq_m);
     const int c = !in ? -1 : (sel_c ? 2 : (sel_m ? 1 : 0));
@@ -298,8 +439,13 @@ __global__ void __launch_bounds__(R * 32) plan_kernel(const int* __restrict__ q_
 }
 
 size_t plan_smem_bytes(int nb, int rows) {
-  return static_cast<size_t>(rows) * ((nb + 1) & ~1) * 8 + static_cast<size_t>(rows) * kPitch * 8 +
-         static_cast<size_t>(kChunk) * kPitch * 8 + static_cast<size_t>(rows) * 256 * 4;
+  const size_t pitch = static_cast<size_t>((nb + 1) & ~1);
+  const size_t common = rows * pitch * 8 + static_cast<size_t>(rows) * 2 * kBuckets * 4 +
+                        static_cast<size_t>(rows) * 2 * kMaxListed * 2;  // keys, two histograms, two index lists
+  // eight rows: score ranges and one bucket byte per key (the column sums come straight from global memory);
+  // fewer rows: the staged column sums as doubles
+  if (rows == 8) return common + 8 * rows * sizeof(float2) + rows * pitch;
+  return common + static_cast<size_t>(rows) * kPitch * 8 + static_cast<size_t>(kChunk) * kPitch * 8;
 }
 
 template <int R>
