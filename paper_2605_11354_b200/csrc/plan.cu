@@ -196,19 +196,21 @@ __global__ void __launch_bounds__(R * 32) plan_kernel(const int* __restrict__ q_
                                                        signed char* __restrict__ cls, int* __restrict__ crit_idx,
                                                        int* __restrict__ marg_idx) {
   constexpr int kThreads = R * 32;
-  constexpr int kGroups = R >= 4 ? 4 : R;        // row groups inside a warp
-  constexpr int kRowsPerLane = R / kGroups;       // rows whose score one lane accumulates
+  constexpr bool kDirect = R >= 8;                // column sums straight from global memory into the fp64 MMA
+  constexpr int kTiles = kDirect ? R / 8 : 1;     // 8-row MMA tiles per warp
+  constexpr int kGroups = R >= 4 ? 4 : R;        // (staged path) row groups inside a warp
+  constexpr int kRowsPerLane = R / kGroups;       // (staged path) rows whose score one lane accumulates
   constexpr int kKeysPerWarp = 32 / kGroups;
-  constexpr int kStep = kKeysPerWarp * R;         // key blocks per staged pass (<= kChunk)
-  static_assert(kStep <= kChunk, "staging buffer too small");
+  constexpr int kStep = kKeysPerWarp * R;         // (staged path) key blocks per staged pass (<= kChunk)
+  static_assert(kDirect || kStep <= kChunk, "staging buffer too small");
 
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int pitch = (nb + 1) & ~1;  // key-row pitch: keeps everything behind the keys 16-byte aligned
   unsigned long long* s_key = reinterpret_cast<unsigned long long*>(smem_raw);        // [R][pitch]
   unsigned int* s_hist = reinterpret_cast<unsigned int*>(s_key + static_cast<size_t>(R) * pitch);  // [R][2][256]
   unsigned short* s_idx = reinterpret_cast<unsigned short*>(s_hist + R * 2 * kBuckets);            // [R][2][kMaxListed]
-  float2* s_range = reinterpret_cast<float2*>(s_idx + R * 2 * kMaxListed);                         // [8][R]     (R == 8)
-  unsigned char* s_bkt = reinterpret_cast<unsigned char*>(s_range + 8 * R);                        // [R][pitch] (R == 8)
+  float2* s_range = reinterpret_cast<float2*>(s_idx + R * 2 * kMaxListed);                         // [R][R]     (direct)
+  unsigned char* s_bkt = reinterpret_cast<unsigned char*>(s_range + R * R);                        // [R][pitch] (direct)
 
   const int row_tiles = (nb + R - 1) / R;
   const int bh = blockIdx.x / row_tiles;
@@ -217,13 +219,15 @@ __global__ void __launch_bounds__(R * 32) plan_kernel(const int* __restrict__ q_
   const int lane = threadIdx.x & 31;
   const size_t bh_rows = static_cast<size_t>(bh) * nb;
 
-  if constexpr (R == 8) {
-    // Phase A, 8 rows x 8 key blocks per warp and step as an fp64 tensor-core product (m8n8k4, 16 k-steps over the
-    // 64 columns): the integer products and sums stay below 2^53, so the result is the exact dot product whatever
-    // the order.  The product does not care which column sits at which k index as long as A and B agree, so lane
-    // (g, t) supplies columns 16 t .. 16 t + 15 of its row (q row g for A, key block g of the warp's eight for B):
-    // 64 contiguous bytes of the int32 column sums, read straight from global memory (L2) one step ahead, with no
-    // staging and no barrier.  int32 -> fp64 is exact and takes one xor and one subtraction: the double with high
+  if constexpr (kDirect) {
+    // Phase A, R rows x 8 key blocks per warp and step as fp64 tensor-core products (m8n8k4, 16 k-steps over the 64
+    // columns, one 8-row tile after the other against the same B values): the integer products and sums stay below
+    // 2^53, so the result is the exact dot product whatever the order.  The product does not care which column sits
+    // at which k index as long as A and B agree, so lane (g, t) supplies columns 16 t .. 16 t + 15 of its row (q
+    // row g of each tile for A, key block g of the warp's eight for B): 64 contiguous bytes of the int32 column
+    // sums, read straight from global memory (L2) one step ahead, with no staging and no barrier.  Every CTA
+    // streams all column sums of its (b, h) once, which is what bounds this phase: hence as many rows per CTA as
+    // shared memory allows.  int32 -> fp64 is exact and takes one xor and one subtraction: the double with high
     // word 0x43300000 and low word v ^ 2^31 is 2^52 + 2^31 + v.
     const int g = lane >> 2, t4 = lane & 3;
     auto widen = [](int v) {
@@ -234,29 +238,53 @@ __global__ void __launch_bounds__(R * 32) plan_kernel(const int* __restrict__ q_
 #pragma unroll
       for (int q = 0; q < 4; ++q) dst[q] = in ? __ldg(src + q) : make_int4(0, 0, 0, 0);
     };
-    double q_frag[16];
-    {
+    double q_frag[kTiles][16];
+#pragma unroll
+    for (int m = 0; m < kTiles; ++m) {
       int4 qv[4];
-      load16(q_colsum, bh_rows + i0 + g, i0 + g < nb, qv);
+      load16(q_colsum, bh_rows + i0 + 8 * m + g, i0 + 8 * m + g < nb, qv);
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        q_frag[4 * q] = widen(qv[q].x);
-        q_frag[4 * q + 1] = widen(qv[q].y);
-        q_frag[4 * q + 2] = widen(qv[q].z);
-        q_frag[4 * q + 3] = widen(qv[q].w);
+        q_frag[m][4 * q] = widen(qv[q].x);
+        q_frag[m][4 * q + 1] = widen(qv[q].y);
+        q_frag[m][4 * q + 2] = widen(qv[q].z);
+        q_frag[m][4 * q + 3] = widen(qv[q].w);
       }
     }
+    // the scales of the two key blocks whose scores the lane ends up with travel with the column sums
+    auto load_scales = [&](int j, float dst[2]) {
+#pragma unroll
+      for (int x = 0; x < 2; ++x) dst[x] = j + x < nb ? __ldg(k_scales + bh_rows + j + x) : 0.f;
+    };
     int4 nxt[4];
+    float nxt_ks[2];
     load16(k_colsum, bh_rows + warp * 8 + g, warp * 8 + g < nb, nxt);
-    float lo = INFINITY, hi = -INFINITY;  // range of row g's scores, as far as this lane sees them
+    load_scales(warp * 8 + 2 * t4, nxt_ks);
+    float lo[kTiles], hi[kTiles];  // range of the scores of row 8 m + g, as far as this lane sees them
+#pragma unroll
+    for (int m = 0; m < kTiles; ++m) {
+      lo[m] = INFINITY;
+      hi[m] = -INFINITY;
+    }
     const bool block_pow2 = (block & (block - 1)) == 0;
     const double inv_block = 1.0 / static_cast<double>(block);
-    for (int j0 = warp * 8; j0 < nb; j0 += 64) {
+    for (int j0 = warp * 8; j0 < nb; j0 += 8 * R) {
       int4 cur[4];
 #pragma unroll
       for (int q = 0; q < 4; ++q) cur[q] = nxt[q];
-      if (j0 + 64 < nb) load16(k_colsum, bh_rows + j0 + 64 + g, j0 + 64 + g < nb, nxt);
-      double c[2][2] = {{0.0, 0.0}, {0.0, 0.0}};  // two accumulation chains (even / odd steps) hide the MMA latency
+      const float cur_ks[2] = {nxt_ks[0], nxt_ks[1]};
+      if (j0 + 8 * R < nb) {
+        load16(k_colsum, bh_rows + j0 + 8 * R + g, j0 + 8 * R + g < nb, nxt);
+        load_scales(j0 + 8 * R + 2 * t4, nxt_ks);
+      }
+      // per tile two accumulation chains (even / odd k-steps), which hide the MMA latency; four were slower
+      constexpr int kChains = 2;
+      double c[kTiles][kChains][2];
+#pragma unroll
+      for (int m = 0; m < kTiles; ++m) {
+#pragma unroll
+        for (int n = 0; n < kChains; ++n) c[m][n][0] = c[m][n][1] = 0.0;
+      }
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const int vals[4] = {cur[q].x, cur[q].y, cur[q].z, cur[q].w};
@@ -264,35 +292,45 @@ __global__ void __launch_bounds__(R * 32) plan_kernel(const int* __restrict__ q_
         for (int y = 0; y < 4; ++y) {
           const int st = 4 * q + y;
           const double bv = widen(vals[y]);
-          asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
-                       : "+d"(c[st & 1][0]), "+d"(c[st & 1][1])
-                       : "d"(q_frag[st]), "d"(bv));
+#pragma unroll
+          for (int m = 0; m < kTiles; ++m) {
+            asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+                         : "+d"(c[m][st % kChains][0]), "+d"(c[m][st % kChains][1])
+                         : "d"(q_frag[m][st]), "d"(bv));
+          }
         }
       }
-      // the lane ends with the scores of row g against key blocks 2 t and 2 t + 1 of the warp's eight
-      const double cc[2] = {c[0][0] + c[1][0], c[0][1] + c[1][1]};
+      // the lane ends with the scores of rows 8 m + g against key blocks 2 t and 2 t + 1 of the warp's eight
 #pragma unroll
       for (int x = 0; x < 2; ++x) {
         const int j = j0 + 2 * t4 + x;
         if (j < nb) {
           const int valid = min(block, tokens - j * block);
-          // a full block of 2^n tokens divides exactly by a multiplication; only the last block can be shorter
-          const double num = cc[x] * static_cast<double>(k_scales[bh_rows + j]);
-          const double tt = (valid == block && block_pow2 ? num * inv_block : num / static_cast<double>(valid)) + 0.0;
-          s_key[static_cast<size_t>(g) * pitch + j] = order_key(tt);
-          // range of the row in single precision, for the bucket histogram of the selection
-          const float tf = static_cast<float>(tt);
-          lo = fminf(lo, tf);
-          hi = fmaxf(hi, tf);
+          const double ks = static_cast<double>(cur_ks[x]);
+          const bool full = valid == block && block_pow2;
+#pragma unroll
+          for (int m = 0; m < kTiles; ++m) {
+            // a full block of 2^n tokens divides exactly by a multiplication; only the last block can be shorter
+            const double num = (c[m][0][x] + c[m][1][x]) * ks;
+            const double tt = (full ? num * inv_block : num / static_cast<double>(valid)) + 0.0;
+            s_key[static_cast<size_t>(8 * m + g) * pitch + j] = order_key(tt);
+            // range of the row in single precision, for the bucket histogram of the selection
+            const float tf = static_cast<float>(tt);
+            lo[m] = fminf(lo[m], tf);
+            hi[m] = fmaxf(hi[m], tf);
+          }
         }
       }
     }
 #pragma unroll
-    for (int o = 1; o <= 2; o <<= 1) {
-      lo = fminf(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, o));
-      hi = fmaxf(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, o));
+    for (int m = 0; m < kTiles; ++m) {
+#pragma unroll
+      for (int o = 1; o <= 2; o <<= 1) {
+        lo[m] = fminf(lo[m], __shfl_xor_sync(0xFFFFFFFFu, lo[m], o));
+        hi[m] = fmaxf(hi[m], __shfl_xor_sync(0xFFFFFFFFu, hi[m], o));
+      }
+      if (t4 == 0) s_range[warp * R + 8 * m + g] = make_float2(lo[m], hi[m]);
     }
-    if (t4 == 0) s_range[warp * R + g] = make_float2(lo, hi);
   } else {
     // Phase A for sequences too long for eight rows of keys per CTA: the column sums of kStep key blocks at a time
     // are staged in shared memory as doubles (fetched with 16-byte loads one pass ahead); a lane owns one key block
@@ -371,10 +409,10 @@ __global__ void __launch_bounds__(R * 32) plan_kernel(const int* __restrict__ q_
   // selection to the radix select.
   float lo = 0.f, scale = 0.f;
   unsigned char* bkt = s_bkt + static_cast<size_t>(warp) * pitch;
-  if constexpr (R == 8) {
-    float2 range = lane < 8 ? s_range[lane * R + warp] : make_float2(INFINITY, -INFINITY);
+  if constexpr (kDirect) {
+    float2 range = lane < R ? s_range[lane * R + warp] : make_float2(INFINITY, -INFINITY);
 #pragma unroll
-    for (int o = 1; o <= 4; o <<= 1) {
+    for (int o = 1; o < R; o <<= 1) {
       range.x = fminf(range.x, __shfl_xor_sync(0xFFFFFFFFu, range.x, o));
       range.y = fmaxf(range.y, __shfl_xor_sync(0xFFFFFFFFu, range.y, o));
     }
@@ -384,7 +422,7 @@ __global__ void __launch_bounds__(R * 32) plan_kernel(const int* __restrict__ q_
     scale = range.y > range.x ? 255.5f / (range.y - range.x) : 0.f;
   }
   auto bucket = [&](int j) -> int {
-    if constexpr (R != 8) return 0;
+    if constexpr (!kDirect) return 0;
     return bkt[j];
   };
 #pragma unroll
@@ -392,7 +430,7 @@ __global__ void __launch_bounds__(R * 32) plan_kernel(const int* __restrict__ q_
   __syncwarp();
   for (int j = lane; j < nb; j += 32) {
     int b = 0;
-    if constexpr (R == 8) {
+    if constexpr (kDirect) {
       // key -> double -> float: every step keeps the order (weakly), which is all the buckets need
       const unsigned long long key = keys[j];
       const unsigned long long u = (key >> 63) ? (key & 0x7FFFFFFFFFFFFFFFull) : ~key;
@@ -442,9 +480,9 @@ size_t plan_smem_bytes(int nb, int rows) {
   const size_t pitch = static_cast<size_t>((nb + 1) & ~1);
   const size_t common = rows * pitch * 8 + static_cast<size_t>(rows) * 2 * kBuckets * 4 +
                         static_cast<size_t>(rows) * 2 * kMaxListed * 2;  // keys, two histograms, two index lists
-  // eight rows: score ranges and one bucket byte per key (the column sums come straight from global memory);
+  // eight rows or more: score ranges and one bucket byte per key (the column sums come straight from global memory);
   // fewer rows: the staged column sums as doubles
-  if (rows == 8) return common + 8 * rows * sizeof(float2) + rows * pitch;
+  if (rows >= 8) return common + static_cast<size_t>(rows) * rows * sizeof(float2) + rows * pitch;
   return common + static_cast<size_t>(rows) * kPitch * 8 + static_cast<size_t>(kChunk) * kPitch * 8;
 }
 
