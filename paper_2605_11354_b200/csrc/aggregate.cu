@@ -113,37 +113,45 @@ aggregate_mma_kernel(const __grid_constant__ CUtensorMap map_s, const signed cha
     const bool row_ok = i < nb;
     const signed char* row_ptr = cls + (bh_rows + (row_ok ? i : 0)) * nb;
     bool ok = true;
+    // The 64 class bytes of this row for chunk c, as the 17 aligned 32-bit words that hold them (rows start at any
+    // byte); fetched one chunk ahead, so that the latency hides behind the wait for the stage and the expansion.
+    auto fetch = [&](int c, uint32_t w[17]) {
+      const int j0 = c * kChunk;
+      const uintptr_t addr = reinterpret_cast<uintptr_t>(row_ptr + j0);
+      const uint32_t* wp = reinterpret_cast<const uint32_t*>(addr & ~uintptr_t(3));
+      const int len = min(kChunk, nb - j0);                            // in-range class bytes of this chunk
+      const int words = (static_cast<int>(addr & 3u) + len + 3) / 4;   // aligned words that hold them
+#pragma unroll
+      for (int k = 0; k < 17; ++k) w[k] = (row_ok && c < chunks && k < words) ? __ldg(wp + k) : 0u;
+    };
+    uint32_t w[17];
+    fetch(0, w);
     for (int c = 0; c < chunks; ++c) {
       const int st = c % kStages;
-      if (!(ok = mbar_wait(&bars->empty[st], ((c / kStages) & 1) ^ 1, abort_flag, status, 404))) break;
       const int j0 = c * kChunk;
-      // 64 class bytes of this row starting at j0, fetched as aligned 32-bit words and realigned
-      const uintptr_t addr = reinterpret_cast<uintptr_t>(row_ptr + j0);
-      const uint32_t shift = static_cast<uint32_t>(addr & 3u) * 8u;
-      const uint32_t* wp = reinterpret_cast<const uint32_t*>(addr & ~uintptr_t(3));
-      const int len = min(kChunk, nb - j0);                                  // in-range class bytes of this chunk
-      const int words = (static_cast<int>(addr & 3u) + len + 3) / 4;         // aligned words that hold them
-      uint32_t w[17];
+      const uint32_t shift = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(row_ptr + j0) & 3u) * 8u;
+      const int len = min(kChunk, nb - j0);
+      // realigned class bytes; bit 0 of a class (0 negligible, 1 marginal, 2 critical) says "marginal"
+      uint32_t m[16];
 #pragma unroll
-      for (int k = 0; k < 17; ++k) w[k] = (row_ok && k < words) ? __ldg(wp + k) : 0u;
+      for (int k = 0; k < 16; ++k) m[k] = __funnelshift_r(w[k], w[k + 1], shift) & 0x01010101u;
+      if (len < kChunk) {  // last chunk: the bytes past the row belong to the next row
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          const int left = len - 4 * k;  // in-range bytes of this word
+          m[k] = left >= 4 ? m[k] : (left <= 0 ? 0u : (m[k] & (0xFFFFFFFFu >> (32 - 8 * left))));
+        }
+      }
+      fetch(c + 1, w);
+      if (!(ok = mbar_wait(&bars->empty[st], ((c / kStages) & 1) ^ 1, abort_flag, status, 404))) break;
       uint8_t* arow = smem + kOffA + st * kABytes + r * 128;
 #pragma unroll
       for (int ch = 0; ch < 8; ++ch) {  // 8 mask entries (two class words) per 16-byte chunk
-        uint32_t out[4];
-#pragma unroll
-        for (int hw = 0; hw < 2; ++hw) {
-          const int k = ch * 2 + hw;
-          const uint32_t bytes = __funnelshift_r(w[k], w[k + 1], shift);
-          uint32_t e[4];
-#pragma unroll
-          for (int b = 0; b < 4; ++b) {
-            const int j = j0 + k * 4 + b;
-            e[b] = (((bytes >> (8 * b)) & 0xFFu) == 1u && j < nb) ? 0x3F80u : 0u;
-          }
-          out[hw * 2] = e[0] | (e[1] << 16);
-          out[hw * 2 + 1] = e[2] | (e[3] << 16);
-        }
-        *reinterpret_cast<uint4*>(arow + ((ch ^ (r & 7)) << 4)) = make_uint4(out[0], out[1], out[2], out[3]);
+        // bytes (b0 b1 b2 b3) of 0/1 -> bf16 pairs: (b0 | b1 << 16) * 0x3F80 has 1.0 where the byte is 1
+        const uint32_t lo = m[2 * ch], hi = m[2 * ch + 1];
+        const uint32_t o0 = __byte_perm(lo, 0u, 0x4140) * 0x3F80u, o1 = __byte_perm(lo, 0u, 0x4342) * 0x3F80u;
+        const uint32_t o2 = __byte_perm(hi, 0u, 0x4140) * 0x3F80u, o3 = __byte_perm(hi, 0u, 0x4342) * 0x3F80u;
+        *reinterpret_cast<uint4*>(arow + ((ch ^ (r & 7)) << 4)) = make_uint4(o0, o1, o2, o3);
       }
       fence_proxy_async_smem();
       mbar_arrive(&bars->a_full[st]);
@@ -152,32 +160,55 @@ aggregate_mma_kernel(const __grid_constant__ CUtensorMap map_s, const signed cha
       tc_fence_after();
       const uint32_t lane_addr = tmem + ((static_cast<uint32_t>(quarter) * 32u) << 16);
       const size_t out_row = bh_rows + i;
+      // A thread owns one accumulator row, so direct stores would touch 32 different lines per instruction.  Each
+      // warp turns its 32 rows x 128 bytes (64 bf16 columns) around in shared memory (the operand stages are free:
+      // every MMA has completed) and stores whole 128-byte row segments, four rows per instruction.
+      uint8_t* const stage = smem + quarter * 4096;
 #pragma unroll 1
-      for (int part = 0; part < kTileN / 32; ++part) {
-        const int n = n_tile * kTileN + part * 32;
+      for (int pp = 0; pp < kTileN / 64; ++pp) {
+        const int n = n_tile * kTileN + pp * 64;
         if (n >= kSummaryRow) break;
-        uint32_t v[32];
-        tmem_ld32(lane_addr + part * 32, v);
-        tmem_wait_ld();
-        if (!row_ok) continue;
         if (n < kHeadDim * kHeadDim) {
-          uint4* dst = reinterpret_cast<uint4*>(g16 + out_row * kHeadDim * kHeadDim + n);
+          uint32_t pk[32];
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            uint32_t pk[4];
+          for (int half = 0; half < 2; ++half) {
+            uint32_t v[32];
+            tmem_ld32(lane_addr + pp * 64 + half * 32, v);
+            tmem_wait_ld();
 #pragma unroll
-            for (int x = 0; x < 4; ++x) {
-              __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[q * 8 + 2 * x]), __uint_as_float(v[q * 8 + 2 * x + 1]));
-              pk[x] = *reinterpret_cast<uint32_t*>(&h);
+            for (int x = 0; x < 16; ++x) {
+              __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[2 * x]), __uint_as_float(v[2 * x + 1]));
+              pk[half * 16 + x] = *reinterpret_cast<uint32_t*>(&h);
             }
-            dst[q] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
           }
-        } else {
-          float4* dst = reinterpret_cast<float4*>(zeta + out_row * kHeadDim + (n - kHeadDim * kHeadDim));
 #pragma unroll
-          for (int q = 0; q < 8; ++q)
-            dst[q] = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]), __uint_as_float(v[4 * q + 2]),
-                                 __uint_as_float(v[4 * q + 3]));
+          for (int ch = 0; ch < 8; ++ch)
+            *reinterpret_cast<uint4*>(stage + lane * 128 + ((ch ^ (lane & 7)) << 4)) =
+                make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
+          __syncwarp();
+          const int ch = lane & 7;
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const int rr = 4 * k + (lane >> 3);
+            const int ir = i0 + quarter * 32 + rr;
+            const uint4 val = *reinterpret_cast<const uint4*>(stage + rr * 128 + ((ch ^ (rr & 7)) << 4));
+            if (ir < nb)
+              *reinterpret_cast<uint4*>(g16 + (bh_rows + ir) * kHeadDim * kHeadDim + n + ch * 8) = val;
+          }
+          __syncwarp();
+        } else {
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            uint32_t v[32];
+            tmem_ld32(lane_addr + pp * 64 + half * 32, v);
+            tmem_wait_ld();
+            if (!row_ok) continue;
+            float4* dst = reinterpret_cast<float4*>(zeta + out_row * kHeadDim + (n - kHeadDim * kHeadDim) + half * 32);
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              dst[q] = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
+                                   __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
+          }
         }
       }
     }
