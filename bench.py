@@ -34,12 +34,12 @@ FP8_OVER_BF16 = 2.0  # nominal dense ratio (4.5 vs 2.25 PFLOP/s)
 # DRAM bytes (read + write) of one launch, keyed by (workload, kernel), from the ncu captures summarised under
 # profiles/; a kernel that changed since its capture has no entry.
 DRAM_BYTES_PER_LAUNCH = {
-    ("vggt8", "attention"): 82515712,
-    ("vggt8", "plan"): 1466880,
-    ("vggt8", "quantize_qkv"): 72599040,
-    ("vggt8", "summary"): 22852864,
-    ("vggt8", "aggregation"): 23396352,
-    ("vggt8", "prep"): 11289344,
+    ("vggt8", "attention"): 83469824,
+    ("vggt8", "plan"): 1488384,
+    ("vggt8", "quantize_qkv"): 72978176,
+    ("vggt8", "summary"): 22844672,
+    ("vggt8", "aggregation"): 23396096,
+    ("vggt8", "prep"): 11299072,
 }
 
 
