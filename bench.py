@@ -122,10 +122,10 @@ def kernel_work(wl, plan):
         "quantize_qkv": ("hbm", 3 * (valid_elems * src_bytes + elems + tiles * 4) + 2 * tiles * 256),
         # fp64 FMAs of the pooled scores (the selection itself is integer work on top)
         "plan": ("alu_fp64", 2.0 * wl.batch * wl.heads * nb * nb * wl.head_dim),
-        # read V codes, write fp16 operand
+        # read V codes, write fp16 operand (a pass of its own only without a linear branch)
         "prep": ("hbm", elems * 3),
-        # read K and V codes, write one bf16 summary row per tile
-        "summary": ("hbm", 2 * elems + tiles * 4160 * 2),
+        # read K and V codes, write one bf16 summary row per tile and, next to a sparse branch, the fp16 V operand
+        "summary": ("hbm", 2 * elems + tiles * 4160 * 2 + (elems * 2 if plan.k_crit > 0 else 0)),
         # 0/1-mask GEMM over the summaries
         "aggregation": ("tensor_bf16", 2.0 * wl.batch * wl.heads * nb * nb * 4160),
         # QK^T and PV of every (query block, critical key block) pair

@@ -106,7 +106,7 @@ lite3r_status launch_attention(const AttentionLaunch& a, cudaStream_t stream);
 
 // Per-key-block summaries ((H_j W)^T | z_j) in bf16, one kSummaryRow-wide row per (b, h, key block).
 lite3r_status launch_summary(const lite3r_fp8& k, const lite3r_fp8& v, const float* proj, long long proj_head_stride,
-                             const lite3r_shape& s, int phi, __nv_bfloat16* hws, int* device_status,
+                             const lite3r_shape& s, int phi, __nv_bfloat16* hws, __half* v16, int* device_status,
                              cudaStream_t stream);
 
 // Marginal aggregation G_i = sum over marginal j of the summary rows, as a 0/1-mask GEMM on tensor cores.

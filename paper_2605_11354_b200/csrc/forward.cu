@@ -89,7 +89,10 @@ lite3r_status run_forward(const ForwardArgs& a, cudaStream_t stream) {
   const Workspace w = carve(a.workspace, s);
   lite3r_status st;
   profile_mark(0, stream);
-  if (a.plan.k_crit > 0) {
+  // With a linear branch the summary kernel reads every V row anyway and writes the fp16 operand on the way; the
+  // stand-alone pass runs only when there is no linear branch.
+  const bool v16_from_summary = a.plan.k_marg > 0;
+  if (a.plan.k_crit > 0 && !v16_from_summary) {
     const size_t words = static_cast<size_t>(rows) * BS * kHeadDim / 16;  // 16 codes per thread and pass
     int sms = 0;
     if ((st = sm_count(&sms)) != LITE3R_OK) return st;
@@ -100,7 +103,8 @@ lite3r_status run_forward(const ForwardArgs& a, cudaStream_t stream) {
   }
   if (a.plan.k_marg > 0) {
     profile_mark(2, stream);
-    st = launch_summary(a.k, a.v, a.proj, a.proj_head_stride, s, a.phi, w.hws, a.device_status, stream);
+    st = launch_summary(a.k, a.v, a.proj, a.proj_head_stride, s, a.phi, w.hws, a.plan.k_crit > 0 ? w.v16 : nullptr,
+                        a.device_status, stream);
     if (st != LITE3R_OK) return st;
     profile_mark(3, stream);
     profile_mark(4, stream);

@@ -13,7 +13,9 @@
 // TMEM sub-partition), one key block at block 128.  Per round the 128 compute threads (one token row each) dequantise
 // their K row, apply the feature map, and write phi and the V code values to shared memory in the operands' swizzled
 // layouts; one thread of a fifth warp issues the MMAs; the compute threads then move H from TMEM to shared memory
-// (scaled, fp16), and finally (H W)^T from TMEM to global memory.  Rounds of one CTA are serial; four CTAs per SM
+// (scaled, fp16), and finally (H W)^T from TMEM to global memory (rows parked in shared memory first, so that stores
+// write whole 128-byte rows).  Next to a sparse branch the kernel also writes the dequantised V rows it has just read
+// (fp16, the attention kernel's P V operand), which saves a pass of its own over V.  Rounds of one CTA are serial; four CTAs per SM
 // overlap their phases.  Every barrier wait is bounded.
 #include "common.cuh"
 #include "sm100.cuh"
@@ -53,6 +55,7 @@ struct SummaryParams {
   int heads, tokens, nb, phi;
   int rounds_per_head, rounds;
   __nv_bfloat16* hws;
+  __half* v16;  // when not NULL: also writes the dequantised V rows (code value x block scale, fp16) read on the way
   int* status;
 };
 
@@ -290,6 +293,28 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) summary_kernel(const Sum
           store_row_swizzled(smem + kOffV, t, vw);
         }
         store_row_swizzled(smem + kOffA, t, pw);
+        if (p.v16 != nullptr && j < p.nb) {
+          // The attention kernel's P V operand (code value x block scale as fp16, the stand-alone pass's arithmetic),
+          // from the rows this warp has just put into the V operand tile (zeros past the end of the sequence): read
+          // back so that a store instruction writes four whole 128-byte rows.
+          __syncwarp();
+          const float sv = __ldg(p.v_scales + bh_rows + j);
+          const int r0 = warp * 32, ch = lane & 7;
+          uint4* dst = reinterpret_cast<uint4*>(p.v16 + ((bh_rows + j) * BS + (r0 % BS)) * kHeadDim) + ch;
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const int rr = 4 * k + (lane >> 3), row = r0 + rr;
+            const uint4 raw = *reinterpret_cast<const uint4*>(smem + kOffV + row * 128 + ((ch ^ (row & 7)) << 4));
+            const uint32_t in[4] = {raw.x, raw.y, raw.z, raw.w};
+            uint32_t o[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const float2 f = half2_bits_to_float2(in[q]);
+              o[q] = float2_to_half2_bits(f.x * sv, f.y * sv);
+            }
+            dst[rr * 8] = make_uint4(o[0], o[1], o[2], o[3]);
+          }
+        }
       }
       fence_proxy_async_smem();
       mbar_arrive(&bars->ab_full);
@@ -330,21 +355,29 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) summary_kernel(const Sum
         tmem_wait_ld();
         tc_fence_before();
         const int j = j0 + hf;
-        if (acc_live && j < p.nb) {
+        if (acc_live && j < p.nb)
           p.hws[(bh_rows + j) * kSummaryRow + kHeadDim * kHeadDim + d_row] = __float2bfloat16_rn(__uint_as_float(zbits));
-          uint4* dst = reinterpret_cast<uint4*>(p.hws + (bh_rows + j) * kSummaryRow + d_row * kHeadDim);
+        // A thread owns one 128-byte row of (H W)^T; stored directly, an instruction would touch 32 lines.  The warp
+        // parks its 32 rows in its own part of the V / H operand space (both MMAs have completed; the same threads
+        // refill exactly these rows in the next round) and stores four whole rows per instruction.
+        uint32_t ow[32];
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            dst[c] = make_uint4(float2_to_bf162_bits(__uint_as_float(lo[8 * c]), __uint_as_float(lo[8 * c + 1])),
-                                float2_to_bf162_bits(__uint_as_float(lo[8 * c + 2]), __uint_as_float(lo[8 * c + 3])),
-                                float2_to_bf162_bits(__uint_as_float(lo[8 * c + 4]), __uint_as_float(lo[8 * c + 5])),
-                                float2_to_bf162_bits(__uint_as_float(lo[8 * c + 6]), __uint_as_float(lo[8 * c + 7])));
-            dst[4 + c] = make_uint4(float2_to_bf162_bits(__uint_as_float(hi[8 * c]), __uint_as_float(hi[8 * c + 1])),
-                                    float2_to_bf162_bits(__uint_as_float(hi[8 * c + 2]), __uint_as_float(hi[8 * c + 3])),
-                                    float2_to_bf162_bits(__uint_as_float(hi[8 * c + 4]), __uint_as_float(hi[8 * c + 5])),
-                                    float2_to_bf162_bits(__uint_as_float(hi[8 * c + 6]), __uint_as_float(hi[8 * c + 7])));
-          }
+        for (int c = 0; c < 16; ++c) {
+          ow[c] = float2_to_bf162_bits(__uint_as_float(lo[2 * c]), __uint_as_float(lo[2 * c + 1]));
+          ow[16 + c] = float2_to_bf162_bits(__uint_as_float(hi[2 * c]), __uint_as_float(hi[2 * c + 1]));
         }
+        store_row_swizzled(smem + kOffV, warp * 32 + lane, ow);
+        __syncwarp();
+        const int ch = lane & 7;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const int rr = 4 * k + (lane >> 3), src_row = warp * 32 + rr;
+          const uint4 val = *reinterpret_cast<const uint4*>(smem + kOffV + src_row * 128 + ((ch ^ (src_row & 7)) << 4));
+          const int hf_r = rr >> 4, j_r = j0 + hf_r;  // lane rr of the warp holds row warp * 16 + (rr & 15) of tile hf_r
+          if (hf_r < kTilesPerRound && j_r < p.nb)
+            *reinterpret_cast<uint4*>(p.hws + (bh_rows + j_r) * kSummaryRow + (warp * 16 + (rr & 15)) * kHeadDim + ch * 8) = val;
+        }
+        __syncwarp();
       }
     }
     (void)ok;
@@ -371,7 +404,7 @@ lite3r_status launch(const SummaryParams& p, int sm_count, cudaStream_t stream) 
 }  // namespace
 
 lite3r_status launch_summary(const lite3r_fp8& k, const lite3r_fp8& v, const float* proj, long long proj_head_stride,
-                             const lite3r_shape& s, int phi, __nv_bfloat16* hws, int* device_status,
+                             const lite3r_shape& s, int phi, __nv_bfloat16* hws, __half* v16, int* device_status,
                              cudaStream_t stream) {
   SummaryParams p;
   p.k_codes = k.codes;
@@ -387,6 +420,7 @@ lite3r_status launch_summary(const lite3r_fp8& k, const lite3r_fp8& v, const flo
   p.rounds_per_head = ceil_div(p.nb, 128 / s.block);
   p.rounds = s.batch * s.heads * p.rounds_per_head;
   p.hws = hws;
+  p.v16 = v16;
   p.status = device_status;
   int sms = 0;
   lite3r_status st = sm_count(&sms);
