@@ -268,6 +268,45 @@ def run_ours(args, wl):
         out = eng.run(dev["q"], dev["k"], dev["v"], proj)
         out_host.copy_(out, non_blocking=True)
 
+    def timed_e2e(steps):
+        """`steps` steps through the public API, each with its sources copied in from pinned host memory and its
+        result copied back to pinned host memory, everything inside one timed region.  Three streams (copy-in,
+        compute, copy-out) and two sets of device sources and results: the copies of neighbouring steps overlap the
+        kernels and each other (PCIe is full duplex).  L2 is not flushed inside the region; a step touches about
+        0.2 GB (sources, codes, operands, result), more than the 126 MB of L2."""
+        cur = torch.cuda.current_stream(device)
+        s_in, s_out = torch.cuda.Stream(device), torch.cuda.Stream(device)
+        srcs = [dev, {n: torch.empty_like(dev[n]) for n in dev}]
+        outs = [eng.out, torch.empty_like(eng.out)]
+        out_hosts = [out_host, torch.empty_like(out_host).pin_memory()]
+        consumed, read_back = [None, None], [None, None]
+        flush.fill_(1)
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        start.record(cur)
+        s_in.wait_stream(cur)
+        s_out.wait_stream(cur)
+        for i in range(steps):
+            b = i & 1
+            with torch.cuda.stream(s_in):
+                if consumed[b] is not None:
+                    s_in.wait_event(consumed[b])  # the step that last used these source buffers has run
+                for n in ("q", "k", "v"):
+                    srcs[b][n].copy_(host[n], non_blocking=True)
+                arrived = s_in.record_event()
+            cur.wait_event(arrived)
+            if read_back[b] is not None:
+                cur.wait_event(read_back[b])  # this result buffer has reached the host
+            eng.run(srcs[b]["q"], srcs[b]["k"], srcs[b]["v"], proj, out=outs[b])
+            consumed[b] = cur.record_event()
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(consumed[b])
+                out_hosts[b].copy_(outs[b], non_blocking=True)
+                read_back[b] = s_out.record_event()
+        cur.wait_stream(s_out)  # the region ends when the last result is on the host
+        end.record(cur)
+        end.synchronize()
+        return start.elapsed_time(end)
+
     def timed(fn, steps, collect_stages):
         total_ms, stages = 0.0, []
         for _ in range(steps):
@@ -297,7 +336,7 @@ def run_ours(args, wl):
     launches = lt.launch_count() - launches0
     torch.cuda.synchronize(device)
     pdist.barrier(device)
-    e2e_total, _ = timed(step_e2e, args.steps, False)
+    e2e_total = timed_e2e(args.steps)
     torch.cuda.synchronize(device)
     pdist.barrier(device)
     clocks = sampler.stop()
@@ -343,6 +382,7 @@ def run_ours(args, wl):
                        "head_dim": wl.head_dim, "block": wl.block, "crit": wl.crit, "neg": wl.neg,
                        "k_crit": eng.plan.k_crit, "k_marg": eng.plan.k_marg, "k_neg": eng.plan.k_neg,
                        "source_dtype": wl.src_dtype, "l2": f"flushed between timed steps ({L2_FLUSH_BYTES >> 20} MiB write)",
+                       "e2e_pipeline": "copy-in, compute and copy-out streams over two buffer sets; no L2 flush inside",
                        "parallelism": "independent replicas, no collective" if world > 1 else "single GPU"},
             "e2e": {"value": e2e_flops / 1e12, "unit": UNIT, "h2d_bytes_per_step": in_bytes,
                     "d2h_bytes_per_step": out_bytes},

@@ -297,12 +297,14 @@ class SlaForward:
     def make_plan(self, stream=None):
         lite3r_sla_plan(self.q8, self.k8, self.shape, self.crit, self.neg, self.plan, stream)
 
-    def forward(self, proj, stream=None):
-        lite3r_sla_forward(self.q8, self.k8, self.v8, proj, self.shape, self.phi, self.plan, self.out,
+    def forward(self, proj, stream=None, out=None):
+        """out: optional result tensor of the engine's output shape (default: the engine's own ``out``)."""
+        out = self.out if out is None else out
+        lite3r_sla_forward(self.q8, self.k8, self.v8, proj, self.shape, self.phi, self.plan, out,
                            self.workspace, self.status, stream)
-        return self.out
+        return out
 
-    def run(self, q, k, v, proj, stream=None):
+    def run(self, q, k, v, proj, stream=None, out=None):
         self.quantize(q, k, v, stream)
         self.make_plan(stream)
-        return self.forward(proj, stream)
+        return self.forward(proj, stream, out)
