@@ -8,8 +8,7 @@
 // round-to-nearest-even and written with 8-byte stores.  The same pass emits, where asked for, the per-tile column
 // sums of the code values as exact integers (units of 2^-9), which is all the block plan needs.  HBM traffic: 2
 // (bf16) or 4 (fp32) bytes read and 1 byte written per element; the instruction count per element decides how
-// close the kernel gets to that, hence the packed fp32x2 arithmetic and the bf16 maximum taken on bit patterns.
-// Sources are expected to be finite (a NaN would become the tile maximum).
+// close the kernel gets to that, hence the packed fp32x2 arithmetic.
 #include "common.cuh"
 #include "sm100.cuh"
 
@@ -64,16 +63,6 @@ __device__ __forceinline__ void unpack8(const float* p, float v[8]) {
   v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
   v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
 }
-
-// Largest magnitude of eight values as a float.  bf16 magnitudes are ordered like their bit patterns, so two of them
-// are compared per 16-bit-pair instruction before anything is unpacked.
-__device__ __forceinline__ uint32_t amax8_bits(const __nv_bfloat16* p, uint32_t acc) {
-  const uint4 w = *reinterpret_cast<const uint4*>(p);
-  acc = __vmaxu2(acc, __vmaxu2(w.x & 0x7FFF7FFFu, w.y & 0x7FFF7FFFu));
-  return __vmaxu2(acc, __vmaxu2(w.z & 0x7FFF7FFFu, w.w & 0x7FFF7FFFu));
-}
-__device__ __forceinline__ uint32_t amax8_bits(const float*, uint32_t acc) { return acc; }  // fp32 sources compare as floats
-__device__ __forceinline__ float amax_finish(uint32_t acc) { return __uint_as_float(max(acc << 16, acc & 0xFFFF0000u)); }
 
 // Persistent CTAs walk the tiles with a stride of the grid size.  Tiles travel global -> shared memory through
 // asynchronous copies, kDepth tiles ahead of the one being processed, so the bytes a CTA keeps in flight are set by
@@ -157,23 +146,12 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const __grid_constan
     float v[kKeep ? kPasses : 1][8];
     const uint8_t* const mine = ring + slot * kTileBytes + threadIdx.x * kSegBytes;
     float amax = 0.f;
-    if (sizeof(SrcT) == 2) {
-      uint32_t acc = 0;
 #pragma unroll
-      for (int p = 0; p < kPasses; ++p) {
-        const SrcT* const src = reinterpret_cast<const SrcT*>(mine + p * kThreads * kSegBytes);
-        acc = amax8_bits(src, acc);
-        if (kKeep) unpack8(src, v[kKeep ? p : 0]);
-      }
-      amax = amax_finish(acc);
-    } else {
+    for (int p = 0; p < kPasses; ++p) {
+      float* const vp = v[kKeep ? p : 0];
+      unpack8(reinterpret_cast<const SrcT*>(mine + p * kThreads * kSegBytes), vp);
 #pragma unroll
-      for (int p = 0; p < kPasses; ++p) {
-        float* const vp = v[kKeep ? p : 0];
-        unpack8(reinterpret_cast<const SrcT*>(mine + p * kThreads * kSegBytes), vp);
-#pragma unroll
-        for (int c = 0; c < 8; ++c) amax = fmaxf(amax, fabsf(vp[c]));
-      }
+      for (int c = 0; c < 8; ++c) amax = fmaxf(amax, fabsf(vp[c]));
     }
     slot = slot + 1 == kDepth ? 0 : slot + 1;
 
