@@ -59,6 +59,9 @@ WORKLOADS = {
     "vggt32": Workload("vggt32", 3, 1, 16, 32 * TOKENS_PER_FRAME, 64, 64, 0.05, 0.75, 64, 0.3, "bf16"),
     "da3l": Workload("da3l", 4, 4, 16, 16 * TOKENS_PER_FRAME, 64, 128, 0.08, 0.70, 128, 0.5, "bf16"),
     "stress100": Workload("stress100", 5, 1, 16, 100 * TOKENS_PER_FRAME, 64, 64, 0.10, 0.60, 64, 0.3, "bf16"),
+    # frame attention: every frame is a sequence of its own (batch = frames), 22 blocks of 64 tokens, the last one
+    # with 30; the short-sequence regime where launch, plan and ragged-block costs weigh most
+    "frame32": Workload("frame32", 6, 32, 16, TOKENS_PER_FRAME, 64, 64, 0.25, 0.50, 64, 0.3, "bf16"),
 }
 STRESS_SWEEP = ((0.02, 0.60), (0.05, 0.60), (0.10, 0.60), (0.25, 0.60), (1.00, 0.00))
 

@@ -179,8 +179,14 @@ def test_da3l_cut_every_block():
     full_parity(wl, wk.make_inputs(wl))
 
 
+def test_frame_attention_cut_every_block():
+    """Frame attention (one short sequence per frame, batch = frames): three frames, two heads, every query block."""
+    wl = wk.scaled_down(wk.WORKLOADS["frame32"], heads=2, batch=3)
+    full_parity(wl, wk.make_inputs(wl))
+
+
 @pytest.mark.parametrize("name,oracle_heads,samples", [("vggt8", [0, 7, 15], 40), ("vggt32", [3, 12], 32),
-                                                       ("da3l", [5], 32)])
+                                                       ("da3l", [5], 32), ("frame32", [4, 11], 48)])
 def test_full_size_configs_on_sampled_blocks(name, oracle_heads, samples):
     """The launch configuration the benchmark times, checked on a seeded sample of query blocks (always block 0,
     the ragged last block and one block per checked head); quantiser and plan are compared in full for those heads."""
