@@ -45,7 +45,7 @@ typedef enum {
 typedef enum { LITE3R_F32 = 0, LITE3R_BF16 = 1 } lite3r_dtype;
 
 /* Feature map of the linear branch.  SOFTMAX: softmax over the head_dim components (the benchmark
- * contract).  ELU1: ELU(x)+1 (Algorithm 1, line 6). */
+ * contract).  ELU1: ELU(x)+1 (the feature map Algorithm 1 prints). */
 typedef enum { LITE3R_PHI_SOFTMAX = 0, LITE3R_PHI_ELU1 = 1 } lite3r_phi;
 
 typedef struct {
@@ -89,7 +89,7 @@ LITE3R_API lite3r_status lite3r_fp8_sizes(const lite3r_shape* shape, size_t* cod
 
 /* Per-row class counts and plan buffer sizes.  Counts: k_crit = 0 if crit == 0, else
  * min(Nb, max(1, floor(crit*Nb + 0.5))); k_neg = min(Nb - k_crit, floor(neg*Nb + 0.5)); k_marg is the rest
- * (the row-wise TopKMask of Algorithm 1 line 3 with its keep ratio, applied to blocks).  Host-only. */
+ * (the row-wise TopKMask of Algorithm 1 with its keep ratio, applied to blocks).  Host-only. */
 LITE3R_API lite3r_status lite3r_plan_sizes(const lite3r_shape* shape, double crit, double neg, size_t* cls_bytes,
                                 size_t* crit_idx_bytes, size_t* marg_idx_bytes, int* k_crit, int* k_marg,
                                 int* k_neg);
@@ -112,7 +112,7 @@ LITE3R_API lite3r_status lite3r_quantize_fp8_qkv(const lite3r_tensor* q, const l
                                       const lite3r_shape* shape, lite3r_fp8 q_out, lite3r_fp8 k_out, lite3r_fp8 v_out,
                                       void* stream);
 
-/* Pooled scores and row-wise top-k classification (Algorithm 1 lines 2-3 on block means):
+/* Pooled scores and row-wise top-k classification (the score and TopKMask steps of Algorithm 1 on block means):
  *   s_ij = mean_i(q_hat) . mean_j(k_hat) / sqrt(D), means over valid tokens of the dequantised blocks;
  *   row i ranks j by (s_ij descending, j ascending); first k_crit critical, last k_neg negligible.
  * Scores are evaluated from the exact integer column sums in fp64, so the ranking can differ from an exact
@@ -121,7 +121,7 @@ LITE3R_API lite3r_status lite3r_quantize_fp8_qkv(const lite3r_tensor* q, const l
 LITE3R_API lite3r_status lite3r_sla_plan(const lite3r_fp8* q, const lite3r_fp8* k, const lite3r_shape* shape, double crit,
                               double neg, lite3r_plan* plan, void* stream);
 
-/* The SLA forward (Eq. 1; Algorithm 1 lines 4-10) for a given plan.
+/* The SLA forward (Eq. 1; Algorithm 1 from the sparse softmax on) for a given plan.
  *   sparse branch: per query token, softmax over exactly the valid keys of the critical blocks of
  *     (q_hat . k_hat) / sqrt(D), times v_hat;
  *   linear branch: (phi(q_hat) G_i) / (phi(q_hat) . zeta_i) with G_i = sum over marginal blocks of

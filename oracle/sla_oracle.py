@@ -18,9 +18,9 @@ Conventions
 * Pins (checked in tests/test_oracle_pins.py): the e4m3 codec against the
   closed-form format definition and torch's float8_e4m3fn cast; crit=1 against
   dense softmax attention; crit=0,neg=0 against the global linear-attention
-  closed form (Algorithm 1, lines 6-10); brute-force per-query evaluation on
+  closed form (Algorithm 1, its linear branch, projection and sum); brute-force per-query evaluation on
   tiny inputs; constant-V, phi-summary and permutation invariants; block=1
-  against Algorithm 1 lines 2-5 evaluated per token.  Beyond those pins the
+  against Algorithm 1's score, mask and sparse-softmax steps evaluated per token.  Beyond those pins the
   output values of the general three-class case rest on the definition itself
   (the paper prints no worked numeric example): parity unpinned past the pins.
 """
@@ -129,7 +129,7 @@ def block_means(xhat: np.ndarray, block: int) -> np.ndarray:
 
 def pooled_scores(qhat: np.ndarray, khat: np.ndarray, block: int) -> np.ndarray:
     """Compressed scores s_ij = (mean_i(q) . mean_j(k)) / sqrt(D): [B,H,Nb,Nb]
-    (Algorithm 1 line 2 applied to block means)."""
+    (the score step of Algorithm 1 applied to block means)."""
     D = qhat.shape[-1]
     return np.einsum("bhid,bhjd->bhij", block_means(qhat, block), block_means(khat, block)) / math.sqrt(D)
 
@@ -144,7 +144,7 @@ def class_counts(nb: int, crit: float, neg: float):
 
 
 def classify(scores: np.ndarray, crit: float, neg: float) -> np.ndarray:
-    """Row-wise top-k (Algorithm 1 line 3, per query block): rank the key blocks of each row
+    """Row-wise top-k (the TopKMask step of Algorithm 1, per query block): rank the key blocks of each row
     by score descending, ties to the lower key-block index; the first k_crit are critical (2),
     the last k_neg negligible (0), the rest marginal (1).  Returns int8 [B,H,Nb,Nb]."""
     nb = scores.shape[-1]
@@ -182,7 +182,7 @@ def phi_softmax(x: np.ndarray) -> np.ndarray:
 
 
 def phi_elu1(x: np.ndarray) -> np.ndarray:
-    """Feature map of Algorithm 1 line 6: ELU(x) + 1."""
+    """Feature map of Algorithm 1: ELU(x) + 1."""
     return np.where(x > 0, x + 1.0, np.exp(np.minimum(x, 0.0)))
 
 
@@ -192,7 +192,7 @@ PHI = {"softmax": phi_softmax, "elu1": phi_elu1}
 # --------------------------------------------------------------------------- linear-branch summaries
 def kv_summaries(khat: np.ndarray, vhat: np.ndarray, block: int, phi: str = "softmax"):
     """Per key block j: H_j = phi(K_j)^T V_j [D,D] and z_j = phi(K_j)^T 1 [D]
-    (Algorithm 1 lines 7-8 restricted to one block), valid tokens only."""
+    (the KV-summary and normaliser steps of Algorithm 1 restricted to one block), valid tokens only."""
     B, H, N, D = khat.shape
     Nb = n_blocks(N, block)
     f = PHI[phi]
@@ -211,11 +211,11 @@ def sla_forward(qhat, khat, vhat, proj, cls, block, phi="softmax", query_blocks=
     """A_SLA = A_sparse + Proj(A_lin) (Eq. 1), block-level classes taken from ``cls``.
 
     qhat/khat/vhat: dequantised fp64 [B,H,N,D]; proj: [H,D,D] (or [D,D] shared), applied as
-    O_lin @ W (Algorithm 1 line 10, no bias); cls: int8 [B,H,Nb,Nb].
+    O_lin @ W (the projection-and-sum step of Algorithm 1, no bias); cls: int8 [B,H,Nb,Nb].
     For the query tokens of block i of (b, h):
-      sparse branch (lines 4-5): softmax over exactly the valid keys of the critical blocks of
+      sparse branch (Algorithm 1's masked softmax and its product with V): softmax over exactly the valid keys of the critical blocks of
         (q . k) / sqrt(D), times V; zero when there is no critical block;
-      linear branch (lines 6-9) over the valid keys of the marginal blocks only:
+      linear branch (Algorithm 1's feature map, summaries and normalised output) over the valid keys of the marginal blocks only:
         (phi(q) G_i) / (phi(q) . zeta_i) with G_i, zeta_i the sums of the per-block
         summaries; zero when there is no marginal block.
     ``query_blocks``: iterable of (b, h, i) to evaluate (default all).  Returns fp64 [B,H,N,D]

@@ -1,4 +1,4 @@
-// K4: critical-block softmax attention + linear branch + add (Algorithm 1 lines 4-5, 9-10) on tcgen05 / TMEM / TMA.
+// K4: critical-block softmax attention + linear branch + add (Algorithm 1's sparse branch, linear output, projection and sum) on tcgen05 / TMEM / TMA.
 //
 // One CTA owns 128 query rows of one (b, h): at block 64 a PAIR of query blocks (two M=64 accumulators interleaved
 // in the two 16-lane halves of every TMEM sub-partition), at block 128 one query block (M=128).  Work advances in

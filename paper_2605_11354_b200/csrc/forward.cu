@@ -1,11 +1,11 @@
-// K3 / K3b / K4: the SLA forward for a given block plan (Eq. 1; Algorithm 1 lines 4-10).
+// K3 / K3b / K4: the SLA forward for a given block plan (Eq. 1; Algorithm 1 from the sparse softmax on).
 //
-//   K3  summary.cu        per key block j:  H_j = phi(K_j)^T V_j, z_j = phi(K_j)^T 1  (lines 7-8 per block), stored as
+//   K3  summary.cu        per key block j:  H_j = phi(K_j)^T V_j, z_j = phi(K_j)^T 1  (KV summary and normaliser, per block), stored as
 //                         (H_j W)^T and z_j in bf16 (output projection folded in early).
 //   K3b aggregate.cu      per query block i:  G_i = sum over marginal j of (H_j W)^T,  zeta_i = sum of z_j.
-//   K4  attention.cu      per query block i: online-softmax attention over the critical key blocks (lines 4-5),
-//                         then the linear branch (line 9) phi(q) G_i / (phi(q) . zeta_i), the sum of the two
-//                         (line 10) and the store.
+//   K4  attention.cu      per query block i: online-softmax attention over the critical key blocks (sparse branch),
+//                         then the linear output phi(q) G_i / (phi(q) . zeta_i), the sum of the two
+//                         and the store.
 //   prep_kernel           dequantised V as fp16 for the attention kernel's P V product.
 #include <algorithm>
 

@@ -1,4 +1,4 @@
-// K2: pooled scores and row-wise top-k block classification (Algorithm 1 lines 2-3 on block means).
+// K2: pooled scores and row-wise top-k block classification (the score and TopKMask steps of Algorithm 1 on block means).
 //
 // The pooled mean of block i is colsum_i * 2^-9 * scale_i / valid_i with colsum an exact integer vector, so
 //   s_ij = (colsum^Q_i . colsum^K_j) * [scale^K_j / valid_j] * [scale^Q_i / (valid_i * 8 * 2^18)].
@@ -7,16 +7,20 @@
 // roundings separate t_ij from the exact value; the ranking is therefore the exact one except between
 // scores that agree to ~1e-15 relative.  Ranking order: score descending, then key-block index ascending.
 //
-// One CTA of R warps handles R consecutive query blocks (rows) of one (b, h).
-//   Phase A (whole CTA): the scores of the R rows against all key blocks, 64 staged key blocks at a time; a lane
-//     owns one key block and R/4 rows, so every staged value feeds several fp64 FMAs.  Scores are kept in shared
-//     memory as order-preserving 64-bit keys.
-//   Phase B (one warp per row): "the k best of the row" is found by a most-significant-digit-first radix select
-//     over the 64-bit keys (8-bit digits placed at the highest bit on which the remaining candidates differ,
-//     per-warp histogram in shared memory): it yields a key prefix such that
-//     every entry above it is selected, and of the entries equal to it the first `take` in index order are.  That
-//     is exactly the total order (score descending, index ascending), at O(Nb) work per row.  Two selections
-//     give the classes: the best k_crit are critical, the best Nb - k_neg are critical-or-marginal.
+// One CTA of R warps handles R consecutive query blocks (rows) of one (b, h); R = 8 unless the row keys of a very
+// long sequence do not fit in shared memory.
+//   Phase A (whole CTA): the scores of the R rows against all key blocks, kept in shared memory as order-preserving
+//     64-bit keys.  R = 8: fp64 tensor-core products (m8n8k4) fed with the int32 column sums straight from global
+//     memory, no staging and no barrier.  R < 8: 64 key blocks at a time staged in shared memory as doubles; a lane
+//     owns one key block and R/4 rows, so every staged value feeds several fp64 FMAs.
+//   Phase B (one warp per row): "the k best of the row".  A histogram over 256 buckets that are linear in the score
+//     places the k-th best in a bucket of usually a handful of keys; those are listed by index and a
+//     most-significant-digit-first radix select over their 64-bit keys (8-bit digits placed at the highest bit on
+//     which the remaining candidates differ, per-warp histogram in shared memory) decides between them: it yields a
+//     key prefix such that every entry above it is selected, and of the entries equal to it the first `take` in
+//     index order are.  That is exactly the total order (score descending, index ascending), at O(Nb) work per
+//     row.  Two selections give the classes: the best k_crit are critical, the best Nb - k_neg are
+//     critical-or-marginal.
 //   Phase C (same warp): class row and ascending index lists, written with ballot prefix sums.
 #include "common.cuh"
 

@@ -1,4 +1,4 @@
-// K3: per-key-block summaries of the linear branch (Algorithm 1 lines 6-8, per block) on tcgen05 tensor cores.
+// K3: per-key-block summaries of the linear branch (Algorithm 1's feature map, KV summary and normaliser, per block) on tcgen05 tensor cores.
 //
 // For key block j:  H_j = phi(K_j)^T V_j  (64 x 64),  z_j = phi(K_j)^T 1  (64), with the output projection folded in
 // early: the kernel stores (H_j W)^T and z_j in bf16.  Folding is exact algebra:

@@ -166,10 +166,10 @@ def test_all_marginal_equals_linear_attention_closed_form(phi):
         fq, fk = torch.softmax(tq, -1), torch.softmax(tk, -1)
     else:
         fq, fk = torch.nn.functional.elu(tq) + 1, torch.nn.functional.elu(tk) + 1
-    T = fk.transpose(-1, -2) @ tv  # phi(K)^T V   (Algorithm 1 line 7)
-    z = fk.sum(dim=-2)  # phi(K)^T 1   (line 8)
-    lin = (fq @ T) / (fq @ z.unsqueeze(-1))  # line 9
-    ref = (lin @ tw.unsqueeze(0)).numpy()  # line 10 with O_sparse = 0
+    T = fk.transpose(-1, -2) @ tv  # phi(K)^T V   (Algorithm 1, KV summary)
+    z = fk.sum(dim=-2)  # phi(K)^T 1   (normaliser)
+    lin = (fq @ T) / (fq @ z.unsqueeze(-1))  # linear output
+    ref = (lin @ tw.unsqueeze(0)).numpy()  # projection and sum with O_sparse = 0
     assert np.allclose(out, ref, rtol=1e-11, atol=1e-13)
 
 
@@ -302,12 +302,12 @@ def test_block_one_equals_token_level_topk_attention():
     cls = orc.classify(orc.pooled_scores(qh, kh, 1), lam, 1.0 - lam)
     assert orc.class_counts(N, lam, 1.0 - lam) == (10, 0, 30)
     out = orc.sla_forward(qh, kh, vh, w, cls, 1)
-    S = qh[0, 0] @ kh[0, 0].T / math.sqrt(D)  # Algorithm 1 line 2
+    S = qh[0, 0] @ kh[0, 0].T / math.sqrt(D)  # Algorithm 1, scores
     ref = np.zeros((N, D))
     for t in range(N):
-        keep = sorted(range(N), key=lambda s: (-S[t, s], s))[:10]  # line 3
-        e = np.exp(S[t, keep] - S[t, keep].max())  # line 4 with masked entries excluded
-        ref[t] = (e / e.sum()) @ vh[0, 0, keep]  # line 5
+        keep = sorted(range(N), key=lambda s: (-S[t, s], s))[:10]  # TopKMask
+        e = np.exp(S[t, keep] - S[t, keep].max())  # sparse softmax with masked entries excluded
+        ref[t] = (e / e.sum()) @ vh[0, 0, keep]  # sparse output
     assert np.allclose(out[0, 0], ref, rtol=1e-12, atol=1e-14)
 
 
