@@ -227,10 +227,13 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) summary_kernel(const Sum
           const size_t tile = bh_rows + j;
           const uint4* ksrc = reinterpret_cast<const uint4*>(p.k_codes + (tile * BS + s) * kHeadDim);
           const uint4* vsrc = reinterpret_cast<const uint4*>(p.v_codes + (tile * BS + s) * kHeadDim);
-          {  // V code values are exact in fp16: straight conversion, stored before the K row needs the registers
-            uint4 vraw[4];
+          // both rows are requested before either is used, so that only one memory latency is exposed
+          uint4 vraw[4], kraw[4];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) vraw[c] = __ldg(vsrc + c);
+          for (int c = 0; c < 4; ++c) vraw[c] = __ldg(vsrc + c);
+#pragma unroll
+          for (int c = 0; c < 4; ++c) kraw[c] = __ldg(ksrc + c);
+          {  // V code values are exact in fp16: straight conversion, stored before the K row needs the registers
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
               const uint32_t vwd[4] = {vraw[c].x, vraw[c].y, vraw[c].z, vraw[c].w};
@@ -242,9 +245,6 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) summary_kernel(const Sum
             }
             store_row_swizzled(smem + kOffV, t, vw);
           }
-          uint4 kraw[4];
-#pragma unroll
-          for (int c = 0; c < 4; ++c) kraw[c] = __ldg(ksrc + c);
           const float sk = __ldg(p.k_scales + tile);
           float x[64];
 #pragma unroll
