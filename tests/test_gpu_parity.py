@@ -168,6 +168,30 @@ def test_ties_resolve_to_lower_index():
     assert np.array_equal(eng.plan.cls.cpu().numpy(), ref["cls"])
 
 
+def test_all_scores_tied_in_a_long_row():
+    """Zero queries make every pooled score of a row equal (one bucket holding all 150 blocks, more than the
+    candidate list keeps): the selection must fall back to index order, exactly as the oracle ranks them."""
+    wl = small_workload("alltied", tokens=150 * 64, heads=1, src_dtype="bf16", crit=0.2, neg=0.5)
+    inputs = wk.make_inputs(wl)
+    inputs["q"][:] = 0.0
+    eng, _ = pu.run_gpu(inputs, wl)
+    ref = oracle_subset(inputs, wl, [0], query_blocks=[])
+    assert (ref["scores"] == 0).all()
+    cls = eng.plan.cls.cpu().numpy()
+    assert np.array_equal(cls, ref["cls"])
+    k_c, k_m = eng.plan.k_crit, eng.plan.k_marg
+    assert (cls[0, 0, :, :k_c] == 2).all() and (cls[0, 0, :, k_c:k_c + k_m] == 1).all()
+
+
+def test_plan_of_a_very_long_sequence():
+    """3000 blocks: the row keys of eight query blocks no longer fit in shared memory, so the plan kernel runs with
+    four rows per CTA, staged column sums and the whole selection in the radix select.  Quantiser and plan are
+    compared in full, the output on a few sampled query blocks."""
+    wl = small_workload("long", tokens=3000 * 64 - 17, heads=1, src_dtype="bf16", crit=0.01, neg=0.95)
+    inputs = wk.make_inputs(wl)
+    full_parity(wl, inputs, query_blocks=pu.sample_blocks(wl, [0], 6, seed=5))
+
+
 # ------------------------------------------------------------------------------------------------ benchmark shapes
 def test_vggt8_two_heads_every_block():
     wl = wk.scaled_down(wk.WORKLOADS["vggt8"], heads=2)
