@@ -5,11 +5,17 @@
 // accumulation is fp32 in TMEM, so this equals the gather-and-add of the summaries while reading each summary once per
 // 128 query blocks instead of once per query block.
 //
-// One CTA computes a 128 (query blocks) x 256 (summary columns) tile; the reduction runs over key blocks in chunks of
-// 64.  Per chunk: TMA brings the 64 x 256 slab of summaries (MN-major B operand, four 64-column boxes, 128B swizzle);
-// 128 threads expand the class bytes of their query-block row into the bf16 0/1 A tile (K-major, 128B swizzle); one
-// thread issues four 128x256x16 MMAs.  Epilogue: the same 128 threads read their accumulator row from TMEM and store
-// the first 4096 columns as bf16 (the attention kernel's B operand) and the last 64 (zeta) as fp32.
+// One CTA computes a 128 (rows) x 256 (summary columns) tile; the reduction runs over key blocks in chunks of 64.  Rows
+// and keys are numbered through all (b, h).  Tiles either stay inside one (b, h), or, for short sequences, run through
+// the (b, h) boundaries so that several small problems share a tile (the mask is then block-diagonal); the launcher
+// takes the cheaper tiling.  Per chunk: TMA brings the 64 x 256 slab of summaries (MN-major B operand, four 64-column
+// boxes, 128B swizzle); 128 threads expand the class bytes of their row (fetched a chunk ahead) into the bf16 0/1 A
+// tile (K-major, 128B swizzle) with byte permutes; one thread issues four 128x256x16 MMAs.  Epilogue: the same 128
+// threads read their accumulator row from TMEM, turn the rows around in shared memory so that stores write whole
+// 128-byte segments, and store the first 4096 columns as bf16 (the attention kernel's B operand) and the last 64
+// (zeta) as fp32.
+#include <algorithm>
+
 #include "common.cuh"
 #include "sm100.cuh"
 
@@ -38,7 +44,7 @@ struct Bars {
 
 __global__ void __launch_bounds__(kThreads, 2)
 aggregate_mma_kernel(const __grid_constant__ CUtensorMap map_s, const signed char* __restrict__ cls, int nb,
-                     __nv_bfloat16* __restrict__ g16, float* __restrict__ zeta, int* status) {
+                     int total_rows, int flat, __nv_bfloat16* __restrict__ g16, float* __restrict__ zeta, int* status) {
   extern __shared__ __align__(1024) uint8_t smem[];
   Bars* bars = reinterpret_cast<Bars*>(smem + kOffBar);
   volatile int* abort_flag = &bars->abort;
@@ -49,10 +55,24 @@ aggregate_mma_kernel(const __grid_constant__ CUtensorMap map_s, const signed cha
   }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_tile = blockIdx.x;           // 0..16, 256 summary columns each (the last one holds zeta)
-  const int i0 = blockIdx.y * kTileM;      // first query block of the tile
-  const int bh = blockIdx.z;
-  const size_t bh_rows = static_cast<size_t>(bh) * nb;
-  const int chunks = (nb + kChunk - 1) / kChunk;
+  // Rows and keys are numbered through all (b, h): row R = (b h) Nb + i, key (b h) Nb + j, the row numbers of the class
+  // matrix, the summaries and the outputs.  A tile is 128 consecutive rows and reduces over the keys of the (b, h) it
+  // touches.  Long sequences: the tile stays inside one (b, h) (grid z).  Short ones (flat): tiles run through the
+  // (b, h) boundaries, so several small problems share one tile instead of each padding its own; the mask is then
+  // block-diagonal, a row only ever selecting keys of its own (b, h).
+  int row0, row_limit, key0, key_end;
+  if (flat) {
+    row0 = blockIdx.y * kTileM;
+    row_limit = total_rows;
+    key0 = (row0 / nb) * nb;
+    key_end = (min(row0 + kTileM, total_rows) - 1) / nb * nb + nb;
+  } else {
+    key0 = blockIdx.z * nb;
+    key_end = key0 + nb;
+    row0 = key0 + blockIdx.y * kTileM;
+    row_limit = key_end;
+  }
+  const int chunks = (key_end - key0 + kChunk - 1) / kChunk;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -80,7 +100,7 @@ aggregate_mma_kernel(const __grid_constant__ CUtensorMap map_s, const signed cha
         const int st = c % kStages;
         if (!mbar_wait(&bars->empty[st], ((c / kStages) & 1) ^ 1, abort_flag, status, 401)) break;
         mbar_arrive_expect_tx(&bars->b_full[st], kBBytes);
-        const int row = static_cast<int>(bh_rows) + c * kChunk;
+        const int row = key0 + c * kChunk;
         for (int q = 0; q < 4; ++q)  // columns past 4160 and rows past the tensor are zero-filled by TMA
           tma_load_2d(smem + kOffB + st * kBBytes + q * 8192, &map_s, &bars->b_full[st], n_tile * kTileN + q * 64, row);
       }
@@ -108,38 +128,44 @@ aggregate_mma_kernel(const __grid_constant__ CUtensorMap map_s, const signed cha
     }
   } else {
     const int quarter = warp & 3;
-    const int r = quarter * 32 + lane;  // accumulator row = TMEM lane = query block i0 + r
-    const int i = i0 + r;
-    const bool row_ok = i < nb;
-    const signed char* row_ptr = cls + (bh_rows + (row_ok ? i : 0)) * nb;
+    const int r = quarter * 32 + lane;  // accumulator row = TMEM lane = row row0 + r
+    const int row = row0 + r;
+    const bool row_ok = row < row_limit;
+    const int own0 = row_ok ? row / nb * nb : 0;  // first key of this row's (b, h)
+    const signed char* row_ptr = cls + static_cast<size_t>(row_ok ? row : 0) * nb;
     bool ok = true;
-    // The 64 class bytes of this row for chunk c, as the 17 aligned 32-bit words that hold them (rows start at any
-    // byte); fetched one chunk ahead, so that the latency hides behind the wait for the stage and the expansion.
+    // Chunk c covers keys key0 + 64 c ..; of those, positions p_lo .. p_hi - 1 belong to this row's (b, h) and have a
+    // class byte, at row_ptr + (key - own0).  The bytes travel as the aligned 32-bit words that hold them (rows start
+    // at any byte; words without an in-range byte are not read), fetched one chunk ahead, so that the latency hides
+    // behind the wait for the stage and the expansion.
     auto fetch = [&](int c, uint32_t w[17]) {
-      const int j0 = c * kChunk;
-      const uintptr_t addr = reinterpret_cast<uintptr_t>(row_ptr + j0);
-      const uint32_t* wp = reinterpret_cast<const uint32_t*>(addr & ~uintptr_t(3));
-      const int len = min(kChunk, nb - j0);                            // in-range class bytes of this chunk
-      const int words = (static_cast<int>(addr & 3u) + len + 3) / 4;   // aligned words that hold them
+      const int j0 = key0 + c * kChunk - own0;  // class-byte index of position 0: negative before the row's keys
+      const int p_lo = max(0, -j0), p_hi = min(kChunk, nb - j0);
+      const intptr_t addr = reinterpret_cast<intptr_t>(row_ptr) + j0;
+      const uint32_t* wp = reinterpret_cast<const uint32_t*>(addr & ~intptr_t(3));
+      const int a = static_cast<int>(addr & 3);  // word k holds positions 4 k - a .. 4 k - a + 3
+      const int k_lo = (p_lo + a) >> 2;          // first and one-past-last word with an in-range byte
+      const int k_n = (row_ok && c < chunks) ? ((p_hi + a + 3) >> 2) - k_lo : 0;
 #pragma unroll
-      for (int k = 0; k < 17; ++k) w[k] = (row_ok && c < chunks && k < words) ? __ldg(wp + k) : 0u;
+      for (int k = 0; k < 17; ++k) w[k] = static_cast<unsigned>(k - k_lo) < static_cast<unsigned>(max(k_n, 0)) ? __ldg(wp + k) : 0u;
     };
     uint32_t w[17];
     fetch(0, w);
     for (int c = 0; c < chunks; ++c) {
       const int st = c % kStages;
-      const int j0 = c * kChunk;
-      const uint32_t shift = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(row_ptr + j0) & 3u) * 8u;
-      const int len = min(kChunk, nb - j0);
+      const int j0 = key0 + c * kChunk - own0;
+      const int p_lo = max(0, -j0), p_hi = min(kChunk, nb - j0);
+      const uint32_t shift = static_cast<uint32_t>((reinterpret_cast<intptr_t>(row_ptr) + j0) & 3) * 8u;
       // realigned class bytes; bit 0 of a class (0 negligible, 1 marginal, 2 critical) says "marginal"
       uint32_t m[16];
 #pragma unroll
       for (int k = 0; k < 16; ++k) m[k] = __funnelshift_r(w[k], w[k + 1], shift) & 0x01010101u;
-      if (len < kChunk) {  // last chunk: the bytes past the row belong to the next row
+      if (p_lo > 0 || p_hi < kChunk) {  // positions outside the row's keys hold other rows' bytes
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
-          const int left = len - 4 * k;  // in-range bytes of this word
-          m[k] = left >= 4 ? m[k] : (left <= 0 ? 0u : (m[k] & (0xFFFFFFFFu >> (32 - 8 * left))));
+          const int lo = min(max(p_lo - 4 * k, 0), 4), hi = min(max(p_hi - 4 * k, 0), 4);  // bytes lo .. hi - 1 stay
+          const uint32_t keep = lo < hi ? (0xFFFFFFFFu >> (32 - 8 * hi)) & (0xFFFFFFFFu << (8 * lo)) : 0u;
+          m[k] &= keep;
         }
       }
       fetch(c + 1, w);
@@ -159,7 +185,6 @@ aggregate_mma_kernel(const __grid_constant__ CUtensorMap map_s, const signed cha
     if (ok && (ok = mbar_wait(&bars->acc_full, 0, abort_flag, status, 405))) {
       tc_fence_after();
       const uint32_t lane_addr = tmem + ((static_cast<uint32_t>(quarter) * 32u) << 16);
-      const size_t out_row = bh_rows + i;
       // A thread owns one accumulator row, so direct stores would touch 32 different lines per instruction.  Each
       // warp turns its 32 rows x 128 bytes (64 bf16 columns) around in shared memory (the operand stages are free:
       // every MMA has completed) and stores whole 128-byte row segments, four rows per instruction.
@@ -190,10 +215,10 @@ aggregate_mma_kernel(const __grid_constant__ CUtensorMap map_s, const signed cha
 #pragma unroll
           for (int k = 0; k < 8; ++k) {
             const int rr = 4 * k + (lane >> 3);
-            const int ir = i0 + quarter * 32 + rr;
+            const int ir = row0 + quarter * 32 + rr;
             const uint4 val = *reinterpret_cast<const uint4*>(stage + rr * 128 + ((ch ^ (rr & 7)) << 4));
-            if (ir < nb)
-              *reinterpret_cast<uint4*>(g16 + (bh_rows + ir) * kHeadDim * kHeadDim + n + ch * 8) = val;
+            if (ir < row_limit)
+              *reinterpret_cast<uint4*>(g16 + static_cast<size_t>(ir) * kHeadDim * kHeadDim + n + ch * 8) = val;
           }
           __syncwarp();
         } else {
@@ -203,7 +228,7 @@ aggregate_mma_kernel(const __grid_constant__ CUtensorMap map_s, const signed cha
             tmem_ld32(lane_addr + pp * 64 + half * 32, v);
             tmem_wait_ld();
             if (!row_ok) continue;
-            float4* dst = reinterpret_cast<float4*>(zeta + out_row * kHeadDim + (n - kHeadDim * kHeadDim) + half * 32);
+            float4* dst = reinterpret_cast<float4*>(zeta + static_cast<size_t>(row) * kHeadDim + (n - kHeadDim * kHeadDim) + half * 32);
 #pragma unroll
             for (int q = 0; q < 8; ++q)
               dst[q] = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
@@ -234,8 +259,33 @@ lite3r_status launch_aggregate(const __nv_bfloat16* hws, const signed char* cls,
   st = record_cuda(cudaFuncSetAttribute(aggregate_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         static_cast<int>(kSmemBytes)));
   if (st != LITE3R_OK) return st;
-  const dim3 grid(ceil_div(kSummaryRow, kTileN), ceil_div(nb, kTileM), s.batch * s.heads);
-  aggregate_mma_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_s, cls, nb, g16, zeta, device_status);
+  if (rows > 0x7FFFFFFFull - kTileM) return LITE3R_ERR_UNSUPPORTED;
+  const int total_rows = static_cast<int>(rows), bh = s.batch * s.heads;
+  // Tiles through the (b, h) boundaries pay with a longer reduction (the keys of every (b, h) a tile touches), tiles
+  // inside one (b, h) with padding when Nb is not a multiple of 128.  Estimate of either: waves of CTAs (two per SM)
+  // times the cost of a CTA, its set-up and drain counted as three 64-key chunks (at Nb = 172 the two tilings are
+  // measured on a par at about that ratio).
+  int sms = 0;
+  if ((st = sm_count(&sms)) != LITE3R_OK) return st;
+  constexpr double kFixed = 3.0;
+  const long long slots = 2ll * sms, col_tiles = ceil_div(kSummaryRow, kTileN);
+  const long long ctas_inside = col_tiles * bh * ceil_div(nb, kTileM);
+  const double time_inside = static_cast<double>((ctas_inside + slots - 1) / slots) * (kFixed + ceil_div(nb, kChunk));
+  const long long row_tiles = ceil_div(total_rows, kTileM);
+  // chunks of a flat tile: one (b, h) when it starts and ends in the same one, else every (b, h) it touches
+  double flat_chunks = 0.0;
+  const long long probe = std::min<long long>(row_tiles, 4096);  // the pattern repeats; a prefix is representative
+  for (long long t = 0; t < probe; ++t) {
+    const int r0 = static_cast<int>(t) * kTileM;
+    const int k0 = r0 / nb * nb, k1 = (std::min(r0 + kTileM, total_rows) - 1) / nb * nb + nb;
+    flat_chunks += ceil_div(k1 - k0, kChunk);
+  }
+  flat_chunks /= static_cast<double>(probe);
+  const long long ctas_flat = col_tiles * row_tiles;
+  const double time_flat = static_cast<double>((ctas_flat + slots - 1) / slots) * (kFixed + flat_chunks);
+  const int flat = time_flat < time_inside ? 1 : 0;
+  const dim3 grid(ceil_div(kSummaryRow, kTileN), flat ? ceil_div(total_rows, kTileM) : ceil_div(nb, kTileM), flat ? 1 : bh);
+  aggregate_mma_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_s, cls, nb, total_rows, flat, g16, zeta, device_status);
   return after_launch();
 }
 
