@@ -73,6 +73,9 @@ typedef struct {
 
 /* The block plan (all DEVICE pointers, caller-allocated):
  *   cls       int8  [B, H, Nb, Nb]    class of key block j for query block i: 0 negligible, 1 marginal, 2 critical
+ *                                     (a plan handed to lite3r_sla_forward must hold no other value: the forward reads
+ *                                     bit 0 as "marginal"; the array is read in aligned 32-bit words, so up to three
+ *                                     bytes next to either end of it are touched and must be addressable)
  *   crit_idx  int32 [B, H, Nb, k_crit] key-block indices of the critical blocks of row i, ascending
  *   marg_idx  int32 [B, H, Nb, k_marg] same for the marginal blocks; may be NULL (not written then)
  * k_crit / k_marg / k_neg are the per-row counts lite3r_plan_sizes reports. */
