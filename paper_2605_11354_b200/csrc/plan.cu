@@ -458,17 +458,19 @@ __global__ void __launch_bounds__(R * 32) plan_kernel(const int* __restrict__ q_
   for (int j0 = 0; j0 < nb; j0 += 32) {
     const int j = j0 + lane;
     const bool in = j < nb;
-    const unsigned long long key = in ? keys[j] : 0ull;
     const int bk = in ? bucket(j) : -2;
-    const unsigned long long kc = key & sc.mask, km = key & sm.mask;
-    const bool eq_c = bk == sc.bucket && kc == sc.prefix, eq_m = bk == sm.bucket && km == sm.prefix;
-    const unsigned b_eq_c = __ballot_sync(0xFFFFFFFFu, eq_c), b_eq_m = __ballot_sync(0xFFFFFFFFu, eq_m);
-    const bool sel_c = in && (bk > sc.bucket || (bk == sc.bucket && kc > sc.prefix) ||
-                              (eq_c && tie_c + __popc(b_eq_c & below) < sc.take));
-    const bool sel_m = in && (bk > sm.bucket || (bk == sm.bucket && km > sm.prefix) ||
-                              (eq_m && tie_m + __popc(b_eq_m & below) < sm.take));
-    tie_c += __popc(b_eq_c);
-    tie_m += __popc(b_eq_m);
+    bool sel_c = in && bk > sc.bucket, sel_m = in && bk > sm.bucket;
+    // the 64-bit keys only matter for entries inside one of the two threshold buckets: most groups of 32 have none
+    if (__any_sync(0xFFFFFFFFu, bk == sc.bucket || bk == sm.bucket)) {
+      const unsigned long long key = in ? keys[j] : 0ull;
+      const unsigned long long kc = key & sc.mask, km = key & sm.mask;
+      const bool eq_c = bk == sc.bucket && kc == sc.prefix, eq_m = bk == sm.bucket && km == sm.prefix;
+      const unsigned b_eq_c = __ballot_sync(0xFFFFFFFFu, eq_c), b_eq_m = __ballot_sync(0xFFFFFFFFu, eq_m);
+      sel_c = sel_c || (bk == sc.bucket && kc > sc.prefix) || (eq_c && tie_c + __popc(b_eq_c & below) < sc.take);
+      sel_m = sel_m || (bk == sm.bucket && km > sm.prefix) || (eq_m && tie_m + __popc(b_eq_m & below) < sm.take);
+      tie_c += __popc(b_eq_c);
+      tie_m += __popc(b_eq_m);
+    }
     const int c = !in ? -1 : (sel_c ? 2 : (sel_m ? 1 : 0));
     if (in) out_cls[j] = static_cast<signed char>(c);
     const unsigned m_crit = __ballot_sync(0xFFFFFFFFu, c == 2);
