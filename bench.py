@@ -34,11 +34,11 @@ FP8_OVER_BF16 = 2.0  # nominal dense ratio (4.5 vs 2.25 PFLOP/s)
 # DRAM bytes (read + write) of one launch, keyed by (workload, kernel), from the ncu captures summarised under
 # profiles/; a kernel that changed since its capture has no entry.
 DRAM_BYTES_PER_LAUNCH = {
-    ("vggt8", "attention"): 82876928,
-    ("vggt8", "plan"): 1488384,
-    ("vggt8", "quantize_qkv"): 72570112,
-    ("vggt8", "summary"): 23942144,
-    ("vggt8", "aggregation"): 23397888,
+    ("vggt8", "attention"): 85612288,
+    ("vggt8", "plan"): 1488128,
+    ("vggt8", "quantize_qkv"): 72935680,
+    ("vggt8", "summary"): 23836928,
+    ("vggt8", "aggregation"): 23399168,
 }
 
 
