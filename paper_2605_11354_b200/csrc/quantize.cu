@@ -172,8 +172,8 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const __grid_constan
     // x / scale must be the IEEE quotient, but only its e4m3 rounding is kept.  The quotient lies strictly between
     // x * r_lo and x * r_hi with r = 1 / scale widened by 2^-20 either way (the reciprocal, the product and the
     // quotient itself are each rounded by at most 2^-24), and rounding to e4m3 is monotone: when both products give
-    // the same code, that is the code of the quotient.  Otherwise (a few elements per 10^5, next to a rounding
-    // boundary of the e4m3 grid) the group of eight is redone with the division.
+    // the same code, that is the code of the quotient.  Otherwise (next to, or exactly on, a rounding boundary of the
+    // e4m3 grid) the pair is redone with the division.
     const float r = __frcp_rn(scale);
     const float r_lo = r * (1.0f - 0x1p-20f), r_hi = r * (1.0f + 0x1p-20f);
 
@@ -188,7 +188,6 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const __grid_constan
       float* const vp = v[kKeep ? p : 0];
       if (!kKeep) unpack8(reinterpret_cast<const SrcT*>(mine + p * kThreads * kSegBytes), vp);
       uint32_t two[4];
-      bool same = true;
 #pragma unroll
       for (int c = 0; c < 8; c += 2) {
         // the saturating conversion clamps to +-448 exactly like clamp-then-cast
@@ -199,19 +198,19 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const __grid_constan
         unpack_f32x2(fma_f32x2(x2, r_hi2, neg0), y_hi.x, y_hi.y);
         const uint32_t lo = __nv_cvt_float2_to_fp8x2(y_lo, __NV_SATFINITE, __NV_E4M3);
         two[c >> 1] = __nv_cvt_float2_to_fp8x2(y_hi, __NV_SATFINITE, __NV_E4M3);
-        same &= lo == two[c >> 1];
-      }
-      if (!same) {
-#pragma unroll
-        for (int c = 0; c < 8; c += 2)
+        // bf16 sources put about one quotient in a thousand exactly on a rounding boundary of the e4m3 grid, so some
+        // lane of a warp gets here every few passes: only the pair in question is redone with the division
+        if (lo != two[c >> 1])
           two[c >> 1] = __nv_cvt_float2_to_fp8x2(make_float2(__fdiv_rn(vp[c], scale), __fdiv_rn(vp[c + 1], scale)),
                                                  __NV_SATFINITE, __NV_E4M3);
       }
+      if (colsum != nullptr) {
 #pragma unroll
-      for (int c = 0; c < 8; c += 2) {
-        const __half2_raw back = __nv_cvt_fp8x2_to_halfraw2(static_cast<__nv_fp8x2_storage_t>(two[c >> 1]), __NV_E4M3);
-        const float2 f = __half22float2(__half2(back));
-        sums2[c >> 1] = add_f32x2(sums2[c >> 1], pack_f32x2(f.x, f.y));
+        for (int c = 0; c < 8; c += 2) {
+          const __half2_raw back = __nv_cvt_fp8x2_to_halfraw2(static_cast<__nv_fp8x2_storage_t>(two[c >> 1]), __NV_E4M3);
+          const float2 f = __half22float2(__half2(back));
+          sums2[c >> 1] = add_f32x2(sums2[c >> 1], pack_f32x2(f.x, f.y));
+        }
       }
       *reinterpret_cast<uint2*>(dst + static_cast<size_t>(row) * kHeadDim) =
           make_uint2(two[0] | (two[1] << 16), two[2] | (two[3] << 16));
