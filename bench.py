@@ -36,7 +36,7 @@ FP8_OVER_BF16 = 2.0  # nominal dense ratio (4.5 vs 2.25 PFLOP/s)
 DRAM_BYTES_PER_LAUNCH = {
     ("vggt8", "attention"): 85612288,
     ("vggt8", "plan"): 1488128,
-    ("vggt8", "quantize_qkv"): 72935680,
+    ("vggt8", "quantize_qkv"): 73029632,
     ("vggt8", "summary"): 23836928,
     ("vggt8", "aggregation"): 23399168,
 }
