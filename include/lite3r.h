@@ -142,6 +142,25 @@ LITE3R_API lite3r_status lite3r_sla_forward(const lite3r_fp8* q, const lite3r_fp
                                  long long out_stride_h, long long out_stride_n, void* workspace,
                                  size_t workspace_bytes, int* device_status, void* stream);
 
+/* lite3r_sla_forward in two halves, for callers that overlap the block plan with the part of the forward that does
+ * not depend on it.  The per-key-block summaries of the linear branch (Algorithm 1's feature map, KV summary and
+ * normaliser, with proj folded in) and the fp16 copy of V read only K, V and proj, so
+ *     lite3r_sla_forward_begin  (stream A)  may run beside  lite3r_sla_plan  (stream B),
+ * and lite3r_sla_forward_finish (aggregation over the marginal blocks, attention, linear output, sum) follows once
+ * both have completed (the caller orders the streams).  begin followed by finish on one stream is exactly
+ * lite3r_sla_forward: same kernels, same results.  begin takes the three class counts lite3r_plan_sizes reports
+ * (they depend on the fractions only) and clears *device_status; finish does not clear it.  Both use the same
+ * workspace, which must not be touched in between.  Arguments otherwise as for lite3r_sla_forward. */
+LITE3R_API lite3r_status lite3r_sla_forward_begin(const lite3r_fp8* k, const lite3r_fp8* v, const float* proj,
+                                       long long proj_head_stride, const lite3r_shape* shape, lite3r_phi phi,
+                                       int k_crit, int k_marg, int k_neg, void* workspace, size_t workspace_bytes,
+                                       int* device_status, void* stream);
+LITE3R_API lite3r_status lite3r_sla_forward_finish(const lite3r_fp8* q, const lite3r_fp8* k, const lite3r_fp8* v,
+                                        const lite3r_shape* shape, lite3r_phi phi, const lite3r_plan* plan,
+                                        float* out, long long out_stride_b, long long out_stride_h,
+                                        long long out_stride_n, void* workspace, size_t workspace_bytes,
+                                        int* device_status, void* stream);
+
 /* The same forward for callers that cannot provide scratch memory.  (The paper has no counterpart: this entry
  * point exists for deployments, not for the method.)
  *

@@ -45,7 +45,8 @@ class Plan(C.Structure):
 EXPORTS = ("lite3r_fp8_sizes", "lite3r_plan_sizes", "lite3r_forward_workspace", "lite3r_quantize_fp8",
            "lite3r_sla_plan", "lite3r_sla_forward", "lite3r_status_string", "lite3r_last_cuda_error",
            "lite3r_launch_count", "lite3r_profile_enable", "lite3r_profile_stage_ms",
-           "lite3r_sla_forward_static_scratch", "lite3r_quantize_fp8_qkv", "lite3r_selftest_wait_expiry")
+           "lite3r_sla_forward_static_scratch", "lite3r_quantize_fp8_qkv", "lite3r_selftest_wait_expiry",
+           "lite3r_sla_forward_begin", "lite3r_sla_forward_finish")
 STATIC_SCRATCH_BYTES = 32 << 20  # LITE3R_STATIC_SCRATCH_BYTES
 
 
@@ -76,6 +77,14 @@ def lib() -> C.CDLL:
                                                     C.c_void_p, C.c_longlong, C.c_longlong, C.c_longlong, C.c_void_p,
                                                     C.c_void_p]
     L.lite3r_sla_forward_static_scratch.restype = C.c_int
+    L.lite3r_sla_forward_begin.argtypes = [C.POINTER(Fp8), C.POINTER(Fp8), C.c_void_p, C.c_longlong, C.POINTER(Shape),
+                                           C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_size_t, C.c_void_p,
+                                           C.c_void_p]
+    L.lite3r_sla_forward_begin.restype = C.c_int
+    L.lite3r_sla_forward_finish.argtypes = [C.POINTER(Fp8), C.POINTER(Fp8), C.POINTER(Fp8), C.POINTER(Shape), C.c_int,
+                                            C.POINTER(Plan), C.c_void_p, C.c_longlong, C.c_longlong, C.c_longlong,
+                                            C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+    L.lite3r_sla_forward_finish.restype = C.c_int
     L.lite3r_selftest_wait_expiry.argtypes = [C.c_void_p, C.c_ulonglong, C.c_void_p]
     L.lite3r_selftest_wait_expiry.restype = C.c_int
     L.lite3r_status_string.argtypes = [C.c_int]
@@ -248,6 +257,34 @@ def lite3r_sla_forward(q: Fp8Tensor, k: Fp8Tensor, v: Fp8Tensor, proj: torch.Ten
                                     _stream_ptr(stream)), "lite3r_sla_forward")
 
 
+def lite3r_sla_forward_begin(k: Fp8Tensor, v: Fp8Tensor, proj: torch.Tensor, shape: Shape, phi: int,
+                             plan: PlanBuffers, workspace: torch.Tensor, device_status=None, stream=None) -> None:
+    """First half of the forward (summaries, fp16 V): needs only the plan's class counts, not its contents."""
+    if proj.dtype != torch.float32 or not proj.is_cuda or not proj.is_contiguous():
+        raise Lite3rError("lite3r_sla_forward_begin: proj must be a contiguous CUDA float32 tensor")
+    head_stride = proj.stride(0) if proj.dim() == 3 else 0
+    ks, vs = k.c_struct(), v.c_struct()
+    _check(lib().lite3r_sla_forward_begin(C.byref(ks), C.byref(vs), proj.data_ptr(), head_stride, C.byref(shape), phi,
+                                          plan.k_crit, plan.k_marg, plan.k_neg, workspace.data_ptr(),
+                                          workspace.numel() * workspace.element_size(),
+                                          device_status.data_ptr() if device_status is not None else None,
+                                          _stream_ptr(stream)), "lite3r_sla_forward_begin")
+
+
+def lite3r_sla_forward_finish(q: Fp8Tensor, k: Fp8Tensor, v: Fp8Tensor, shape: Shape, phi: int, plan: PlanBuffers,
+                              out: torch.Tensor, workspace: torch.Tensor, device_status=None, stream=None) -> None:
+    """Second half of the forward (aggregation, attention, linear output, sum); after begin and the plan."""
+    if out.dtype != torch.float32 or not out.is_cuda or out.stride(3) != 1:
+        raise Lite3rError("lite3r_sla_forward_finish: out must be a CUDA float32 tensor [B,H,N,D] with contiguous D")
+    p = plan.c_struct()
+    qs, ks, vs = q.c_struct(), k.c_struct(), v.c_struct()
+    _check(lib().lite3r_sla_forward_finish(C.byref(qs), C.byref(ks), C.byref(vs), C.byref(shape), phi, C.byref(p),
+                                           out.data_ptr(), out.stride(0), out.stride(1), out.stride(2),
+                                           workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                           device_status.data_ptr() if device_status is not None else None,
+                                           _stream_ptr(stream)), "lite3r_sla_forward_finish")
+
+
 def lite3r_sla_forward_static_scratch(q: Fp8Tensor, k: Fp8Tensor, v: Fp8Tensor, proj: torch.Tensor, shape: Shape,
                                       phi: int, plan: PlanBuffers, out: torch.Tensor, device_status=None,
                                       stream=None) -> None:
@@ -285,6 +322,7 @@ class SlaForward:
         self.workspace = self.workspace[off:off + nbytes]
         self.out = torch.empty((batch, heads, tokens, head_dim), dtype=torch.float32, device=self.device)
         self.status = torch.zeros(1, dtype=torch.int32, device=self.device)
+        self._side = None  # stream of the overlapped first half of the forward, made on first use
 
     def quantize(self, q, k, v, stream=None):
         if q.dtype == k.dtype == v.dtype:
@@ -304,7 +342,23 @@ class SlaForward:
                            self.workspace, self.status, stream)
         return out
 
-    def run(self, q, k, v, proj, stream=None, out=None):
-        self.quantize(q, k, v, stream)
-        self.make_plan(stream)
-        return self.forward(proj, stream, out)
+    def run(self, q, k, v, proj, stream=None, out=None, overlap=False):
+        """Quantise, plan, forward.  overlap=True runs the plan-independent first half of the forward (summaries, fp16
+        V) on a side stream beside the plan kernel; the results are the same."""
+        if not overlap or self.plan.k_marg == 0:
+            self.quantize(q, k, v, stream)
+            self.make_plan(stream)
+            return self.forward(proj, stream, out)
+        main = torch.cuda.current_stream(self.device) if stream is None else stream
+        if self._side is None:
+            self._side = torch.cuda.Stream(self.device)
+        out = self.out if out is None else out
+        self.quantize(q, k, v, main)
+        self._side.wait_stream(main)  # codes and scales are ready
+        lite3r_sla_forward_begin(self.k8, self.v8, proj, self.shape, self.phi, self.plan, self.workspace, self.status,
+                                 self._side)
+        self.make_plan(main)
+        main.wait_stream(self._side)
+        lite3r_sla_forward_finish(self.q8, self.k8, self.v8, self.shape, self.phi, self.plan, out, self.workspace,
+                                  self.status, main)
+        return out

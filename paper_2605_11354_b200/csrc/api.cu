@@ -207,31 +207,37 @@ lite3r_status lite3r_sla_plan(const lite3r_fp8* q, const lite3r_fp8* k, const li
   return launch_plan(*q, *k, *shape, c, *plan, static_cast<cudaStream_t>(stream));
 }
 
-lite3r_status lite3r_sla_forward(const lite3r_fp8* q, const lite3r_fp8* k, const lite3r_fp8* v, const float* proj,
-                                 long long proj_head_stride, const lite3r_shape* shape, lite3r_phi phi,
-                                 const lite3r_plan* plan, float* out, long long out_stride_b,
-                                 long long out_stride_h, long long out_stride_n, void* workspace,
-                                 size_t workspace_bytes, int* device_status, void* stream) {
+// Shared argument checks and launch of lite3r_sla_forward and its two halves (phases as in launch_forward).
+static lite3r_status forward_phases(int phases, const lite3r_fp8* q, const lite3r_fp8* k, const lite3r_fp8* v,
+                                    const float* proj, long long proj_head_stride, const lite3r_shape* shape,
+                                    lite3r_phi phi, const lite3r_plan* plan, float* out, long long out_stride_b,
+                                    long long out_stride_h, long long out_stride_n, void* workspace,
+                                    size_t workspace_bytes, int* device_status, void* stream) {
   lite3r_status st = check_shape(shape);
   if (st != LITE3R_OK) return st;
-  if ((st = check_fp8(q, true, false)) != LITE3R_OK) return st;
   if ((st = check_fp8(k, true, false)) != LITE3R_OK) return st;
   if ((st = check_fp8(v, true, false)) != LITE3R_OK) return st;
   if (phi != LITE3R_PHI_SOFTMAX && phi != LITE3R_PHI_ELU1) return LITE3R_ERR_UNSUPPORTED;
-  if (proj == nullptr || !aligned(proj, 16) || proj_head_stride < 0 || (proj_head_stride % 4)) return LITE3R_ERR_INVALID_ARG;
-  if (out == nullptr || !aligned(out, 16)) return LITE3R_ERR_INVALID_ARG;
-  if (out_stride_n < kHeadDim || out_stride_b < 0 || out_stride_h < 0) return LITE3R_ERR_INVALID_ARG;
-  if ((out_stride_b % 4) || (out_stride_h % 4) || (out_stride_n % 4)) return LITE3R_ERR_INVALID_ARG;
-  if (plan == nullptr || plan->cls == nullptr) return LITE3R_ERR_INVALID_ARG;
+  if (plan == nullptr) return LITE3R_ERR_INVALID_ARG;
   const int nb = ceil_div(shape->tokens, shape->block);
   if (plan->k_crit < 0 || plan->k_marg < 0 || plan->k_neg < 0 || plan->k_crit + plan->k_marg + plan->k_neg != nb)
     return LITE3R_ERR_INVALID_ARG;
-  if (plan->k_crit > 0 && plan->crit_idx == nullptr) return LITE3R_ERR_INVALID_ARG;
+  if (phases & 1) {
+    if (proj == nullptr || !aligned(proj, 16) || proj_head_stride < 0 || (proj_head_stride % 4)) return LITE3R_ERR_INVALID_ARG;
+  }
+  if (phases & 2) {
+    if ((st = check_fp8(q, true, false)) != LITE3R_OK) return st;
+    if (out == nullptr || !aligned(out, 16)) return LITE3R_ERR_INVALID_ARG;
+    if (out_stride_n < kHeadDim || out_stride_b < 0 || out_stride_h < 0) return LITE3R_ERR_INVALID_ARG;
+    if ((out_stride_b % 4) || (out_stride_h % 4) || (out_stride_n % 4)) return LITE3R_ERR_INVALID_ARG;
+    if (plan->cls == nullptr) return LITE3R_ERR_INVALID_ARG;
+    if (plan->k_crit > 0 && plan->crit_idx == nullptr) return LITE3R_ERR_INVALID_ARG;
+  }
   const Counts c{plan->k_crit, plan->k_marg, plan->k_neg};
   if (workspace == nullptr || !aligned(workspace, 256)) return LITE3R_ERR_INVALID_ARG;
   if (workspace_bytes < forward_workspace_bytes(*shape, c)) return LITE3R_ERR_WORKSPACE;
-  ForwardArgs a;
-  a.q = *q;
+  ForwardArgs a = {};
+  if (q != nullptr) a.q = *q;
   a.k = *k;
   a.v = *v;
   a.proj = proj;
@@ -246,7 +252,37 @@ lite3r_status lite3r_sla_forward(const lite3r_fp8* q, const lite3r_fp8* k, const
   a.workspace = workspace;
   a.workspace_bytes = workspace_bytes;
   a.device_status = device_status;
-  return launch_forward(a, static_cast<cudaStream_t>(stream));
+  return launch_forward(a, phases, static_cast<cudaStream_t>(stream));
+}
+
+lite3r_status lite3r_sla_forward(const lite3r_fp8* q, const lite3r_fp8* k, const lite3r_fp8* v, const float* proj,
+                                 long long proj_head_stride, const lite3r_shape* shape, lite3r_phi phi,
+                                 const lite3r_plan* plan, float* out, long long out_stride_b,
+                                 long long out_stride_h, long long out_stride_n, void* workspace,
+                                 size_t workspace_bytes, int* device_status, void* stream) {
+  return forward_phases(3, q, k, v, proj, proj_head_stride, shape, phi, plan, out, out_stride_b, out_stride_h,
+                        out_stride_n, workspace, workspace_bytes, device_status, stream);
+}
+
+lite3r_status lite3r_sla_forward_begin(const lite3r_fp8* k, const lite3r_fp8* v, const float* proj,
+                                       long long proj_head_stride, const lite3r_shape* shape, lite3r_phi phi,
+                                       int k_crit, int k_marg, int k_neg, void* workspace, size_t workspace_bytes,
+                                       int* device_status, void* stream) {
+  lite3r_plan counts = {};
+  counts.k_crit = k_crit;
+  counts.k_marg = k_marg;
+  counts.k_neg = k_neg;
+  return forward_phases(1, nullptr, k, v, proj, proj_head_stride, shape, phi, &counts, nullptr, 0, 0, 0, workspace,
+                        workspace_bytes, device_status, stream);
+}
+
+lite3r_status lite3r_sla_forward_finish(const lite3r_fp8* q, const lite3r_fp8* k, const lite3r_fp8* v,
+                                        const lite3r_shape* shape, lite3r_phi phi, const lite3r_plan* plan,
+                                        float* out, long long out_stride_b, long long out_stride_h,
+                                        long long out_stride_n, void* workspace, size_t workspace_bytes,
+                                        int* device_status, void* stream) {
+  return forward_phases(2, q, k, v, nullptr, 0, shape, phi, plan, out, out_stride_b, out_stride_h, out_stride_n,
+                        workspace, workspace_bytes, device_status, stream);
 }
 
 lite3r_status lite3r_selftest_wait_expiry(int* device_status, unsigned long long limit_ns, void* stream) {

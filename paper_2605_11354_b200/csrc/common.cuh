@@ -121,6 +121,7 @@ lite3r_status make_tensor_map_2d(CUtensorMap* map, CUtensorMapDataType type, int
 
 lite3r_status launch_wait_expiry_probe(int* status, unsigned long long limit_ns, cudaStream_t stream);
 size_t forward_workspace_bytes(const lite3r_shape& s, const Counts& c);
-lite3r_status launch_forward(const ForwardArgs& a, cudaStream_t stream);
+// phases: 1 = the plan-independent first part, 2 = the rest, 3 = the whole forward
+lite3r_status launch_forward(const ForwardArgs& a, int phases, cudaStream_t stream);
 
 }  // namespace lite3r

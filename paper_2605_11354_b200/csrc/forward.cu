@@ -81,18 +81,19 @@ Workspace carve(void* base, const lite3r_shape& s) {
   return w;
 }
 
+// phases: bit 0 = the part that does not depend on the plan's contents (summaries, fp16 V operand), bit 1 = the rest.
 template <int BS>
-lite3r_status run_forward(const ForwardArgs& a, cudaStream_t stream) {
+lite3r_status run_forward(const ForwardArgs& a, int phases, cudaStream_t stream) {
   const lite3r_shape& s = a.s;
   const int nb = ceil_div(s.tokens, BS);
   const int rows = s.batch * s.heads * nb;
   const Workspace w = carve(a.workspace, s);
-  lite3r_status st;
-  profile_mark(0, stream);
+  lite3r_status st = LITE3R_OK;
+  if (phases & 1) profile_mark(0, stream);
   // With a linear branch the summary kernel reads every V row anyway and writes the fp16 operand on the way; the
   // stand-alone pass runs only when there is no linear branch.
   const bool v16_from_summary = a.plan.k_marg > 0;
-  if (a.plan.k_crit > 0 && !v16_from_summary) {
+  if ((phases & 1) && a.plan.k_crit > 0 && !v16_from_summary) {
     const size_t words = static_cast<size_t>(rows) * BS * kHeadDim / 16;  // 16 codes per thread and pass
     int sms = 0;
     if ((st = sm_count(&sms)) != LITE3R_OK) return st;
@@ -101,12 +102,15 @@ lite3r_status run_forward(const ForwardArgs& a, cudaStream_t stream) {
     if ((st = after_launch()) != LITE3R_OK) return st;
     profile_mark(1, stream);
   }
-  if (a.plan.k_marg > 0) {
+  if ((phases & 1) && a.plan.k_marg > 0) {
     profile_mark(2, stream);
     st = launch_summary(a.k, a.v, a.proj, a.proj_head_stride, s, a.phi, w.hws, a.plan.k_crit > 0 ? w.v16 : nullptr,
                         a.device_status, stream);
     if (st != LITE3R_OK) return st;
     profile_mark(3, stream);
+  }
+  if (!(phases & 2)) return st;
+  if (a.plan.k_marg > 0) {
     profile_mark(4, stream);
     if ((st = launch_aggregate(w.hws, a.plan.cls, s, nb, w.g16, w.zeta, a.device_status, stream)) != LITE3R_OK) return st;
     profile_mark(5, stream);
@@ -150,12 +154,12 @@ size_t forward_workspace_bytes(const lite3r_shape& s, const Counts& c) {
   return carve(nullptr, s).bytes;
 }
 
-lite3r_status launch_forward(const ForwardArgs& a, cudaStream_t stream) {
-  if (a.device_status != nullptr) {
+lite3r_status launch_forward(const ForwardArgs& a, int phases, cudaStream_t stream) {
+  if ((phases & 1) && a.device_status != nullptr) {  // the status word is cleared where the forward begins
     lite3r_status st = record_cuda(cudaMemsetAsync(a.device_status, 0, sizeof(int), stream));
     if (st != LITE3R_OK) return st;
   }
-  return a.s.block == 64 ? run_forward<64>(a, stream) : run_forward<128>(a, stream);
+  return a.s.block == 64 ? run_forward<64>(a, phases, stream) : run_forward<128>(a, phases, stream);
 }
 
 }  // namespace lite3r

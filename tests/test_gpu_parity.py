@@ -237,6 +237,23 @@ def test_stress_dense_equivalent_point():
     full_parity(wl, inputs, heads=[4], crit=1.0, neg=0.0, query_blocks=qb)
 
 
+def test_overlapped_run_matches_the_in_order_run():
+    """lite3r_sla_forward_begin on a side stream beside the plan, then lite3r_sla_forward_finish: bit-identical to the
+    three calls in order, also when the two ways alternate on one engine."""
+    wl = small_workload("overlap", tokens=5 * 1374, heads=4, batch=2)
+    inputs = wk.make_inputs(wl)
+    eng, expected = pu.run_gpu(inputs, wl)
+    expected = expected.clone()
+    q, k, v = (pu.to_device(inputs[n], wl.src_dtype) for n in ("q", "k", "v"))
+    proj = torch.from_numpy(inputs["proj"]).cuda()
+    for overlap in (True, True, False, True):
+        eng.out.fill_(float("nan"))
+        out = eng.run(q, k, v, proj, overlap=overlap)
+        torch.cuda.synchronize()
+        assert int(eng.status.item()) == 0
+        assert torch.equal(out, expected), overlap
+
+
 def test_token_major_output_layout():
     """The output may be a [B, N, H, D] buffer viewed as [B, H, N, D]: only the strides change."""
     wl = small_workload("out-strides", tokens=450, batch=2, heads=3)
