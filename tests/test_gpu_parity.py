@@ -168,6 +168,24 @@ def test_ties_resolve_to_lower_index():
     assert np.array_equal(eng.plan.cls.cpu().numpy(), ref["cls"])
 
 
+@pytest.mark.parametrize("seed", [7, 23])
+def test_random_shapes_against_the_oracle(seed):
+    """Seeded sweep over shapes, block sizes, class mixes, feature maps, source types and input structure: every case
+    is checked like the fixed ones (codes, scales, column sums, plan, output)."""
+    rng = np.random.default_rng(seed)
+    for case in range(24):
+        wl = wk.Workload(f"sweep{seed}-{case}", cfg_id=200 + case, batch=int(rng.integers(1, 4)),
+                         heads=int(rng.integers(1, 4)), tokens=int(rng.integers(1, 2600)), head_dim=64,
+                         block=int(rng.choice([64, 128])), crit=float(rng.choice([0.0, 0.05, 0.1, 0.3, 0.6, 1.0])),
+                         neg=float(rng.choice([0.0, 0.2, 0.5, 0.9])), centres=int(rng.choice([0, 8, 32])), sigma=0.3,
+                         src_dtype=str(rng.choice(["bf16", "f32"])))
+        phi = str(rng.choice(["softmax", "elu1"]))
+        blocks = None
+        if wl.n_blocks * wl.batch * wl.heads > 40:
+            blocks = pu.sample_blocks(wl, list(range(wl.heads)), 24, seed=case)
+        full_parity(wl, wk.make_inputs(wl), phi=phi, query_blocks=blocks)
+
+
 def test_all_scores_tied_in_a_long_row():
     """Zero queries make every pooled score of a row equal (one bucket holding all 150 blocks, more than the
     candidate list keeps): the selection must fall back to index order, exactly as the oracle ranks them."""
