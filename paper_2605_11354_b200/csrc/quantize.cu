@@ -21,10 +21,7 @@ using sm100::fma_f32x2;
 using sm100::pack_f32x2;
 using sm100::unpack_f32x2;
 
-#ifndef LITE3R_QUANT_THREADS_SMALL
-#define LITE3R_QUANT_THREADS_SMALL 64
-#endif
-constexpr int kQuantThreadsSmall = LITE3R_QUANT_THREADS_SMALL;  // CTA size for 8 KB tiles
+constexpr int kQuantThreadsSmall = 64;  // CTA size for 8 KB tiles
 
 // Threads per CTA (= per tile).  The per-tile work that does not shrink with the tile (address arithmetic, the two
 // reductions, barriers) is paid per thread, so few threads with many values each keep the instruction count per

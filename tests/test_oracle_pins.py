@@ -364,3 +364,66 @@ def test_subset_of_query_blocks_and_external_plan():
     assert np.array_equal(part["out"][0, 1, 96:], full["out"][0, 1, 96:])
     assert np.array_equal(part["out"][0, 0, :16], full["out"][0, 0, :16])
     assert np.isnan(part["out"][0, 0, 16:]).all()
+
+
+# ------------------------------------------------------------------ the composed path used by every GPU parity test
+def torch_quantize(x, block):
+    """Independent quantiser: scalar fp32 scale per tile, torch's float8_e4m3fn cast, decode through torch's view."""
+    B, H, N, D = x.shape
+    nb = -(-N // block)
+    codes = np.zeros((B, H, nb * block, D), dtype=np.uint8)
+    scales = np.zeros((B, H, nb), dtype=np.float32)
+    xhat = np.zeros((B, H, N, D))
+    for b in range(B):
+        for h in range(H):
+            for i in range(nb):
+                sl = slice(i * block, min(N, (i + 1) * block))
+                tile = x[b, h, sl]
+                s = np.float32(np.float32(np.float32(np.abs(tile).max()) + np.float32(1e-8)) / np.float32(448.0))
+                f8 = torch.from_numpy((tile / s).astype(np.float32)).clamp(-448, 448).to(torch.float8_e4m3fn)
+                codes[b, h, sl] = f8.view(torch.uint8).numpy()
+                scales[b, h, i] = s
+                xhat[b, h, sl] = f8.to(torch.float64).numpy() * float(s)
+    return codes, scales, xhat
+
+
+@pytest.mark.parametrize("phi", ["softmax", "elu1"])
+def test_from_source_composition_against_independent_pieces(phi):
+    """sla_forward_from_source (the function the GPU parity tests take their expected values from) against pieces that
+    do not come from the oracle: torch's cast for the codes, the scalar brute force (which pools, ranks and sums on
+    its own) for the output.  K and V have visibly different magnitudes and crit != neg, so swapped operands,
+    swapped fractions or a wrong block size cannot pass."""
+    block, crit, neg = 16, 0.3, 0.15
+    q, k, v, w = small_problem(21, H=2, N=100, D=4, block=block, scale=1.5)
+    k = (k * np.float32(3.0)).astype(np.float32)
+    v = (v * np.float32(0.2) + np.float32(0.7)).astype(np.float32)
+    res = orc.sla_forward_from_source(q, k, v, w, block, crit, neg, phi=phi)
+    indep = {n: torch_quantize(x, block) for n, x in (("q", q), ("k", k), ("v", v))}
+    for n in ("q", "k", "v"):
+        codes, scales, xhat = indep[n]
+        assert np.array_equal(res[n + "_codes"], codes)
+        assert np.array_equal(res[n + "_scales"], scales)
+        assert np.array_equal(res[n + "hat"], xhat)
+    # the three quantised tensors are different things
+    assert not np.array_equal(res["k_scales"], res["v_scales"]) and not np.array_equal(res["q_scales"], res["k_scales"])
+    qh, kh, vh = indep["q"][2], indep["k"][2], indep["v"][2]
+    nb = -(-100 // block)
+    # scores: explicit block means of the valid tokens
+    for (h, i, j) in ((0, 0, 0), (1, 6, 2), (0, 3, 6), (1, 6, 6)):
+        mq = qh[0, h, i * block:min(100, (i + 1) * block)].mean(axis=0)
+        mk = kh[0, h, j * block:min(100, (j + 1) * block)].mean(axis=0)
+        assert np.isclose(res["scores"][0, h, i, j], float(mq @ mk) / 2.0, rtol=1e-12)
+    assert not np.allclose(res["scores"], np.swapaxes(res["scores"], -1, -2))
+    # classes: the counts of these fractions, critical = the largest scores
+    k_c, k_m, k_n = orc.class_counts(nb, crit, neg)
+    assert (k_c, k_m, k_n) == (2, 4, 1)
+    for h in range(2):
+        for i in range(nb):
+            order = sorted(range(nb), key=lambda j: (-res["scores"][0, h, i, j], j))
+            assert set(np.flatnonzero(res["cls"][0, h, i] == 2)) == set(order[:k_c])
+            assert set(np.flatnonzero(res["cls"][0, h, i] == 0)) == set(order[nb - k_n:])
+    ref = brute_force(qh, kh, vh, w.astype(np.float64), block, crit, neg, phi)
+    assert np.allclose(res["out"], ref, rtol=1e-10, atol=1e-12)
+    # and the brute force with the fractions swapped is a different answer (the test would notice the swap)
+    swapped = brute_force(qh, kh, vh, w.astype(np.float64), block, neg, crit, phi)
+    assert not np.allclose(res["out"], swapped, rtol=1e-3, atol=1e-3)
