@@ -42,7 +42,7 @@ typedef enum {
   LITE3R_ERR_TIMEOUT = 5      /* a bounded device-side wait expired (reported through device_status) */
 } lite3r_status;
 
-typedef enum { LITE3R_F32 = 0, LITE3R_BF16 = 1 } lite3r_dtype;
+typedef enum { LITE3R_F32 = 0, LITE3R_BF16 = 1, LITE3R_F16 = 2 } lite3r_dtype;
 
 /* Feature map of the linear branch.  SOFTMAX: softmax over the head_dim components (the benchmark
  * contract).  ELU1: ELU(x)+1 (the feature map Algorithm 1 prints). */

@@ -246,6 +246,7 @@ static lite3r_status forward_phases(int phases, const lite3r_fp8* q, const lite3
   a.phi = static_cast<int>(phi);
   a.plan = *plan;
   a.out = out;
+  a.out_dtype = LITE3R_F32;
   a.out_stride_b = out_stride_b;
   a.out_stride_h = out_stride_h;
   a.out_stride_n = out_stride_n;

@@ -1,29 +1,32 @@
-// K4: critical-block softmax attention + linear branch + add (Algorithm 1's sparse branch, linear output, projection and sum) on tcgen05 / TMEM / TMA.
+// K4: critical-block softmax attention + linear branch + add (Algorithm 1's sparse branch, linear output, projection
+// and sum) on tcgen05 / TMEM / TMA.
 //
-// One CTA owns 128 query rows of one (b, h): at block 64 a PAIR of query blocks (two M=64 accumulators interleaved
-// in the two 16-lane halves of every TMEM sub-partition), at block 128 one query block (M=128).  Work advances in
-// steps of 64 keys.  The steps are dealt alternately to two independent "sets" (even steps -> set 0, odd steps ->
-// set 1).  A set is 128 softmax threads (one query row each, TMEM lane = thread) plus one MMA-issuing thread, with
-// its own score buffer S, probability buffer P, output accumulator O and online-softmax state (reference maximum and
-// row sum); the two partial results are merged exactly at the end, O = (w0 O0 + w1 O1) / (w0 l0 + w1 l1) with
-// w = 2^(m_set - m).  Because the sets never wait for each other, an SM (two CTAs) always has four softmax streams
-// in different phases, which keeps the exponential unit busy while other streams wait on barriers, TMEM loads or
-// shared-memory stores.  Per step t of set b = t & 1:
-//   TMA      K tile(s) (e4m3, 64-byte rows, 64B swizzle) and V tile(s) (dequantised fp16, 128B swizzle) -> smem ring
-//   tcgen05  S_b = Q K^T           kind::f8f6f4, fp32 accumulators in TMEM (64 columns)
-//   softmax  pass 1: row maximum of the 64 scores, lazy-rescale decision; pass 2: exp2 and row sum, 32 columns at a
-//            time; P goes to shared memory as fp16 in the MMA's K-major 128B-swizzled layout
-//   tcgen05  O_b += P V            kind::f16, V as MN-major B operand, fp32 accumulators in TMEM (64 columns)
+// One CTA owns 128 query rows of one (b, h): at block 64 a PAIR of query blocks (two M=64 problems interleaved in the
+// two 16-lane halves of every TMEM sub-partition, each with its own list of critical key blocks), at block 128 one
+// query block (M=128).  Work advances in steps of 64 keys.  Per step t (w = t & 1):
+//   TMA      K tile(s) (e4m3, 64-byte rows, 64B swizzle) and V tile(s) (dequantised fp16, 128B swizzle) -> rings of four
+//   tcgen05  S[w] = Q K^T          kind::f8f6f4, fp32 accumulators in TMEM (64 columns, two buffers)
+//   softmax  warpgroup w, one thread per query row (TMEM lane = thread): the 64 scores are read once into registers,
+//            row maximum, lazy rescale, exp2, row sum; the probabilities go back to TMEM as packed fp16 (P[w], 32 columns)
+//   tcgen05  O += P[w] V           kind::f16 with the A operand read from TMEM, V as MN-major B operand from shared
+//                                  memory, ONE fp32 accumulator in TMEM (64 columns) for all steps
+// The two softmax warpgroups take the even and the odd steps.  Each owns a score buffer and a probability buffer, so
+// Q K^T of step t+2 is issued as soon as warpgroup w has read S[w], and P V of step t runs under the exponentials of
+// the following steps: the softmax threads do not wait for a product in the steady state, and with two CTAs per SM every
+// SM sub-partition holds four softmax warps in different phases, which is what keeps the exponential unit fed.
+// Both warpgroups accumulate into the same O, so they share one reference maximum per row: the thread that handles
+// step t reads the reference left by step t-1 from a shared-memory slot (written early in that step, right after its
+// row maximum is known), applies the lazy-rescale rule and publishes the reference of step t.  Row sums are kept
+// per warpgroup, brought to the final reference and added in the epilogue.
 // P is carried in fp16 (not e4m3): one e4m3 term has a 2.6 % rounding error per probability, which alone is ten
 // times the output tolerance.  V travels as the dequantised value in fp16 (2^-12 relative rounding).
 // Tail: phi(Q) (bf16) times the aggregated, projected summaries G_i (bf16) as one more MMA, divided by
-// phi(Q) . zeta_i, added to the merged softmax output and stored (each set stores 32 of the 64 output columns).
+// phi(Q) . zeta_i, added to the normalised softmax output and stored (each warpgroup handles 32 of the 64 columns).
 //
-// Warp roles (352 threads): warp 0 = TMA producer; warps 1 and 2 = MMA issuers of set 0 and set 1 (a single thread
-// can issue a small tcgen05.mma only every ~50 clocks, so each set has its own); warps 3-6 = softmax set 0,
-// warps 7-10 = softmax set 1.  "Product of step t done" is one barrier per product (rings of six) on which the
-// softmax threads and the TMA producer wait.
-// Every mbarrier wait is bounded (1 s); on expiry the CTA sets *device_status and all roles leave their loops.
+// Warp roles (384 threads): warp 0 = TMA producer, warp 1 = Q K^T issuer, warp 2 = P V issuer (one thread each; all
+// their waits block on mbarriers, nothing polls), warp 3 idle, warps 4-7 / 8-11 = softmax warpgroups 0 / 1.  The
+// control warps give registers back (setmaxnreg) so that a softmax thread can hold a whole row of scores.
+// Every wait is bounded (1 s); on expiry the CTA sets *device_status and all roles leave their loops.
 #include "common.cuh"
 #include "sm100.cuh"
 
@@ -33,50 +36,57 @@ namespace {
 
 using namespace sm100;
 
-constexpr int kStages = 3;
-constexpr int kSetThreads = 128;
+constexpr int kStages = 4;  // K and V rings
+constexpr int kSetThreads = 128;                 // one softmax warpgroup
 constexpr int kSoftmaxThreads = 2 * kSetThreads;
-constexpr int kCtrlWarps = 3;
+constexpr int kCtrlWarps = 4;
 constexpr int kThreads = kCtrlWarps * 32 + kSoftmaxThreads;
-constexpr uint32_t kBackoffNs = 100;  // sleep between polls of the single-thread roles
-constexpr int kRing = 6;              // lcm of the two sets and the three K/V stages
+constexpr int kCtrlRegs = 32, kSoftmaxRegs = 104;  // 128 * 32 + 256 * 104 = 384 * 80, the launch allocation
+constexpr uint32_t kBackoffNs = 64;  // sleep between polls of the single-thread roles
 constexpr int kStepKeys = 64;
 constexpr uint32_t kTmemCols = 256;
-constexpr uint32_t kColS = 0, kColO = 128, kColL = 0;  // S_b at 64 b, O_b at 128 + 64 b; the linear branch reuses S_0
+// TMEM columns: S buffers at 0 and 64, O at 128, P buffers (packed fp16, 32 columns each) at 192 and 224; the linear
+// branch's product reuses S buffer 0.
+constexpr uint32_t kColS = 0, kColO = 128, kColP = 192, kColL = 0;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRescaleThreshold = 8.0f;  // lazy rescale: keep the old reference max until it is beaten by 2^8
 constexpr float kNoMax = -1.0e30f;         // reference maximum of a row that has seen no valid key yet
-constexpr uint32_t kOffX = 8192;           // epilogue exchange between the sets: reuses K stage 0 (4 KB)
 
 // shared-memory map (bytes from a 1024-aligned base)
-constexpr uint32_t kQBytes = 8192, kKStage = 8192, kVStage = 16384, kPBuf = 16384;
+constexpr uint32_t kQBytes = 8192, kKStage = 8192, kVStage = 16384;
 constexpr uint32_t kOffQ = 0;
 constexpr uint32_t kOffK = kOffQ + kQBytes;
 constexpr uint32_t kOffV = kOffK + kStages * kKStage;
-constexpr uint32_t kOffP = kOffV + kStages * kVStage;
-constexpr uint32_t kOffG = kOffK + kKStage;  // aggregated summaries of the linear branch: K stages 1-2 (16 KB)
-constexpr uint32_t kOffZeta = kOffX + 4096;  // their denominators zeta_i (256 B per query block): rest of K stage 0
-constexpr uint32_t kOffBar = kOffP + 2 * kPBuf;
-constexpr uint32_t kSmemBytes = kOffBar + 256;  // two CTAs per SM: 2 * (114944 + 1024 reserved) <= 232448
+constexpr uint32_t kOffZeta = kOffV + kStages * kVStage;  // zeta_i of the linear branch (256 B per query block)
+constexpr uint32_t kOffRef = kOffZeta + 512;              // per row: {reference maximum, number of steps published}
+constexpr uint32_t kOffX = kOffRef + 1024;                // epilogue exchange between the warpgroups (2 x 128 x 8 B)
+constexpr uint32_t kOffBar = kOffX + 2048;
+constexpr uint32_t kSmemBytes = kOffBar + 512;  // two CTAs per SM: 2 * (110592 + 1024 reserved) <= 232448
+// after the main loop the rings are reused: aggregated summaries G_i in K stages 0-1 (16 KB), the phi(Q) operand in
+// K stages 2-3 (16 KB), the output rows in the V ring (32 KB)
+constexpr uint32_t kOffG = kOffK;
+constexpr uint32_t kOffPhi = kOffK + 2 * kKStage;
+constexpr uint32_t kOffOut = kOffV;
 
 struct Bars {
-  uint64_t q_full, g_full, phi_full, l_full, x_full;
-  uint64_t k_full[kStages], v_full[kStages];  // TMA -> issuers
-  uint64_t qk_done[kRing], pv_done[kRing];    // product of step t complete: barrier t % 6, phase (t / 6)
-  uint64_t s_empty[2], p_full[2];             // softmax set b -> issuer b
+  uint64_t q_full, z_full, g_full, phi_full, l_full, x_full;
+  uint64_t k_full[kStages], v_full[kStages];  // TMA -> issuer
+  uint64_t k_free[kStages];                   // Q K^T of the step in this stage complete -> producer
+  uint64_t pv_done[kStages];                  // P V of the step in this stage complete -> producer, softmax
+  uint64_t qk_done[2];                        // S buffer written -> softmax
+  uint64_t s_empty[2], p_full[2];             // softmax -> issuer
   uint32_t tmem_base;
   int abort;
 };
 
 struct AttnParams {
-  const uint8_t* q_codes;
   const float* q_scales;
   const float* k_scales;
-  const int* crit_idx; // [B*H*Nb][k_crit]
-  const float* zeta;   // [B*H*Nb][64]
-  float* out;
+  const int* crit_idx;  // [B*H*Nb][k_crit]
+  const float* zeta;    // [B*H*Nb][64]
+  void* out;
   long long out_stride_b, out_stride_h, out_stride_n;
-  int heads, tokens, nb, k_crit, k_marg, phi;
+  int heads, tokens, nb, k_crit, k_marg, phi, out_dtype;
   int* status;
 };
 
@@ -92,6 +102,57 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 __device__ __forceinline__ uint32_t pack_bf162(float a, float b) {
   __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<uint32_t*>(&h);
+}
+// D[tmem] (+)= A[tmem] * B[smem], kind::f16: the A operand (M x 16 halves per instruction = 8 columns of packed
+// pairs, row = TMEM lane) is read from tensor memory.
+__device__ __forceinline__ void mma_f16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                           uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// One aligned 8-byte word of shared memory, read / written by a single instruction that the compiler may neither
+// drop nor reorder against other volatile accesses.
+__device__ __forceinline__ uint2 lds_volatile_v2(uint32_t addr) {
+  uint2 v;
+  asm volatile("ld.volatile.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void sts_volatile_v2(uint32_t addr, uint32_t x, uint32_t y) {
+  asm volatile("st.volatile.shared.v2.u32 [%0], {%1, %2};" ::"r"(addr), "r"(x), "r"(y) : "memory");
+}
+
+// Polls a row's reference slot until `count` steps have been published (bounded like every other wait).
+static __device__ __noinline__ bool reference_wait_slow(uint32_t slot, int count, uint2& v, volatile int* abort_flag, int* status) {
+  const uint64_t t0 = global_timer_ns();
+  uint32_t polls = 0;
+  while (true) {
+    v = lds_volatile_v2(slot);
+    if (static_cast<int>(v.y) == count) return true;
+    if ((++polls & 0x3Fu) == 0) {
+      if (*abort_flag != 0) return false;
+      if (global_timer_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 309;
+        if (status != nullptr) atomicCAS(status, 0, 309);
+        return false;
+      }
+    }
+  }
+}
+// Scales the 64 accumulator columns of this thread's TMEM lane by alpha (lazy rescale of O; rare).
+static __device__ __noinline__ void rescale_accumulator(uint32_t o_addr, float alpha) {
+#pragma unroll 1
+  for (int part = 0; part < 4; ++part) {
+    uint32_t o[16];
+    tmem_ld16(o_addr + part * 16, o);
+    tmem_wait_ld();
+#pragma unroll
+    for (int k = 0; k < 16; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
+    tmem_st16(o_addr + part * 16, o);
+  }
 }
 
 // exp2 of 32 scaled scores, packed to fp16 pairs; returns the sum.  Arguments and sums run on pairs of columns
@@ -145,19 +206,19 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
   if (threadIdx.x == 0) {
     mbar_init(&bars->q_full, 1);
+    mbar_init(&bars->z_full, 1);
+    mbar_init(&bars->x_full, kSoftmaxThreads);
     mbar_init(&bars->g_full, 1);
     mbar_init(&bars->phi_full, kSoftmaxThreads);
     mbar_init(&bars->l_full, 1);
-    mbar_init(&bars->x_full, kSoftmaxThreads);
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&bars->k_full[s], 1);
       mbar_init(&bars->v_full[s], 1);
-    }
-    for (int r = 0; r < kRing; ++r) {
-      mbar_init(&bars->qk_done[r], 1);
-      mbar_init(&bars->pv_done[r], 1);
+      mbar_init(&bars->k_free[s], 1);
+      mbar_init(&bars->pv_done[s], 1);
     }
     for (int b = 0; b < 2; ++b) {
+      mbar_init(&bars->qk_done[b], 1);
       mbar_init(&bars->s_empty[b], kSetThreads);
       mbar_init(&bars->p_full[b], kSetThreads);
     }
@@ -168,11 +229,16 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     tmem_alloc(&bars->tmem_base, kTmemCols);
     tmem_relinquish();
   }
+  if (threadIdx.x >= kCtrlWarps * 32 && threadIdx.x < kCtrlWarps * 32 + 128)
+    reinterpret_cast<uint2*>(smem + kOffRef)[threadIdx.x - kCtrlWarps * 32] = make_uint2(__float_as_uint(kNoMax), 0u);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = bars->tmem_base;
+  // each branch below starts by giving registers back (control warps) or taking them (softmax warps)
 
+  if (warp < kCtrlWarps) {
+  setmaxnreg_dec<kCtrlRegs>();
   if (warp == 0) {
     // ------------------------------------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -187,6 +253,11 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         tma_load_2d(smem + kOffQ, &map_q, &bars->q_full, 0, static_cast<int>((bh_rows + i_q[0]) * 128));
         tma_load_2d(smem + kOffQ + 4096, &map_q, &bars->q_full, 0, static_cast<int>((bh_rows + i_q[0]) * 128 + 64));
       }
+      if (p.k_marg > 0) {  // the denominators of the linear branch have a place of their own: fetched right away
+        mbar_arrive_expect_tx(&bars->z_full, kHalves * 256);
+        for (int hf = 0; hf < kHalves; ++hf)
+          bulk_load(smem + kOffZeta + hf * 256, p.zeta + (bh_rows + i_q[hf]) * kHeadDim, 256, &bars->z_full);
+      }
       const int* list0 = p.crit_idx + (bh_rows + i_q[0]) * p.k_crit;
       const int* list1 = p.crit_idx + (bh_rows + i_q[1]) * p.k_crit;
       // tile row (in the code tensors) of step t for query block hf
@@ -194,133 +265,98 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         if (kPair) return static_cast<int>((bh_rows + ldg_pinned((hf ? list1 : list0) + t)) * 64);
         return static_cast<int>((bh_rows + ldg_pinned(list0 + t / 2)) * 128 + (t & 1) * 64);
       };
-      // K and V tiles are loaded by two independent cursors: a K stage is free after the Q K^T of three steps
-      // earlier, a V stage only after that step's P V, and neither load may wait behind the other's condition.
-      // The rows of each cursor's next step are fetched one step ahead.
-      int tk = 0, tv = 0;
+      // The K cursor runs one step ahead of the V cursor (a K stage is free after the Q K^T of four steps earlier,
+      // a V stage only after that step's P V, and Q K^T of step t is issued before P V of step t-1).  The events the
+      // two cursors wait for alternate in time in exactly this order, so blocking waits lose nothing.  The tile rows
+      // of each cursor's next step are fetched one step ahead.
       int rk[2] = {0, 0}, rv[2] = {0, 0};
       if (steps > 0) {
         for (int hf = 0; hf < kHalves; ++hf) rk[hf] = rv[hf] = tile_row(0, hf);
       }
-      IdleGuard guard;
       bool ok = true;
-      while (ok && (tk < steps || tv < steps)) {
-        bool moved = false;
+      for (int i = 0; ok && i <= steps; ++i) {
+        const int tk = i, tv = i - 1;
         if (tk < steps) {
-          const int u = tk - kStages;
-          if (u < 0 || mbar_test(&bars->qk_done[u % kRing], (u / kRing) & 1)) {
-            const int st = tk % kStages;
-            mbar_arrive_expect_tx(&bars->k_full[st], kKTx);
-            for (int hf = 0; hf < kHalves; ++hf)
-              tma_load_2d(smem + kOffK + st * kKStage + hf * 4096, &map_k, &bars->k_full[st], 0, rk[hf]);
-            if (++tk < steps) {
-              for (int hf = 0; hf < kHalves; ++hf) rk[hf] = tile_row(tk, hf);
-            }
-            moved = true;
+          const int st = tk % kStages;
+          if (tk >= kStages)
+            ok = mbar_wait(&bars->k_free[st], ((tk - kStages) / kStages) & 1, abort_flag, p.status, 101, kBackoffNs);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&bars->k_full[st], kKTx);
+          for (int hf = 0; hf < kHalves; ++hf)
+            tma_load_2d(smem + kOffK + st * kKStage + hf * 4096, &map_k, &bars->k_full[st], 0, rk[hf]);
+          if (tk + 1 < steps) {
+            for (int hf = 0; hf < kHalves; ++hf) rk[hf] = tile_row(tk + 1, hf);
           }
         }
-        if (tv < steps) {
-          const int u = tv - kStages;
-          if (u < 0 || mbar_test(&bars->pv_done[u % kRing], (u / kRing) & 1)) {
-            const int st = tv % kStages;
-            mbar_arrive_expect_tx(&bars->v_full[st], kVTx);
-            for (int hf = 0; hf < kHalves; ++hf)
-              tma_load_2d(smem + kOffV + st * kVStage + hf * 8192, &map_v, &bars->v_full[st], 0, rv[hf]);
-            if (++tv < steps) {
-              for (int hf = 0; hf < kHalves; ++hf) rv[hf] = tile_row(tv, hf);
-            }
-            moved = true;
+        if (tv >= 0) {
+          const int st = tv % kStages;
+          if (tv >= kStages)
+            ok = mbar_wait(&bars->pv_done[st], ((tv - kStages) / kStages) & 1, abort_flag, p.status, 102, kBackoffNs);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&bars->v_full[st], kVTx);
+          for (int hf = 0; hf < kHalves; ++hf)
+            tma_load_2d(smem + kOffV + st * kVStage + hf * 8192, &map_v, &bars->v_full[st], 0, rv[hf]);
+          if (tv + 1 < steps) {
+            for (int hf = 0; hf < kHalves; ++hf) rv[hf] = tile_row(tv + 1, hf);
           }
-        }
-        if (moved) {
-          guard.progress();
-        } else {
-          ok = guard.idle(abort_flag, p.status, 101, kBackoffNs);
         }
       }
       if (ok && p.k_marg > 0) {
-        // The aggregated summaries go to K stages 1 and 2, which are free once the last three Q K^T products have
+        // The aggregated summaries go to K stages 0 and 1, which are free once the last Q K^T products have
         // completed: well before the last P V products, so this load is off the tail's critical path.
         for (int u = max(0, steps - kStages); u < steps && ok; ++u)
-          ok = mbar_wait(&bars->qk_done[u % kRing], (u / kRing) & 1, abort_flag, p.status, 103, kBackoffNs);
+          ok = mbar_wait(&bars->k_free[u % kStages], (u / kStages) & 1, abort_flag, p.status, 103, kBackoffNs);
         if (ok) {
-          mbar_arrive_expect_tx(&bars->g_full, kHalves * (8192 + 256));
-          for (int hf = 0; hf < kHalves; ++hf) {
+          mbar_arrive_expect_tx(&bars->g_full, kHalves * 8192);
+          for (int hf = 0; hf < kHalves; ++hf)
             tma_load_2d(smem + kOffG + hf * 8192, &map_g, &bars->g_full, 0, static_cast<int>((bh_rows + i_q[hf]) * 64));
-            bulk_load(smem + kOffZeta + hf * 256, p.zeta + (bh_rows + i_q[hf]) * kHeadDim, 256, &bars->g_full);
-          }
         }
       }
     }
-  } else if (warp < kCtrlWarps) {
-    // ------------------------------------------------------------------------------------------ MMA issuer of set b
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------------------------------ Q K^T issuer
+    // One thread issues a small tcgen05.mma about every 55 clocks and pays some 100 clocks per barrier it looks
+    // at, so the two products of a step have an issuing thread each (this warp and the next); a single issuer for
+    // both was measured to be the bottleneck of the whole kernel.  Operand descriptors are built once and advanced by
+    // adding byte offsets (in 16-byte units) to their address field.
     if (lane == 0) {
-      const int b = warp - 1;
       constexpr uint32_t idesc_qk = instr_desc(0, kM, 64, 0, 0);   // e4m3 x e4m3, both K-major
-      constexpr uint32_t idesc_pv = instr_desc(0, kM, 64, 0, 1);   // f16 x f16, V MN-major
       constexpr uint32_t idesc_lin = instr_desc(1, kM, 64, 0, 0);  // bf16 x bf16, both K-major
-      const uint32_t q_addr = smem_u32(smem + kOffQ), k_addr = smem_u32(smem + kOffK);
-      const uint32_t v_addr = smem_u32(smem + kOffV), p_addr = smem_u32(smem + kOffP) + b * kPBuf;
-      const uint32_t s_tmem = tmem + kColS + b * 64, o_tmem = tmem + kColO + b * 64;
+      const uint32_t q_addr = smem_u32(smem + kOffQ);
+      const uint64_t k_desc0 = smem_desc(smem_u32(smem + kOffK), 16, 512, kSwizzle64);
       bool ok = mbar_wait(&bars->q_full, 0, abort_flag, p.status, 201, kBackoffNs);
-      auto issue_qk = [&](int t) {  // S_b = Q K(t)^T
+      uint64_t q_desc[2][kHalves];
+#pragma unroll
+      for (int kk = 0; kk < 2; ++kk)
+#pragma unroll
+        for (int hf = 0; hf < kHalves; ++hf)
+          q_desc[kk][hf] = smem_desc(q_addr + (kPair ? hf * 4096 : 0) + kk * 32, 16, 512, kSwizzle64);
+      // S[t&1] = Q K(t)^T needs the K tile of step t and S[t&1] drained by the softmax threads of step t-2; it runs
+      // one step ahead of the softmax threads, so the scores of step t are waiting when step t-1 is finished.
+      for (int t = 0; ok && t < steps; ++t) {
         const int st = t % kStages;
+        ok = mbar_wait(&bars->k_full[st], (t / kStages) & 1, abort_flag, p.status, 202, kBackoffNs);
+        if (ok && t >= 2)
+          ok = mbar_wait(&bars->s_empty[t & 1], ((t - 2) >> 1) & 1, abort_flag, p.status, 203, kBackoffNs);
+        if (!ok) break;
+        const uint32_t s_tmem = tmem + kColS + (t & 1) * 64;
+        const uint64_t k_desc = k_desc0 + static_cast<uint64_t>((st * kKStage) >> 4);
         tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < 2; ++kk) {
 #pragma unroll
-          for (int hf = 0; hf < kHalves; ++hf) {
-            const uint64_t a = smem_desc(q_addr + (kPair ? hf * 4096 : 0) + kk * 32, 16, 512, kSwizzle64);
-            const uint64_t bd = smem_desc(k_addr + st * kKStage + hf * 4096 + kk * 32, 16, 512, kSwizzle64);
-            mma_f8(s_tmem + ((hf * 16u) << 16), a, bd, idesc_qk, kk);
-          }
+          for (int hf = 0; hf < kHalves; ++hf)
+            mma_f8(s_tmem + ((hf * 16u) << 16), q_desc[kk][hf], k_desc + ((hf * 4096 + kk * 32) >> 4), idesc_qk, kk);
         }
-        mma_commit(&bars->qk_done[t % kRing]);
-      };
-      auto issue_pv = [&](int t) {  // O_b += P(t) V(t)
-        const int st = t % kStages;
-        tc_fence_after();
-#pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
-#pragma unroll
-          for (int hf = 0; hf < kHalves; ++hf) {
-            const uint64_t a = smem_desc(p_addr + (kPair ? hf * 8192 : 0) + kk * 32, 16, 1024, kSwizzle128);
-            const uint64_t bd = smem_desc(v_addr + st * kVStage + hf * 8192 + kk * 2048, 8192, 1024, kSwizzle128);
-            mma_f16(o_tmem + ((hf * 16u) << 16), a, bd, idesc_pv, (t >= 2 || kk > 0) ? 1u : 0u);
-          }
-        }
-        mma_commit(&bars->pv_done[t % kRing]);
-      };
-      // Two cursors, polled without blocking, so that neither product waits behind the other's operands:
-      //   Q K^T of step tq needs its K tile and S_b drained by the softmax of the set's previous step (tq - 2);
-      //   P V of step tp needs its V tile and the probabilities of step tp.
-      int tq = b, tp = b;
-      IdleGuard guard;
-      while (ok && tp < steps) {
-        bool moved = false;
-        if (mbar_test(&bars->p_full[b], (tp >> 1) & 1) && mbar_test(&bars->v_full[tp % kStages], (tp / kStages) & 1)) {
-          issue_pv(tp);
-          tp += 2;
-          moved = true;
-        }
-        if (tq < steps && mbar_test(&bars->k_full[tq % kStages], (tq / kStages) & 1) &&
-            mbar_test(&bars->s_empty[b], ((tq >> 1) & 1) ^ 1)) {
-          issue_qk(tq);
-          tq += 2;
-          moved = true;
-        }
-        if (moved) {
-          guard.progress();
-        } else {
-          ok = guard.idle(abort_flag, p.status, 202, 0);
-        }
+        mma_commit(&bars->qk_done[t & 1]);
+        mma_commit(&bars->k_free[st]);
       }
-      if (b == 0 && ok && p.k_marg > 0) {
+      if (ok && p.k_marg > 0) {
         ok = mbar_wait(&bars->g_full, 0, abort_flag, p.status, 206, kBackoffNs) &&
              mbar_wait(&bars->phi_full, 0, abort_flag, p.status, 207, kBackoffNs);
         if (ok) {
           tc_fence_after();
-          const uint32_t phi_addr = smem_u32(smem + kOffP), g_addr = smem_u32(smem + kOffG);
+          const uint32_t phi_addr = smem_u32(smem + kOffPhi), g_addr = smem_u32(smem + kOffG);
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk) {
 #pragma unroll
@@ -334,33 +370,68 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
       }
     }
+  } else if (warp == 2) {
+    // ------------------------------------------------------------------------------------------ P V issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_pv = instr_desc(0, kM, 64, 0, 1);  // f16 x f16, P from TMEM, V MN-major
+      const uint64_t v_desc0 = smem_desc(smem_u32(smem + kOffV), 8192, 1024, kSwizzle128);
+      const uint32_t o_tmem = tmem + kColO;
+      bool ok = true;
+      for (int t = 0; ok && t < steps; ++t) {  // O += P[t&1] V(t)
+        const int st = t % kStages;
+        ok = mbar_wait(&bars->v_full[st], (t / kStages) & 1, abort_flag, p.status, 205, kBackoffNs) &&
+             mbar_wait(&bars->p_full[t & 1], (t >> 1) & 1, abort_flag, p.status, 204, kBackoffNs);
+        if (!ok) break;
+        const uint32_t p_tmem = tmem + kColP + (t & 1) * 32;
+        const uint64_t v_desc = v_desc0 + static_cast<uint64_t>((st * kVStage) >> 4);
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+#pragma unroll
+          for (int hf = 0; hf < kHalves; ++hf)
+            mma_f16_ts(o_tmem + ((hf * 16u) << 16), p_tmem + ((hf * 16u) << 16) + kk * 8,
+                       v_desc + ((hf * 8192 + kk * 2048) >> 4), idesc_pv, (t > 0 || kk > 0) ? 1u : 0u);
+        }
+        mma_commit(&bars->pv_done[st]);
+      }
+    }
+  }
   } else {
     // ------------------------------------------------------------------------------------------ softmax + epilogue
+    setmaxnreg_inc<kSoftmaxRegs>();
     const int quarter = warp & 3;                       // TMEM sub-partition this warp may touch
-    const int b = (warp - kCtrlWarps) >> 2;             // set: steps t with (t & 1) == b
+    const int w = (warp - kCtrlWarps) >> 2;             // warpgroup: steps t with (t & 1) == w
     const int hf = kPair ? (lane >> 4) : 0;             // which query block of the pair this thread serves
     const int row_in_block = kPair ? quarter * 16 + (lane & 15) : quarter * 32 + lane;
-    const int p_row = kPair ? hf * 64 + row_in_block : row_in_block;  // row inside the P / phi tile
+    const int p_row = kPair ? hf * 64 + row_in_block : row_in_block;  // row inside the 128-row tile
     const int iq = i_q[hf];
     const size_t q_tile = bh_rows + iq;
     const uint32_t lane_addr = tmem + ((static_cast<uint32_t>(quarter) * 32u) << 16);
-    const uint32_t s_addr = lane_addr + kColS + b * 64, o_addr = lane_addr + kColO + b * 64;
+    const uint32_t s_addr = lane_addr + kColS + w * 64, p_addr = lane_addr + kColP + w * 32, o_addr = lane_addr + kColO;
     const float sq = __ldg(p.q_scales + q_tile);
     const float qk_scale = sq * (kLog2e * 0.125f);
     const int* list = p.crit_idx + q_tile * p.k_crit;
-    uint8_t* const prow = smem + kOffP + b * kPBuf + p_row * 128;  // this thread's 128-byte row of P_b
-    const int swz = p_row & 7;
+    const uint32_t ref_slot = smem_u32(smem + kOffRef) + p_row * 8;
 
-    float m_ref = kNoMax, l = 0.f;
+    float m_seen = kNoMax, l = 0.f;  // reference this warpgroup's row sum is relative to; the row sum
     bool ok = true;
 
-    // per-step scalars: the key-block index is fetched two of the set's steps ahead and its scale one ahead, so
-    // that no load in the loop waits for the address produced by another load of the same iteration
-    int j_cur = b < steps ? ldg_pinned(list + b / kStepsPerBlock) : 0;
-    int j_nxt = b + 2 < steps ? ldg_pinned(list + (b + 2) / kStepsPerBlock) : 0;
-    float sk_cur = b < steps ? ldg_pinned(p.k_scales + bh_rows + j_cur) : 0.f;
+    // Waits until `count` steps have published their reference for this row and returns it.  The slot is one aligned
+    // 8-byte word written by a single store, so value and count are always seen together.
+    auto reference_after = [&](int count, float& m) -> bool {
+      uint2 v = lds_volatile_v2(ref_slot);
+      if (static_cast<int>(v.y) != count && !reference_wait_slow(ref_slot, count, v, abort_flag, p.status)) return false;
+      m = __uint_as_float(v.x);
+      return true;
+    };
 
-    for (int t = b; t < steps; t += 2) {
+    // per-step scalars: the key-block index is fetched two of the warpgroup's steps ahead and its scale one ahead, so
+    // that no load in the loop waits for the address produced by another load of the same iteration
+    int j_cur = w < steps ? ldg_pinned(list + w / kStepsPerBlock) : 0;
+    int j_nxt = w + 2 < steps ? ldg_pinned(list + (w + 2) / kStepsPerBlock) : 0;
+    float sk_cur = w < steps ? ldg_pinned(p.k_scales + bh_rows + j_cur) : 0.f;
+
+    for (int t = w; t < steps; t += 2) {
       const int j = j_cur;
       const float c = qk_scale * sk_cur;
       j_cur = j_nxt;
@@ -369,37 +440,42 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       int valid = p.tokens - j * BS - (kPair ? 0 : (t & 1) * kStepKeys);
       valid = max(0, min(kStepKeys, valid));
 
-      if (!(ok = mbar_wait(&bars->qk_done[t % kRing], (t / kRing) & 1, abort_flag, p.status, 301))) break;
+      if (!(ok = mbar_wait_far(&bars->qk_done[w], (t >> 1) & 1, abort_flag, p.status, 301))) break;
       tc_fence_after();
-
-      // pass 1: row maximum of the raw scores (c > 0 commutes with max), four independent chains
-      float tile_max;
+      uint32_t xa[32];
+      float mx4[4];
       {
-        uint32_t x[32], y[32];
-        tmem_ld32(s_addr, x);
-        tmem_ld32(s_addr + 32, y);
+        uint32_t xb[32];
+        tmem_ld32(s_addr, xa);
+        tmem_ld32(s_addr + 32, xb);
         tmem_wait_ld();
         if (valid < kStepKeys) {
 #pragma unroll
           for (int k = 0; k < 32; ++k) {
-            if (k >= valid) x[k] = 0xFF800000u;  // -inf
-            if (32 + k >= valid) y[k] = 0xFF800000u;
+            if (k >= valid) xa[k] = 0xFF800000u;  // -inf
+            if (32 + k >= valid) xb[k] = 0xFF800000u;
           }
         }
-        float mx4[4];
+        // row maximum of the raw scores (c > 0 commutes with max), four independent chains
 #pragma unroll
-        for (int q = 0; q < 4; ++q) mx4[q] = fmaxf(__uint_as_float(x[q]), __uint_as_float(y[q]));
+        for (int q = 0; q < 4; ++q) mx4[q] = fmaxf(__uint_as_float(xa[q]), __uint_as_float(xb[q]));
 #pragma unroll
         for (int k = 4; k < 32; k += 4) {
 #pragma unroll
-          for (int q = 0; q < 4; ++q) mx4[q] = max3(mx4[q], __uint_as_float(x[k + q]), __uint_as_float(y[k + q]));
+          for (int q = 0; q < 4; ++q) mx4[q] = max3(mx4[q], __uint_as_float(xa[k + q]), __uint_as_float(xb[k + q]));
         }
-        // a step without any valid key (second half of a short last block) leaves the reference where it is
-        tile_max = fmaxf(max3(fmaxf(mx4[0], mx4[1]), mx4[2], mx4[3]) * c, kNoMax);
       }
+      // a step without any valid key (second half of a short last block) leaves the reference where it is
+      const float tile_max = fmaxf(max3(fmaxf(mx4[0], mx4[1]), mx4[2], mx4[3]) * c, kNoMax);
+
+      // the row's reference after step t-1 (published early in that step by the other warpgroup), the lazy-rescale
+      // decision of this step, and its publication for step t+1
+      float m_ref = kNoMax;
+      if (t > 0 && !(ok = reference_after(t, m_ref))) break;
+      if (m_ref != m_seen) l *= ex2(m_seen - m_ref);  // bring this warpgroup's row sum to the current reference
       bool need = false;
       float alpha = 1.f;
-      if (t < 2) {
+      if (t == 0) {
         m_ref = tile_max;
       } else if (tile_max > m_ref + kRescaleThreshold) {
         need = true;
@@ -407,79 +483,64 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         m_ref = tile_max;
         l *= alpha;
       }
-      // P_b is free once the P V product of the set's previous step has completed; asked now, needed after the
-      // first exponentials
-      uint64_t* const pv_bar = &bars->pv_done[(t + kRing - 2) % kRing];
-      const uint32_t pv_par = static_cast<uint32_t>(((t - 2) / kRing) & 1);
-      const bool pv_ok = t < 2 || mbar_try_wait(pv_bar, pv_par);
+      m_seen = m_ref;
+      sts_volatile_v2(ref_slot, __float_as_uint(m_ref), static_cast<uint32_t>(t + 1));
 
-      // pass 2: exponentials and row sum, 32 columns at a time; each half row of P is stored as soon as it exists
+      // P[w] is free once the P V product of step t-2 has completed (long ago in the steady state)
+      if (t >= 2 && !(ok = mbar_wait_far(&bars->pv_done[(t - 2) % kStages], ((t - 2) / kStages) & 1, abort_flag, p.status, 302)))
+        break;
+      tc_fence_after();
       {
-        uint32_t x[32], packed[16];
-        tmem_ld32(s_addr, x);
-        tmem_wait_ld();
-        if (valid < 32) {
-#pragma unroll
-          for (int k = 0; k < 32; ++k)
-            if (k >= valid) x[k] = 0xFF800000u;
-        }
-        l += exp_half_row(x, c, -m_ref, packed);
-        if (!pv_ok && !(ok = mbar_wait(pv_bar, pv_par, abort_flag, p.status, 302))) break;
-#pragma unroll
-        for (int ch = 0; ch < 4; ++ch)
-          *reinterpret_cast<uint4*>(prow + ((ch ^ swz) << 4)) =
-              make_uint4(packed[4 * ch], packed[4 * ch + 1], packed[4 * ch + 2], packed[4 * ch + 3]);
-        tmem_ld32(s_addr + 32, x);
+        // the second half of the row is read again instead of being held across the first half's exponentials;
+        // S[w] is released once it is in registers
+        uint32_t packed[16];
+        l += exp_half_row(xa, c, -m_ref, packed);
+        tmem_st16(p_addr, packed);
+        tmem_ld32(s_addr + 32, xa);
         tmem_wait_ld();
         tc_fence_before();
-        mbar_arrive(&bars->s_empty[b]);  // S_b is in registers: the issuer may overwrite it with the set's next step
+        mbar_arrive(&bars->s_empty[w]);  // the issuer may overwrite S[w] with step t+2
         if (valid < kStepKeys) {
 #pragma unroll
           for (int k = 0; k < 32; ++k)
-            if (32 + k >= valid) x[k] = 0xFF800000u;
+            if (32 + k >= valid) xa[k] = 0xFF800000u;
         }
-        l += exp_half_row(x, c, -m_ref, packed);
-#pragma unroll
-        for (int ch = 0; ch < 4; ++ch)
-          *reinterpret_cast<uint4*>(prow + (((4 + ch) ^ swz) << 4)) =
-              make_uint4(packed[4 * ch], packed[4 * ch + 1], packed[4 * ch + 2], packed[4 * ch + 3]);
+        l += exp_half_row(xa, c, -m_ref, packed);
+        tmem_st16(p_addr + 16, packed);
       }
       if (__any_sync(0xFFFFFFFFu, need)) {
-        // O_b is only touched by the set's own P V products: the previous one has completed (pv_bar above) and the
-        // next one waits for this thread's arrival below
+        // O is being accumulated into by the P V product of step t-1: wait for it, then scale the rows whose
+        // reference moved.  The product of this step waits for this thread's arrival below.
+        if (!(ok = mbar_wait_far(&bars->pv_done[(t - 1) % kStages], ((t - 1) / kStages) & 1, abort_flag, p.status, 303))) break;
         tc_fence_after();
-#pragma unroll
-        for (int part = 0; part < 2; ++part) {
-          uint32_t o[32];
-          tmem_ld32(o_addr + part * 32, o);
-          tmem_wait_ld();
-#pragma unroll
-          for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
-          tmem_st32(o_addr + part * 32, o);
-        }
-        tmem_wait_st();
-        tc_fence_before();
+        rescale_accumulator(o_addr, alpha);
       }
-      fence_proxy_async_smem();
-      mbar_arrive(&bars->p_full[b]);
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(&bars->p_full[w]);
     }
 
-    // linear branch: this thread's 32 columns (set b -> columns 32 b ..) of phi(q) as bf16 A operand, partial
-    // denominator on the side; computed in registers while the last P V products are still running.  The query row
-    // comes from the Q tile in shared memory (64-byte rows, 64B swizzle: 16-byte chunk c of row r sits at chunk
-    // c ^ ((r >> 1) & 3)), zeta_i from the copy that arrived with the aggregated summaries.
+    // linear branch: this thread's 32 columns (warpgroup w -> columns 32 w ..) of phi(q) as bf16 A operand, partial
+    // denominator phi(q) . zeta_i on the side; computed in registers while the last P V products are still running.
+    // The query row comes from the Q tile in shared memory (64-byte rows, 64B swizzle: 16-byte chunk c of row r sits at
+    // chunk c ^ ((r >> 1) & 3)).  Every Q K^T product has completed once both warpgroups are here, which the issuer
+    // of the linear product checks through phi_full; the operand goes to K stages 2 and 3, which this warpgroup's own
+    // steps and, by the order of the products, all earlier ones no longer read.
     float den = 0.f;
-    uint32_t phi_packed[16];
+    const int swz = p_row & 7;
     if (ok && p.k_marg > 0) {
-      ok = mbar_wait(&bars->q_full, 0, abort_flag, p.status, 307) && mbar_wait(&bars->g_full, 0, abort_flag, p.status, 308);
+      ok = mbar_wait_far(&bars->q_full, 0, abort_flag, p.status, 307) && mbar_wait_far(&bars->z_full, 0, abort_flag, p.status, 308);
+      // the other warpgroup's last Q K^T may still be reading K stage 2 or 3: wait for the last two steps' products
+      for (int u = max(0, steps - 2); u < steps && ok; ++u)
+        ok = mbar_wait_far(&bars->k_free[u % kStages], (u / kStages) & 1, abort_flag, p.status, 310);
       const uint8_t* qrow = smem + kOffQ + p_row * 64;
-      const float4* zeta = reinterpret_cast<const float4*>(smem + kOffZeta + hf * 256 + b * 128);
+      const float4* zeta = reinterpret_cast<const float4*>(smem + kOffZeta + hf * 256 + w * 128);
       const int qswz = (p_row >> 1) & 3;
       float e[32];
-      float mx = -INFINITY;
+      float mxq[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int w = 0; w < 4; ++w) {
-        const uint4 raw = *reinterpret_cast<const uint4*>(qrow + ((w ^ qswz) << 4));
+      for (int c4 = 0; c4 < 4; ++c4) {
+        const uint4 raw = *reinterpret_cast<const uint4*>(qrow + ((c4 ^ qswz) << 4));
         const uint32_t words[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
         for (int xw = 0; xw < 4; ++xw) {
@@ -487,122 +548,134 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           e4m3x4_to_float(words[xw], fv);
 #pragma unroll
           for (int y = 0; y < 4; ++y) {
-            mx = fmaxf(mx, fv[y]);
-            if ((w >> 1) == b) e[(w & 1) * 16 + xw * 4 + y] = fv[y];
+            mxq[y] = fmaxf(mxq[y], fv[y]);
+            if ((c4 >> 1) == w) e[(c4 & 1) * 16 + xw * 4 + y] = fv[y];
           }
         }
       }
+      const float mx = fmaxf(fmaxf(mxq[0], mxq[1]), fmaxf(mxq[2], mxq[3]));
       const float cq = sq * kLog2e, shift = mx * cq;  // sq > 0 commutes with max
+      uint8_t* const phirow = smem + kOffPhi + p_row * 128;
+      float den4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int d = 0; d < 32; d += 4) {
-        const float4 z = zeta[d >> 2];
-        const float zz[4] = {z.x, z.y, z.z, z.w};
+      for (int ch = 0; ch < 4; ++ch) {  // 16-byte chunk = 8 columns
+        uint32_t pk4[4];
+        const float4 za = zeta[2 * ch], zb = zeta[2 * ch + 1];
+        const float zz[8] = {za.x, za.y, za.z, za.w, zb.x, zb.y, zb.z, zb.w};
 #pragma unroll
-        for (int y = 0; y < 4; y += 2) {
+        for (int y = 0; y < 8; y += 2) {
+          const int d = ch * 8 + y;
           float e0, e1;
           if (p.phi == LITE3R_PHI_SOFTMAX) {  // the softmax normaliser cancels in the ratio
-            e0 = ex2(fmaf(e[d + y], cq, -shift));
-            e1 = ex2(fmaf(e[d + y + 1], cq, -shift));
+            e0 = ex2(fmaf(e[d], cq, -shift));
+            e1 = ex2(fmaf(e[d + 1], cq, -shift));
           } else {
-            e0 = e[d + y] > 0.f ? fmaf(e[d + y], sq, 1.f) : ex2(e[d + y] * cq);
-            e1 = e[d + y + 1] > 0.f ? fmaf(e[d + y + 1], sq, 1.f) : ex2(e[d + y + 1] * cq);
+            e0 = e[d] > 0.f ? fmaf(e[d], sq, 1.f) : ex2(e[d] * cq);
+            e1 = e[d + 1] > 0.f ? fmaf(e[d + 1], sq, 1.f) : ex2(e[d + 1] * cq);
           }
           const uint32_t pk = pack_bf162(e0, e1);
-          phi_packed[(d + y) >> 1] = pk;
+          pk4[y >> 1] = pk;
           // the denominator uses the same rounded values as the MMA's numerator
-          den = fmaf(__uint_as_float(pk << 16), zz[y], den);
-          den = fmaf(__uint_as_float(pk & 0xFFFF0000u), zz[y + 1], den);
+          den4[y >> 1] = fmaf(__uint_as_float(pk << 16), zz[y], den4[y >> 1]);
+          den4[y >> 1] = fmaf(__uint_as_float(pk & 0xFFFF0000u), zz[y + 1], den4[y >> 1]);
         }
+        *reinterpret_cast<uint4*>(phirow + (((w * 4 + ch) ^ swz) << 4)) = make_uint4(pk4[0], pk4[1], pk4[2], pk4[3]);
       }
-    }
-
-    // both sets' last P V products (the epilogue reads O_0 and O_1, and the phi operand reuses P_0)
-    for (int u = max(0, steps - 2); u < steps && ok; ++u)
-      ok = mbar_wait(&bars->pv_done[u % kRing], (u / kRing) & 1, abort_flag, p.status, 304);
-    tc_fence_after();
-    if (ok && p.k_marg > 0) {
-      uint8_t* const phirow = smem + kOffP + p_row * 128;
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-        *reinterpret_cast<uint4*>(phirow + (((b * 4 + i) ^ swz) << 4)) =
-            make_uint4(phi_packed[4 * i], phi_packed[4 * i + 1], phi_packed[4 * i + 2], phi_packed[4 * i + 3]);
+      den = (den4[0] + den4[1]) + (den4[2] + den4[3]);
       fence_proxy_async_smem();
       mbar_arrive(&bars->phi_full);
     }
 
-    // the two threads of a row (one per set) swap reference maximum, row sum and partial denominator (K stage 0 is
-    // free by now: every Q K^T product has completed before the last P V products did)
-    float w_mine = 0.f, w_other = 0.f, inv_l = 0.f;
+    // the two threads of a row (one per warpgroup) bring their row sums to the final reference and swap them together
+    // with the partial denominators
+    float inv_l = 0.f;
     if (ok) {
-      float4* xbuf = reinterpret_cast<float4*>(smem + kOffX);
-      xbuf[b * 128 + p_row] = make_float4(m_ref, l, den, 0.f);
-      mbar_arrive(&bars->x_full);
-      ok = mbar_wait(&bars->x_full, 0, abort_flag, p.status, 306);
+      float m_fin = kNoMax;
+      if (steps > 0) ok = reference_after(steps, m_fin);
       if (ok) {
-        const float4 other = xbuf[(b ^ 1) * 128 + p_row];
-        const float m = fmaxf(m_ref, other.x);
-        w_mine = ex2(m_ref - m);    // a set without (valid) steps keeps m_ref = kNoMax and l = 0
-        w_other = ex2(other.x - m);
-        const float l_tot = w_mine * l + w_other * other.y;
-        inv_l = steps > 0 ? 1.f / l_tot : 0.f;
-        den += other.z;
+        if (m_fin != m_seen) l *= ex2(m_seen - m_fin);
+        float2* xbuf = reinterpret_cast<float2*>(smem + kOffX);
+        xbuf[w * 128 + p_row] = make_float2(l, den);
+        mbar_arrive(&bars->x_full);
+        ok = mbar_wait_far(&bars->x_full, 0, abort_flag, p.status, 306);
+        if (ok) {
+          const float2 other = xbuf[(w ^ 1) * 128 + p_row];
+          inv_l = steps > 0 ? 1.f / (l + other.x) : 0.f;
+          den += other.y;
+        }
       }
     }
-    if (ok && p.k_marg > 0) {
-      ok = mbar_wait(&bars->l_full, 0, abort_flag, p.status, 305);
-      tc_fence_after();
-    }
+    // the last P V product (commits are cumulative: it covers every earlier one), then the linear product
+    if (ok && steps > 0)
+      ok = mbar_wait_far(&bars->pv_done[(steps - 1) % kStages], ((steps - 1) / kStages) & 1, abort_flag, p.status, 304);
+    if (ok && p.k_marg > 0) ok = mbar_wait_far(&bars->l_full, 0, abort_flag, p.status, 305);
+    tc_fence_after();
 
     ok = __all_sync(0xFFFFFFFFu, ok);  // the store below synchronises the warp
     if (ok) {
       const int bb = bh / p.heads, h = bh % p.heads;
-      // accumulators of a set that ran no step hold no data: they are not read
-      const bool has_mine = steps > b, has_other = steps > (b ^ 1);
       const float l_scale = p.k_marg > 0 ? 1.f / den : 0.f;
-      const float s_mine = has_mine ? w_mine * inv_l : 0.f, s_other = has_other ? w_other * inv_l : 0.f;
+      // The thread's 32 output values go to the V ring (free: every P V product has completed), 16-byte chunks
+      // swizzled by the row so that neither these writes nor the row-wise reads below conflict; then each store
+      // instruction of the warp writes whole half rows (fp32: four rows x 128 bytes, 16-bit: eight rows x 64 bytes).
+      const bool wide = p.out_dtype == LITE3R_F32;
+      const uint32_t row_bytes = wide ? 256u : 128u;
+      uint8_t* const orow = smem + kOffOut + p_row * row_bytes;
       float acc[32];
-#pragma unroll
-      for (int k = 0; k < 32; ++k) acc[k] = 0.f;
       uint32_t v[32];
-      if (has_mine) {
-        tmem_ld32(lane_addr + kColO + b * 64 + b * 32, v);
+      if (steps > 0) {
+        tmem_ld32(o_addr + w * 32, v);
         tmem_wait_ld();
 #pragma unroll
-        for (int k = 0; k < 32; ++k) acc[k] = __uint_as_float(v[k]) * s_mine;
-      }
-      if (has_other) {
-        tmem_ld32(lane_addr + kColO + (b ^ 1) * 64 + b * 32, v);
-        tmem_wait_ld();
+        for (int k = 0; k < 32; ++k) acc[k] = __uint_as_float(v[k]) * inv_l;
+      } else {
 #pragma unroll
-        for (int k = 0; k < 32; ++k) acc[k] = fmaf(__uint_as_float(v[k]), s_other, acc[k]);
+        for (int k = 0; k < 32; ++k) acc[k] = 0.f;
       }
       if (p.k_marg > 0) {
-        tmem_ld32(lane_addr + kColL + b * 32, v);
+        tmem_ld32(lane_addr + kColL + w * 32, v);
         tmem_wait_ld();
 #pragma unroll
         for (int k = 0; k < 32; ++k) acc[k] = fmaf(__uint_as_float(v[k]), l_scale, acc[k]);
       }
-      // A thread owns 128 bytes of one output row, so a direct store would touch 32 different lines per instruction.
-      // The warp's 32 x 128-byte block is turned around in its own rows of P_b (free: P V products and the linear
-      // product have completed) so that every store instruction writes four whole 128-byte row segments.
+      if (wide) {
 #pragma unroll
-      for (int ch = 0; ch < 8; ++ch)
-        *reinterpret_cast<float4*>(prow + ((ch ^ swz) << 4)) =
-            make_float4(acc[4 * ch], acc[4 * ch + 1], acc[4 * ch + 2], acc[4 * ch + 3]);
+        for (int ch = 0; ch < 8; ++ch)
+          *reinterpret_cast<float4*>(orow + (((w * 8 + ch) ^ swz) << 4)) =
+              make_float4(acc[4 * ch], acc[4 * ch + 1], acc[4 * ch + 2], acc[4 * ch + 3]);
+      } else {
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          uint32_t pk[4];
+#pragma unroll
+          for (int y = 0; y < 4; ++y)
+            pk[y] = p.out_dtype == LITE3R_BF16 ? pack_bf162(acc[8 * ch + 2 * y], acc[8 * ch + 2 * y + 1])
+                                                : pack_half2(acc[8 * ch + 2 * y], acc[8 * ch + 2 * y + 1]);
+          *reinterpret_cast<uint4*>(orow + (((w * 4 + ch) ^ swz) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
+      }
       __syncwarp();
-      const int ch = lane & 7;
-      float* const out_bh = p.out + bb * p.out_stride_b + h * p.out_stride_h + b * 32 + ch * 4;
+      const int chunk_shift = wide ? 3 : 2;       // 8 or 4 chunks of 16 bytes per half row
+      const int ch = lane & ((1 << chunk_shift) - 1);
+      const int half_chunks = 1 << chunk_shift;
+      const uint32_t elem = wide ? 4u : 2u;
+      uint8_t* const out_bh = static_cast<uint8_t*>(p.out) +
+                              (static_cast<long long>(bb) * p.out_stride_b + static_cast<long long>(h) * p.out_stride_h) * elem +
+                              w * 32 * elem;
+      const long long row_pitch = p.out_stride_n * static_cast<long long>(elem);
 #pragma unroll
       for (int k = 0; k < 8; ++k) {
-        const int r = 4 * k + (lane >> 3);  // row of this warp's block: the one thread `r` of the warp computed
+        // fp32: pass k covers rows 4k .. 4k+3; 16-bit: rows 8k .. 8k+7, so only k < 4 run
+        if (!wide && k >= 4) break;
+        const int r = wide ? 4 * k + (lane >> 3) : 8 * k + (lane >> 2);  // row of this warp's block: thread r computed it
         const int r_hf = kPair ? (r >> 4) : 0;
         const int r_in_block = kPair ? quarter * 16 + (r & 15) : quarter * 32 + r;
         const int r_p = kPair ? r_hf * 64 + r_in_block : r_in_block;
         const int r_token = i_q[r_hf] * BS + r_in_block;
-        const float4 val =
-            *reinterpret_cast<const float4*>(smem + kOffP + b * kPBuf + r_p * 128 + ((ch ^ (r_p & 7)) << 4));
+        const uint4 val = *reinterpret_cast<const uint4*>(smem + kOffOut + r_p * row_bytes +
+                                                          (((w * half_chunks + ch) ^ (r_p & 7)) << 4));
         if (r_token < p.tokens && (!kPair || r_hf == 0 || i_q[1] != i_q[0]))
-          *reinterpret_cast<float4*>(out_bh + static_cast<long long>(r_token) * p.out_stride_n) = val;
+          *reinterpret_cast<uint4*>(out_bh + r_token * row_pitch + ch * 16) = val;
       }
     }
   }
@@ -628,7 +701,6 @@ lite3r_status launch(const AttentionLaunch& a, cudaStream_t stream) {
   if ((st = make_tensor_map_2d(&map_v, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, a.v16, 64, tiles * BS, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B)) != LITE3R_OK) return st;
   if ((st = make_tensor_map_2d(&map_g, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.g16, 64, tiles * 64, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B)) != LITE3R_OK) return st;
   AttnParams p;
-  p.q_codes = a.q_codes;
   p.q_scales = a.q_scales;
   p.k_scales = a.k_scales;
   p.crit_idx = a.crit_idx;
@@ -643,6 +715,7 @@ lite3r_status launch(const AttentionLaunch& a, cudaStream_t stream) {
   p.k_crit = a.k_crit;
   p.k_marg = a.k_marg;
   p.phi = a.phi;
+  p.out_dtype = a.out_dtype;
   p.status = a.device_status;
   st = record_cuda(cudaFuncSetAttribute(attention_kernel<BS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         static_cast<int>(kSmemBytes)));

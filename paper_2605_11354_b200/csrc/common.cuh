@@ -80,7 +80,8 @@ struct ForwardArgs {
   lite3r_shape s;
   int phi;
   lite3r_plan plan;
-  float* out;
+  void* out;
+  int out_dtype;
   long long out_stride_b, out_stride_h, out_stride_n;
   void* workspace;
   size_t workspace_bytes;
@@ -98,7 +99,8 @@ struct AttentionLaunch {
   const float* zeta;          // [tiles][64]
   const int* crit_idx;
   int k_crit, k_marg, phi;
-  float* out;
+  void* out;
+  int out_dtype;  // lite3r_dtype of the output
   long long out_stride_b, out_stride_h, out_stride_n;
   int* device_status;
 };

@@ -130,6 +130,7 @@ lite3r_status run_forward(const ForwardArgs& a, int phases, cudaStream_t stream)
   att.k_marg = a.plan.k_marg;
   att.phi = a.phi;
   att.out = a.out;
+  att.out_dtype = a.out_dtype;
   att.out_stride_b = a.out_stride_b;
   att.out_stride_h = a.out_stride_h;
   att.out_stride_n = a.out_stride_n;

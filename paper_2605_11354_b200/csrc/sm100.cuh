@@ -60,9 +60,8 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 // backoff_ns > 0 makes the thread sleep between polls: for single-thread roles whose waits are long, so that their
 // polling does not take issue slots from the working warps.
 constexpr uint64_t kWaitLimitNs = 1000000000ull;  // 1 s
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                          int code, uint32_t backoff_ns = 0, uint64_t limit_ns = kWaitLimitNs) {
-  if (mbar_try_wait(bar, parity)) return true;
+__device__ __forceinline__ bool mbar_wait_loop(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                               int code, uint32_t backoff_ns, uint64_t limit_ns) {
   const uint64_t t0 = global_timer_ns();
   uint32_t polls = 0;
   while (true) {
@@ -81,6 +80,22 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
       }
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          int code, uint32_t backoff_ns = 0, uint64_t limit_ns = kWaitLimitNs) {
+  if (mbar_test(bar, parity)) return true;
+  return mbar_wait_loop(bar, parity, abort_flag, status, code, backoff_ns, limit_ns);
+}
+// The same wait with its polling loop in a function of its own (not inlined): a wait that succeeds at once costs the
+// caller two instructions, which keeps a hot loop with several waits small enough for the instruction caches.
+static __device__ __noinline__ bool mbar_wait_loop_far(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                       int* status, int code) {
+  return mbar_wait_loop(bar, parity, abort_flag, status, code, 0, kWaitLimitNs);
+}
+__device__ __forceinline__ bool mbar_wait_far(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                              int code) {
+  if (mbar_test(bar, parity)) return true;
+  return mbar_wait_loop_far(bar, parity, abort_flag, status, code);
 }
 
 // Bounded idling for a single-thread role that polls several barriers without blocking on any of them: call
@@ -178,6 +193,26 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]), "r"(taddr)
       : "memory");
 }
+// 16 consecutive 32-bit columns of the thread's own TMEM lane.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15};"
+      ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(taddr)
+      : "memory");
+}
+// Register budget of the calling warpgroup (all four warps must execute it; count a multiple of 8).
+template <int N> __device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 
 // ------------------------------------------------------------------------------------------------ descriptors
 // Shared-memory operand descriptor (64-bit): start address, leading / stride byte offsets (all >> 4), descriptor
