@@ -524,8 +524,10 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     // denominator phi(q) . zeta_i on the side; computed in registers while the last P V products are still running.
     // The query row comes from the Q tile in shared memory (64-byte rows, 64B swizzle: 16-byte chunk c of row r sits at
     // chunk c ^ ((r >> 1) & 3)).  Every Q K^T product has completed once both warpgroups are here, which the issuer
-    // of the linear product checks through phi_full; the operand goes to K stages 2 and 3, which this warpgroup's own
-    // steps and, by the order of the products, all earlier ones no longer read.
+    // of the linear product checks through phi_full; the operand goes to K stages 2 and 3.
+    // The epilogue's loops over 16-column chunks are deliberately NOT unrolled: the kernel's code has to stay within
+    // the instruction cache of an SM, which its fully unrolled form exceeded several times over (the kernel was then
+    // bound by instruction fetch from the GPC-level cache, not by any arithmetic unit).
     float den = 0.f;
     const int swz = p_row & 7;
     if (ok && p.k_marg > 0) {
@@ -534,12 +536,10 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       for (int u = max(0, steps - 2); u < steps && ok; ++u)
         ok = mbar_wait_far(&bars->k_free[u % kStages], (u / kStages) & 1, abort_flag, p.status, 310);
       const uint8_t* qrow = smem + kOffQ + p_row * 64;
-      const float4* zeta = reinterpret_cast<const float4*>(smem + kOffZeta + hf * 256 + w * 128);
       const int qswz = (p_row >> 1) & 3;
-      float e[32];
       float mxq[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-      for (int c4 = 0; c4 < 4; ++c4) {
+#pragma unroll 1
+      for (int c4 = 0; c4 < 4; ++c4) {  // row maximum over the 64 components
         const uint4 raw = *reinterpret_cast<const uint4*>(qrow + ((c4 ^ qswz) << 4));
         const uint32_t words[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
@@ -547,39 +547,46 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           float fv[4];
           e4m3x4_to_float(words[xw], fv);
 #pragma unroll
-          for (int y = 0; y < 4; ++y) {
-            mxq[y] = fmaxf(mxq[y], fv[y]);
-            if ((c4 >> 1) == w) e[(c4 & 1) * 16 + xw * 4 + y] = fv[y];
-          }
+          for (int y = 0; y < 4; ++y) mxq[y] = fmaxf(mxq[y], fv[y]);
         }
       }
       const float mx = fmaxf(fmaxf(mxq[0], mxq[1]), fmaxf(mxq[2], mxq[3]));
       const float cq = sq * kLog2e, shift = mx * cq;  // sq > 0 commutes with max
       uint8_t* const phirow = smem + kOffPhi + p_row * 128;
       float den4[4] = {0.f, 0.f, 0.f, 0.f};
+      const bool phi_softmax = p.phi == LITE3R_PHI_SOFTMAX;
+#pragma unroll 1
+      for (int cc = 0; cc < 2; ++cc) {  // this warpgroup's two chunks of 16 components
+        const int c4 = 2 * w + cc;
+        const uint4 raw = *reinterpret_cast<const uint4*>(qrow + ((c4 ^ qswz) << 4));
+        const uint32_t words[4] = {raw.x, raw.y, raw.z, raw.w};
+        const float4* zeta = reinterpret_cast<const float4*>(smem + kOffZeta + hf * 256 + c4 * 64);
+        uint32_t pk8[8];
 #pragma unroll
-      for (int ch = 0; ch < 4; ++ch) {  // 16-byte chunk = 8 columns
-        uint32_t pk4[4];
-        const float4 za = zeta[2 * ch], zb = zeta[2 * ch + 1];
-        const float zz[8] = {za.x, za.y, za.z, za.w, zb.x, zb.y, zb.z, zb.w};
+        for (int xw = 0; xw < 4; ++xw) {
+          float fv[4];
+          e4m3x4_to_float(words[xw], fv);
+          const float4 z = zeta[xw];
+          const float zz[4] = {z.x, z.y, z.z, z.w};
 #pragma unroll
-        for (int y = 0; y < 8; y += 2) {
-          const int d = ch * 8 + y;
-          float e0, e1;
-          if (p.phi == LITE3R_PHI_SOFTMAX) {  // the softmax normaliser cancels in the ratio
-            e0 = ex2(fmaf(e[d], cq, -shift));
-            e1 = ex2(fmaf(e[d + 1], cq, -shift));
-          } else {
-            e0 = e[d] > 0.f ? fmaf(e[d], sq, 1.f) : ex2(e[d] * cq);
-            e1 = e[d + 1] > 0.f ? fmaf(e[d + 1], sq, 1.f) : ex2(e[d + 1] * cq);
+          for (int y = 0; y < 4; y += 2) {
+            float e0, e1;
+            if (phi_softmax) {  // the softmax normaliser cancels in the ratio
+              e0 = ex2(fmaf(fv[y], cq, -shift));
+              e1 = ex2(fmaf(fv[y + 1], cq, -shift));
+            } else {
+              e0 = fv[y] > 0.f ? fmaf(fv[y], sq, 1.f) : ex2(fv[y] * cq);
+              e1 = fv[y + 1] > 0.f ? fmaf(fv[y + 1], sq, 1.f) : ex2(fv[y + 1] * cq);
+            }
+            const uint32_t pk = pack_bf162(e0, e1);
+            pk8[xw * 2 + (y >> 1)] = pk;
+            // the denominator uses the same rounded values as the MMA's numerator
+            den4[y] = fmaf(__uint_as_float(pk << 16), zz[y], den4[y]);
+            den4[y + 1] = fmaf(__uint_as_float(pk & 0xFFFF0000u), zz[y + 1], den4[y + 1]);
           }
-          const uint32_t pk = pack_bf162(e0, e1);
-          pk4[y >> 1] = pk;
-          // the denominator uses the same rounded values as the MMA's numerator
-          den4[y >> 1] = fmaf(__uint_as_float(pk << 16), zz[y], den4[y >> 1]);
-          den4[y >> 1] = fmaf(__uint_as_float(pk & 0xFFFF0000u), zz[y + 1], den4[y >> 1]);
         }
-        *reinterpret_cast<uint4*>(phirow + (((w * 4 + ch) ^ swz) << 4)) = make_uint4(pk4[0], pk4[1], pk4[2], pk4[3]);
+        *reinterpret_cast<uint4*>(phirow + (((c4 * 2) ^ swz) << 4)) = make_uint4(pk8[0], pk8[1], pk8[2], pk8[3]);
+        *reinterpret_cast<uint4*>(phirow + (((c4 * 2 + 1) ^ swz) << 4)) = make_uint4(pk8[4], pk8[5], pk8[6], pk8[7]);
       }
       den = (den4[0] + den4[1]) + (den4[2] + den4[3]);
       fence_proxy_async_smem();
@@ -619,63 +626,66 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       // swizzled by the row so that neither these writes nor the row-wise reads below conflict; then each store
       // instruction of the warp writes whole half rows (fp32: four rows x 128 bytes, 16-bit: eight rows x 64 bytes).
       const bool wide = p.out_dtype == LITE3R_F32;
+      const bool to_bf16 = p.out_dtype == LITE3R_BF16;
       const uint32_t row_bytes = wide ? 256u : 128u;
       uint8_t* const orow = smem + kOffOut + p_row * row_bytes;
-      float acc[32];
-      uint32_t v[32];
-      if (steps > 0) {
-        tmem_ld32(o_addr + w * 32, v);
-        tmem_wait_ld();
+#pragma unroll 1
+      for (int cc = 0; cc < 2; ++cc) {  // 16 columns at a time
+        float acc[16];
+        uint32_t v[16];
+        if (steps > 0) {
+          tmem_ld16(o_addr + w * 32 + cc * 16, v);
+          tmem_wait_ld();
 #pragma unroll
-        for (int k = 0; k < 32; ++k) acc[k] = __uint_as_float(v[k]) * inv_l;
-      } else {
+          for (int k = 0; k < 16; ++k) acc[k] = __uint_as_float(v[k]) * inv_l;
+        } else {
 #pragma unroll
-        for (int k = 0; k < 32; ++k) acc[k] = 0.f;
-      }
-      if (p.k_marg > 0) {
-        tmem_ld32(lane_addr + kColL + w * 32, v);
-        tmem_wait_ld();
+          for (int k = 0; k < 16; ++k) acc[k] = 0.f;
+        }
+        if (p.k_marg > 0) {
+          tmem_ld16(lane_addr + kColL + w * 32 + cc * 16, v);
+          tmem_wait_ld();
 #pragma unroll
-        for (int k = 0; k < 32; ++k) acc[k] = fmaf(__uint_as_float(v[k]), l_scale, acc[k]);
-      }
-      if (wide) {
+          for (int k = 0; k < 16; ++k) acc[k] = fmaf(__uint_as_float(v[k]), l_scale, acc[k]);
+        }
+        if (wide) {
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch)
-          *reinterpret_cast<float4*>(orow + (((w * 8 + ch) ^ swz) << 4)) =
-              make_float4(acc[4 * ch], acc[4 * ch + 1], acc[4 * ch + 2], acc[4 * ch + 3]);
-      } else {
+          for (int ch = 0; ch < 4; ++ch)
+            *reinterpret_cast<float4*>(orow + (((w * 8 + cc * 4 + ch) ^ swz) << 4)) =
+                make_float4(acc[4 * ch], acc[4 * ch + 1], acc[4 * ch + 2], acc[4 * ch + 3]);
+        } else {
 #pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
-          uint32_t pk[4];
+          for (int ch = 0; ch < 2; ++ch) {
+            uint32_t pk[4];
 #pragma unroll
-          for (int y = 0; y < 4; ++y)
-            pk[y] = p.out_dtype == LITE3R_BF16 ? pack_bf162(acc[8 * ch + 2 * y], acc[8 * ch + 2 * y + 1])
-                                                : pack_half2(acc[8 * ch + 2 * y], acc[8 * ch + 2 * y + 1]);
-          *reinterpret_cast<uint4*>(orow + (((w * 4 + ch) ^ swz) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            for (int y = 0; y < 4; ++y)
+              pk[y] = to_bf16 ? pack_bf162(acc[8 * ch + 2 * y], acc[8 * ch + 2 * y + 1])
+                              : pack_half2(acc[8 * ch + 2 * y], acc[8 * ch + 2 * y + 1]);
+            *reinterpret_cast<uint4*>(orow + (((w * 4 + cc * 2 + ch) ^ swz) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          }
         }
       }
       __syncwarp();
       const int chunk_shift = wide ? 3 : 2;       // 8 or 4 chunks of 16 bytes per half row
       const int ch = lane & ((1 << chunk_shift) - 1);
       const int half_chunks = 1 << chunk_shift;
+      const int rows_per_pass = 32 >> chunk_shift;  // 4 or 8
       const uint32_t elem = wide ? 4u : 2u;
       uint8_t* const out_bh = static_cast<uint8_t*>(p.out) +
                               (static_cast<long long>(bb) * p.out_stride_b + static_cast<long long>(h) * p.out_stride_h) * elem +
-                              w * 32 * elem;
+                              w * 32 * elem + ch * 16;
       const long long row_pitch = p.out_stride_n * static_cast<long long>(elem);
-#pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        // fp32: pass k covers rows 4k .. 4k+3; 16-bit: rows 8k .. 8k+7, so only k < 4 run
-        if (!wide && k >= 4) break;
-        const int r = wide ? 4 * k + (lane >> 3) : 8 * k + (lane >> 2);  // row of this warp's block: thread r computed it
+      const bool second_block_is_copy = kPair && i_q[1] == i_q[0];
+#pragma unroll 1
+      for (int r = lane >> chunk_shift; r < 32; r += rows_per_pass) {  // row of this warp's block: thread r computed it
         const int r_hf = kPair ? (r >> 4) : 0;
         const int r_in_block = kPair ? quarter * 16 + (r & 15) : quarter * 32 + r;
         const int r_p = kPair ? r_hf * 64 + r_in_block : r_in_block;
         const int r_token = i_q[r_hf] * BS + r_in_block;
         const uint4 val = *reinterpret_cast<const uint4*>(smem + kOffOut + r_p * row_bytes +
                                                           (((w * half_chunks + ch) ^ (r_p & 7)) << 4));
-        if (r_token < p.tokens && (!kPair || r_hf == 0 || i_q[1] != i_q[0]))
-          *reinterpret_cast<uint4*>(out_bh + r_token * row_pitch + ch * 16) = val;
+        if (r_token < p.tokens && !(second_block_is_copy && r_hf == 1))
+          *reinterpret_cast<uint4*>(out_bh + r_token * row_pitch) = val;
       }
     }
   }
