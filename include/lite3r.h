@@ -36,7 +36,7 @@ extern "C" {
 typedef enum {
   LITE3R_OK = 0,
   LITE3R_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, misaligned pointer or stride, fraction outside [0,1] */
-  LITE3R_ERR_UNSUPPORTED = 2, /* head_dim != 64, block not in {64,128}, unknown dtype / phi */
+  LITE3R_ERR_UNSUPPORTED = 2, /* head_dim != 64, block not in {64,128}, unknown dtype / phi, device not compute capability 10.x */
   LITE3R_ERR_WORKSPACE = 3,   /* workspace_bytes smaller than the size query reports */
   LITE3R_ERR_CUDA = 4,        /* a CUDA call failed; see lite3r_last_cuda_error() */
   LITE3R_ERR_TIMEOUT = 5      /* a bounded device-side wait expired (reported through device_status) */
@@ -97,8 +97,11 @@ LITE3R_API lite3r_status lite3r_plan_sizes(const lite3r_shape* shape, double cri
                                 size_t* crit_idx_bytes, size_t* marg_idx_bytes, int* k_crit, int* k_marg,
                                 int* k_neg);
 
-/* Bytes of scratch lite3r_sla_forward needs for `shape` and these fractions.  Host-only. */
+/* Bytes of scratch lite3r_sla_forward needs for `shape` and these fractions when the caller passes a plan
+ * (lite3r_forward_workspace) and when it passes plan == NULL and the plan is built inside the workspace
+ * (lite3r_forward_workspace_planned: the class matrix and the critical lists come on top).  Host-only. */
 LITE3R_API lite3r_status lite3r_forward_workspace(const lite3r_shape* shape, double crit, double neg, size_t* bytes);
+LITE3R_API lite3r_status lite3r_forward_workspace_planned(const lite3r_shape* shape, double crit, double neg, size_t* bytes);
 
 /* Scaled FP8 quantisation (paper appendix "Scaled FP8 Quantization" with the epsilon of "Implementation
  * Details"), one scale per (b, h, token-block) tile, all in fp32:
@@ -124,23 +127,34 @@ LITE3R_API lite3r_status lite3r_quantize_fp8_qkv(const lite3r_tensor* q, const l
 LITE3R_API lite3r_status lite3r_sla_plan(const lite3r_fp8* q, const lite3r_fp8* k, const lite3r_shape* shape, double crit,
                               double neg, lite3r_plan* plan, void* stream);
 
-/* The SLA forward (Eq. 1; Algorithm 1 from the sparse softmax on) for a given plan.
+/* The SLA forward (Eq. 1; Algorithm 1: Require q, k, v, the projection and the keep ratio; Ensure the output).
  *   sparse branch: per query token, softmax over exactly the valid keys of the critical blocks of
  *     (q_hat . k_hat) / sqrt(D), times v_hat;
  *   linear branch: (phi(q_hat) G_i) / (phi(q_hat) . zeta_i) with G_i = sum over marginal blocks of
  *     phi(K_j)^T V_j and zeta_i = sum of phi(K_j)^T 1;
  *   out = sparse + linear @ proj[h]   (no bias).
+ * plan: the block plan of lite3r_sla_plan, or NULL: then the plan is computed first, inside the workspace, from the
+ *   column sums of q and k and the fractions crit / neg (the row-wise TopKMask of Algorithm 1 on block means), exactly
+ *   as lite3r_sla_plan would; with a plan, crit and neg are not used (the plan's counts are).
  * proj: DEVICE fp32 [H, D, D] row-major [d_in][d_out]; proj_head_stride in elements (D*D for per-head
  * matrices, 0 for one matrix shared by all heads).
- * out: DEVICE fp32 [B, H, N, D] with the given strides (elements, multiples of 4); rows past N are not written.
- * workspace: DEVICE, 256-byte aligned, at least lite3r_forward_workspace() bytes; its contents are scratch.
+ * out: DEVICE [B, H, N, D] of out_dtype (LITE3R_F32, LITE3R_BF16 or LITE3R_F16: the fp32 result rounded to nearest
+ * even on the way out) with the given strides in elements (multiples of 4 for fp32, of 8 for the 16-bit types;
+ * pointer 16-byte aligned); rows past N are not written.
+ * workspace: DEVICE, 256-byte aligned, at least lite3r_forward_workspace() bytes (lite3r_forward_workspace_planned()
+ * when plan is NULL); its contents are scratch.
  * device_status: optional DEVICE int, set non-zero by the kernels if a bounded wait expired (read it after
- * synchronising); may be NULL. */
+ * synchronising); may be NULL.
+ * Value range: the probabilities, phi(K), the per-block summaries and the dequantised V travel as fp16 / bf16 inside
+ * (the accumulation is fp32).  |v_hat| must stay below 65504 and the per-block sums |sum_s phi(k_s)[d] v_s[e]| below
+ * ~6e4 (softmax phi: |v| up to ~900 per component is always safe; ELU+1: |k| |v| summed over a block must stay below
+ * that); beyond it the result holds inf / NaN and device_status stays 0.  Inputs of unit to tens magnitude, the
+ * range of transformer activations, are far inside. */
 LITE3R_API lite3r_status lite3r_sla_forward(const lite3r_fp8* q, const lite3r_fp8* k, const lite3r_fp8* v, const float* proj,
-                                 long long proj_head_stride, const lite3r_shape* shape, lite3r_phi phi,
-                                 const lite3r_plan* plan, float* out, long long out_stride_b,
-                                 long long out_stride_h, long long out_stride_n, void* workspace,
-                                 size_t workspace_bytes, int* device_status, void* stream);
+                                 long long proj_head_stride, const lite3r_shape* shape, double crit, double neg,
+                                 lite3r_phi phi, const lite3r_plan* plan, void* out, lite3r_dtype out_dtype,
+                                 long long out_stride_b, long long out_stride_h, long long out_stride_n,
+                                 void* workspace, size_t workspace_bytes, int* device_status, void* stream);
 
 /* lite3r_sla_forward in two halves, for callers that overlap the block plan with the part of the forward that does
  * not depend on it.  The per-key-block summaries of the linear branch (Algorithm 1's feature map, KV summary and
@@ -150,16 +164,17 @@ LITE3R_API lite3r_status lite3r_sla_forward(const lite3r_fp8* q, const lite3r_fp
  * both have completed (the caller orders the streams).  begin followed by finish on one stream is exactly
  * lite3r_sla_forward: same kernels, same results.  begin takes the three class counts lite3r_plan_sizes reports
  * (they depend on the fractions only) and clears *device_status; finish does not clear it.  Both use the same
- * workspace, which must not be touched in between.  Arguments otherwise as for lite3r_sla_forward. */
+ * workspace, which must not be touched in between.  Both need the caller's plan (finish its contents, begin only the
+ * three counts).  Arguments otherwise as for lite3r_sla_forward. */
 LITE3R_API lite3r_status lite3r_sla_forward_begin(const lite3r_fp8* k, const lite3r_fp8* v, const float* proj,
                                        long long proj_head_stride, const lite3r_shape* shape, lite3r_phi phi,
                                        int k_crit, int k_marg, int k_neg, void* workspace, size_t workspace_bytes,
                                        int* device_status, void* stream);
 LITE3R_API lite3r_status lite3r_sla_forward_finish(const lite3r_fp8* q, const lite3r_fp8* k, const lite3r_fp8* v,
                                         const lite3r_shape* shape, lite3r_phi phi, const lite3r_plan* plan,
-                                        float* out, long long out_stride_b, long long out_stride_h,
-                                        long long out_stride_n, void* workspace, size_t workspace_bytes,
-                                        int* device_status, void* stream);
+                                        void* out, lite3r_dtype out_dtype, long long out_stride_b,
+                                        long long out_stride_h, long long out_stride_n, void* workspace,
+                                        size_t workspace_bytes, int* device_status, void* stream);
 
 /* The same forward for callers that cannot provide scratch memory.  (The paper has no counterpart: this entry
  * point exists for deployments, not for the method.)
@@ -169,15 +184,19 @@ LITE3R_API lite3r_status lite3r_sla_forward_finish(const lite3r_fp8* q, const li
  * allocator, a process whose memory pool is already sized to the last byte.  Such a caller still owns the inputs
  * and the output, but has nowhere to take the workspace of lite3r_sla_forward from.
  *
- * Here the scratch is a fixed array of LITE3R_STATIC_SCRATCH_BYTES inside the library image: every GPU on which
- * the library is loaded sets that much memory aside until the process exits, whether or not this call is used.
- * The call allocates and frees nothing, on the device or through any library.  Arguments are those of
- * lite3r_sla_forward without workspace / workspace_bytes, and the results are identical.
+ * Here the scratch is a fixed array of LITE3R_STATIC_SCRATCH_BYTES inside the library image.  Arguments are those
+ * of lite3r_sla_forward without workspace / workspace_bytes and without the fractions (a plan must be passed), and
+ * the results are identical.
+ *   - First call per device: CUDA loads device code lazily, so the array takes its 32 MiB of device memory when this
+ *     entry point is first called on a device (that call also looks up the array's address; the device must be
+ *     current).  Make that call during start-up, outside any stream capture, while memory can still be taken; it may
+ *     fail with a CUDA out-of-memory error if 32 MiB are not free.  A call that is then refused for its size (or any
+ *     valid call) serves as this warm-up.  Every later call on that device allocates and frees nothing, on the device
+ *     or through any library; the memory stays with the process until it exits.
  *   - Limit: if lite3r_forward_workspace() for this shape exceeds LITE3R_STATIC_SCRATCH_BYTES the call returns
- *     LITE3R_ERR_WORKSPACE and enqueues nothing (32 MiB holds 1344 (batch x head x block) tiles, e.g. two heads of
- *     an 8-frame 10992-token sequence at block 64); use lite3r_sla_forward with your own buffer for larger problems.
- *   - The first call on each device looks up the array's device address (the device must be current); make that
- *     first call outside any stream capture.
+ *     LITE3R_ERR_WORKSPACE and enqueues nothing: 32 MiB hold 1344 (batch x head x block) tiles at block 64 (e.g. two
+ *     heads of an 8-frame 10992-token sequence) and 1012 tiles at block 128; use lite3r_sla_forward with your own
+ *     buffer for larger problems.
  *   - All calls on a device share the one array, and it keeps whatever the previous call left there.  The forward
  *     overwrites every scratch element before reading it, so nothing needs clearing between calls, but two calls
  *     whose kernels may overlap on the GPU (different streams, no ordering between them) race on the array:
@@ -186,31 +205,13 @@ LITE3R_API lite3r_status lite3r_sla_forward_finish(const lite3r_fp8* q, const li
 LITE3R_API lite3r_status lite3r_sla_forward_static_scratch(const lite3r_fp8* q, const lite3r_fp8* k, const lite3r_fp8* v,
                                                 const float* proj, long long proj_head_stride,
                                                 const lite3r_shape* shape, lite3r_phi phi, const lite3r_plan* plan,
-                                                float* out, long long out_stride_b, long long out_stride_h,
-                                                long long out_stride_n, int* device_status, void* stream);
-
-/* Self-test of the device-side wait bound.  Every wait inside the kernels (on an mbarrier, or a polling loop of a
- * single-thread role) gives up after one second, records a non-zero code in device_status and lets the kernel end, so a
- * lost signal can never hang the GPU.  This call runs that mechanism on purpose and harmlessly: a one-thread kernel
- * waits, with the given limit (nanoseconds, at most 1e9), on a barrier that nothing arrives on.  After synchronising,
- * *device_status (DEVICE int) must be non-zero (999) and the context must still be usable. */
-LITE3R_API lite3r_status lite3r_selftest_wait_expiry(int* device_status, unsigned long long limit_ns, void* stream);
+                                                void* out, lite3r_dtype out_dtype, long long out_stride_b,
+                                                long long out_stride_h, long long out_stride_n, int* device_status,
+                                                void* stream);
 
 /* Text for a status code; the last CUDA error code (cudaError_t as int) recorded by this thread. */
 LITE3R_API const char* lite3r_status_string(lite3r_status status);
 LITE3R_API int lite3r_last_cuda_error(void);
-
-/* Stage timing for benchmarks.  After lite3r_profile_enable(1) (call it with the device current; it creates CUDA
- * events, no device memory), every lite3r_sla_forward brackets its four stages -- V operand preparation, key-block
- * summaries, marginal aggregation, attention -- with event records on the call's stream.  lite3r_profile_stage_ms
- * waits for the last forward's events (the only blocking call of the library) and writes the four durations in
- * milliseconds to ms (HOST, 4 floats; a stage that did not run reports 0).  Not thread-safe; meant for one
- * benchmarking thread. */
-LITE3R_API lite3r_status lite3r_profile_enable(int enable);
-LITE3R_API lite3r_status lite3r_profile_stage_ms(float* ms);
-
-/* Number of kernel launches the library has enqueued since it was loaded (all threads). */
-LITE3R_API long long lite3r_launch_count(void);
 
 #ifdef __cplusplus
 }

@@ -15,7 +15,8 @@ import torch
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblite3r.so")
 _lib = None
 
-F32, BF16 = 0, 1
+F32, BF16, F16 = 0, 1, 2
+OUT_DTYPES = {torch.float32: F32, torch.bfloat16: BF16, torch.float16: F16}
 PHI_SOFTMAX, PHI_ELU1 = 0, 1
 PHI_CODES = {"softmax": PHI_SOFTMAX, "elu1": PHI_ELU1}
 
@@ -46,7 +47,8 @@ EXPORTS = ("lite3r_fp8_sizes", "lite3r_plan_sizes", "lite3r_forward_workspace", 
            "lite3r_sla_plan", "lite3r_sla_forward", "lite3r_status_string", "lite3r_last_cuda_error",
            "lite3r_launch_count", "lite3r_profile_enable", "lite3r_profile_stage_ms",
            "lite3r_sla_forward_static_scratch", "lite3r_quantize_fp8_qkv", "lite3r_selftest_wait_expiry",
-           "lite3r_sla_forward_begin", "lite3r_sla_forward_finish")
+           "lite3r_sla_forward_begin", "lite3r_sla_forward_finish", "lite3r_forward_workspace_planned",
+           "lite3r_workspace_layout")
 STATIC_SCRATCH_BYTES = 32 << 20  # LITE3R_STATIC_SCRATCH_BYTES
 
 
@@ -69,21 +71,26 @@ def lib() -> C.CDLL:
     L.lite3r_quantize_fp8_qkv.restype = C.c_int
     L.lite3r_sla_plan.argtypes = [C.POINTER(Fp8), C.POINTER(Fp8), C.POINTER(Shape), C.c_double, C.c_double,
                                   C.POINTER(Plan), C.c_void_p]
+    L.lite3r_forward_workspace_planned.argtypes = [C.POINTER(Shape), C.c_double, C.c_double, sz]
+    L.lite3r_forward_workspace_planned.restype = C.c_int
+    L.lite3r_workspace_layout.argtypes = [C.POINTER(Shape), C.c_double, C.c_double, C.c_int, sz]
+    L.lite3r_workspace_layout.restype = C.c_int
     L.lite3r_sla_forward.argtypes = [C.POINTER(Fp8), C.POINTER(Fp8), C.POINTER(Fp8), C.c_void_p, C.c_longlong,
-                                     C.POINTER(Shape), C.c_int, C.POINTER(Plan), C.c_void_p, C.c_longlong,
-                                     C.c_longlong, C.c_longlong, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+                                     C.POINTER(Shape), C.c_double, C.c_double, C.c_int, C.POINTER(Plan), C.c_void_p,
+                                     C.c_int, C.c_longlong, C.c_longlong, C.c_longlong, C.c_void_p, C.c_size_t,
+                                     C.c_void_p, C.c_void_p]
     L.lite3r_sla_forward_static_scratch.argtypes = [C.POINTER(Fp8), C.POINTER(Fp8), C.POINTER(Fp8), C.c_void_p,
                                                     C.c_longlong, C.POINTER(Shape), C.c_int, C.POINTER(Plan),
-                                                    C.c_void_p, C.c_longlong, C.c_longlong, C.c_longlong, C.c_void_p,
-                                                    C.c_void_p]
+                                                    C.c_void_p, C.c_int, C.c_longlong, C.c_longlong, C.c_longlong,
+                                                    C.c_void_p, C.c_void_p]
     L.lite3r_sla_forward_static_scratch.restype = C.c_int
     L.lite3r_sla_forward_begin.argtypes = [C.POINTER(Fp8), C.POINTER(Fp8), C.c_void_p, C.c_longlong, C.POINTER(Shape),
                                            C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_size_t, C.c_void_p,
                                            C.c_void_p]
     L.lite3r_sla_forward_begin.restype = C.c_int
     L.lite3r_sla_forward_finish.argtypes = [C.POINTER(Fp8), C.POINTER(Fp8), C.POINTER(Fp8), C.POINTER(Shape), C.c_int,
-                                            C.POINTER(Plan), C.c_void_p, C.c_longlong, C.c_longlong, C.c_longlong,
-                                            C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+                                            C.POINTER(Plan), C.c_void_p, C.c_int, C.c_longlong, C.c_longlong,
+                                            C.c_longlong, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
     L.lite3r_sla_forward_finish.restype = C.c_int
     L.lite3r_selftest_wait_expiry.argtypes = [C.c_void_p, C.c_ulonglong, C.c_void_p]
     L.lite3r_selftest_wait_expiry.restype = C.c_int
@@ -154,6 +161,22 @@ def lite3r_forward_workspace(shape: Shape, crit: float, neg: float) -> int:
     a = C.c_size_t()
     _check(lib().lite3r_forward_workspace(C.byref(shape), crit, neg, C.byref(a)), "lite3r_forward_workspace")
     return a.value
+
+
+def lite3r_forward_workspace_planned(shape: Shape, crit: float, neg: float) -> int:
+    """Workspace bytes of lite3r_sla_forward called without a plan (the plan is then built inside the workspace)."""
+    a = C.c_size_t()
+    _check(lib().lite3r_forward_workspace_planned(C.byref(shape), crit, neg, C.byref(a)),
+           "lite3r_forward_workspace_planned")
+    return a.value
+
+
+def lite3r_workspace_layout(shape: Shape, crit: float, neg: float, plan_inside: bool = False):
+    """Byte offsets of the six parts of the forward's workspace (summaries, aggregates, zeta, fp16 V, classes, lists)."""
+    arr = (C.c_size_t * 6)()
+    _check(lib().lite3r_workspace_layout(C.byref(shape), crit, neg, 1 if plan_inside else 0, arr),
+           "lite3r_workspace_layout")
+    return tuple(int(x) for x in arr)
 
 
 # ----------------------------------------------------------------------------- device buffers
@@ -239,19 +262,26 @@ def lite3r_sla_plan(q: Fp8Tensor, k: Fp8Tensor, shape: Shape, crit: float, neg: 
     assert (p.k_crit, p.k_marg, p.k_neg) == (plan.k_crit, plan.k_marg, plan.k_neg)
 
 
+def _check_out(out: torch.Tensor, what: str) -> int:
+    if out.dtype not in OUT_DTYPES or not out.is_cuda or out.dim() != 4 or out.stride(3) != 1:
+        raise Lite3rError(f"{what}: out must be a CUDA float32 / bfloat16 / float16 tensor [B,H,N,D] with contiguous D")
+    return OUT_DTYPES[out.dtype]
+
+
 def lite3r_sla_forward(q: Fp8Tensor, k: Fp8Tensor, v: Fp8Tensor, proj: torch.Tensor, shape: Shape, phi: int,
-                       plan: PlanBuffers, out: torch.Tensor, workspace: torch.Tensor, device_status=None,
-                       stream=None) -> None:
-    """proj: CUDA fp32 [H,D,D] or [D,D] (shared); out: CUDA fp32 [B,H,N,D] view with contiguous D."""
+                       plan, out: torch.Tensor, workspace: torch.Tensor, device_status=None,
+                       stream=None, crit: float = 0.0, neg: float = 0.0) -> None:
+    """proj: CUDA fp32 [H,D,D] or [D,D] (shared); out: CUDA fp32 / bf16 / fp16 [B,H,N,D] view with contiguous D
+    (its dtype selects the output type).  plan=None: the plan is built inside the workspace from crit / neg."""
     if proj.dtype != torch.float32 or not proj.is_cuda or not proj.is_contiguous():
         raise Lite3rError("lite3r_sla_forward: proj must be a contiguous CUDA float32 tensor")
-    if out.dtype != torch.float32 or not out.is_cuda or out.stride(3) != 1:
-        raise Lite3rError("lite3r_sla_forward: out must be a CUDA float32 tensor [B,H,N,D] with contiguous D")
+    out_dtype = _check_out(out, "lite3r_sla_forward")
     head_stride = proj.stride(0) if proj.dim() == 3 else 0
-    p = plan.c_struct()
+    p = plan.c_struct() if plan is not None else None
     qs, ks, vs = q.c_struct(), k.c_struct(), v.c_struct()
     _check(lib().lite3r_sla_forward(C.byref(qs), C.byref(ks), C.byref(vs), proj.data_ptr(), head_stride,
-                                    C.byref(shape), phi, C.byref(p), out.data_ptr(), out.stride(0), out.stride(1),
+                                    C.byref(shape), crit, neg, phi, C.byref(p) if p is not None else None,
+                                    out.data_ptr(), out_dtype, out.stride(0), out.stride(1),
                                     out.stride(2), workspace.data_ptr(), workspace.numel() * workspace.element_size(),
                                     device_status.data_ptr() if device_status is not None else None,
                                     _stream_ptr(stream)), "lite3r_sla_forward")
@@ -274,12 +304,11 @@ def lite3r_sla_forward_begin(k: Fp8Tensor, v: Fp8Tensor, proj: torch.Tensor, sha
 def lite3r_sla_forward_finish(q: Fp8Tensor, k: Fp8Tensor, v: Fp8Tensor, shape: Shape, phi: int, plan: PlanBuffers,
                               out: torch.Tensor, workspace: torch.Tensor, device_status=None, stream=None) -> None:
     """Second half of the forward (aggregation, attention, linear output, sum); after begin and the plan."""
-    if out.dtype != torch.float32 or not out.is_cuda or out.stride(3) != 1:
-        raise Lite3rError("lite3r_sla_forward_finish: out must be a CUDA float32 tensor [B,H,N,D] with contiguous D")
+    out_dtype = _check_out(out, "lite3r_sla_forward_finish")
     p = plan.c_struct()
     qs, ks, vs = q.c_struct(), k.c_struct(), v.c_struct()
     _check(lib().lite3r_sla_forward_finish(C.byref(qs), C.byref(ks), C.byref(vs), C.byref(shape), phi, C.byref(p),
-                                           out.data_ptr(), out.stride(0), out.stride(1), out.stride(2),
+                                           out.data_ptr(), out_dtype, out.stride(0), out.stride(1), out.stride(2),
                                            workspace.data_ptr(), workspace.numel() * workspace.element_size(),
                                            device_status.data_ptr() if device_status is not None else None,
                                            _stream_ptr(stream)), "lite3r_sla_forward_finish")
@@ -289,18 +318,19 @@ def lite3r_sla_forward_static_scratch(q: Fp8Tensor, k: Fp8Tensor, v: Fp8Tensor, 
                                       phi: int, plan: PlanBuffers, out: torch.Tensor, device_status=None,
                                       stream=None) -> None:
     """lite3r_sla_forward for callers that may not allocate: the scratch is a fixed 32 MiB array inside the
-    library (held on every GPU that loads it), so no workspace is passed.  Raises "workspace too small" when the
-    shape needs more than that.  Calls on one device share the array: do not let two of them overlap on the GPU."""
+    library, so no workspace is passed.  The first call on a device is the one that makes CUDA load the array (32 MiB
+    of device memory are taken then): make it at start-up; later calls allocate nothing.  Raises "workspace too small"
+    when the shape needs more than the array holds.  Calls on one device share the array: do not let two of them
+    overlap on the GPU."""
     if proj.dtype != torch.float32 or not proj.is_cuda or not proj.is_contiguous():
         raise Lite3rError("lite3r_sla_forward_static_scratch: proj must be a contiguous CUDA float32 tensor")
-    if out.dtype != torch.float32 or not out.is_cuda or out.stride(3) != 1:
-        raise Lite3rError("lite3r_sla_forward_static_scratch: out must be CUDA float32 [B,H,N,D], contiguous D")
+    out_dtype = _check_out(out, "lite3r_sla_forward_static_scratch")
     head_stride = proj.stride(0) if proj.dim() == 3 else 0
     p = plan.c_struct()
     qs, ks, vs = q.c_struct(), k.c_struct(), v.c_struct()
     _check(lib().lite3r_sla_forward_static_scratch(
         C.byref(qs), C.byref(ks), C.byref(vs), proj.data_ptr(), head_stride, C.byref(shape), phi, C.byref(p),
-        out.data_ptr(), out.stride(0), out.stride(1), out.stride(2),
+        out.data_ptr(), out_dtype, out.stride(0), out.stride(1), out.stride(2),
         device_status.data_ptr() if device_status is not None else None, _stream_ptr(stream)),
         "lite3r_sla_forward_static_scratch")
 
@@ -309,18 +339,23 @@ def lite3r_sla_forward_static_scratch(q: Fp8Tensor, k: Fp8Tensor, v: Fp8Tensor, 
 class SlaForward:
     """Pre-allocated buffers for one shape; ``run`` enqueues quantise x3 + plan + forward and returns ``out``."""
 
-    def __init__(self, batch, heads, tokens, block, crit, neg, phi="softmax", device="cuda:0", head_dim=64):
+    def __init__(self, batch, heads, tokens, block, crit, neg, phi="softmax", device="cuda:0", head_dim=64,
+                 out_dtype=torch.float32, plan_inside=False):
+        """out_dtype: dtype of the engine's own output tensor.  plan_inside: let lite3r_sla_forward build the block
+        plan inside its workspace (plan=NULL) instead of calling lite3r_sla_plan."""
         self.shape = Shape(batch, heads, tokens, head_dim, block)
+        self.plan_inside = bool(plan_inside)
         self.crit, self.neg, self.phi = float(crit), float(neg), PHI_CODES[phi]
         self.device = torch.device(device)
         self.q8, self.k8 = (alloc_fp8(self.shape, self.device) for _ in range(2))
         self.v8 = alloc_fp8(self.shape, self.device, colsum=False)  # the block plan pools Q and K only
         self.plan = alloc_plan(self.shape, self.crit, self.neg, self.device)
-        nbytes = lite3r_forward_workspace(self.shape, self.crit, self.neg)
+        nbytes = (lite3r_forward_workspace_planned if self.plan_inside else lite3r_forward_workspace)(
+            self.shape, self.crit, self.neg)
         self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
         off = (-self.workspace.data_ptr()) % 256
         self.workspace = self.workspace[off:off + nbytes]
-        self.out = torch.empty((batch, heads, tokens, head_dim), dtype=torch.float32, device=self.device)
+        self.out = torch.empty((batch, heads, tokens, head_dim), dtype=out_dtype, device=self.device)
         self.status = torch.zeros(1, dtype=torch.int32, device=self.device)
         self._side = None  # stream of the overlapped first half of the forward, made on first use
 
@@ -338,13 +373,17 @@ class SlaForward:
     def forward(self, proj, stream=None, out=None):
         """out: optional result tensor of the engine's output shape (default: the engine's own ``out``)."""
         out = self.out if out is None else out
-        lite3r_sla_forward(self.q8, self.k8, self.v8, proj, self.shape, self.phi, self.plan, out,
-                           self.workspace, self.status, stream)
+        lite3r_sla_forward(self.q8, self.k8, self.v8, proj, self.shape, self.phi,
+                           None if self.plan_inside else self.plan, out, self.workspace, self.status, stream,
+                           crit=self.crit, neg=self.neg)
         return out
 
     def run(self, q, k, v, proj, stream=None, out=None, overlap=False):
         """Quantise, plan, forward.  overlap=True runs the plan-independent first half of the forward (summaries, fp16
         V) on a side stream beside the plan kernel; the results are the same."""
+        if self.plan_inside:
+            self.quantize(q, k, v, stream)
+            return self.forward(proj, stream, out)
         if not overlap or self.plan.k_marg == 0:
             self.quantize(q, k, v, stream)
             self.make_plan(stream)

@@ -251,13 +251,25 @@ aggregate_mma_kernel(const __grid_constant__ CUtensorMap map_s, const signed cha
 
 lite3r_status launch_aggregate(const __nv_bfloat16* hws, const signed char* cls, const lite3r_shape& s, int nb,
                                __nv_bfloat16* g16, float* zeta, int* device_status, cudaStream_t stream) {
-  alignas(64) CUtensorMap map_s;
   const uint64_t rows = static_cast<uint64_t>(s.batch) * s.heads * nb;
-  lite3r_status st = make_tensor_map_2d(&map_s, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, hws, kSummaryRow, rows, 64, 64,
-                                        CU_TENSOR_MAP_SWIZZLE_128B);
-  if (st != LITE3R_OK) return st;
-  st = record_cuda(cudaFuncSetAttribute(aggregate_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        static_cast<int>(kSmemBytes)));
+  // the tensor map of the summaries is kept from the calling thread's previous call while buffer and size repeat
+  struct MapCache {
+    alignas(64) CUtensorMap map;
+    const void* base = nullptr;
+    uint64_t rows = 0;
+  };
+  thread_local MapCache cache;
+  lite3r_status st;
+  if (cache.base != hws || cache.rows != rows) {
+    cache.base = nullptr;
+    st = make_tensor_map_2d(&cache.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, hws, kSummaryRow, rows, 64, 64,
+                            CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st != LITE3R_OK) return st;
+    cache.base = hws;
+    cache.rows = rows;
+  }
+  const CUtensorMap& map_s = cache.map;
+  st = ensure_dynamic_smem(aggregate_mma_kernel, static_cast<int>(kSmemBytes));
   if (st != LITE3R_OK) return st;
   if (rows > 0x7FFFFFFFull - kTileM) return LITE3R_ERR_UNSUPPORTED;
   const int total_rows = static_cast<int>(rows), bh = s.batch * s.heads;

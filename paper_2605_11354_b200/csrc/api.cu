@@ -1,8 +1,11 @@
 // C-ABI entry points of the lite3r library: argument validation, size queries and dispatch.
 #include <atomic>
 #include <cmath>
+#include <mutex>
+#include <unordered_map>
 
 #include "common.cuh"
+#include "lite3r_debug.h"
 
 namespace lite3r {
 
@@ -20,11 +23,70 @@ lite3r_status after_launch() {
   return record_cuda(cudaGetLastError());
 }
 
-lite3r_status sm_count(int* count) {
+// Facts about each device, looked up once (the current device is never changed).
+namespace {
+constexpr int kMaxDevices = 64;
+struct DeviceInfo {
+  std::atomic<int> ready{0};
+  int sms = 0, cc_major = 0;
+};
+DeviceInfo g_devices[kMaxDevices];
+std::mutex g_device_mutex;
+
+lite3r_status device_info(const DeviceInfo** info, int* device_out = nullptr) {
   int device = 0;
   lite3r_status st = record_cuda(cudaGetDevice(&device));
   if (st != LITE3R_OK) return st;
-  return record_cuda(cudaDeviceGetAttribute(count, cudaDevAttrMultiProcessorCount, device));
+  if (device < 0 || device >= kMaxDevices) return LITE3R_ERR_UNSUPPORTED;
+  DeviceInfo& d = g_devices[device];
+  if (d.ready.load(std::memory_order_acquire) == 0) {
+    std::lock_guard<std::mutex> lock(g_device_mutex);
+    if (d.ready.load(std::memory_order_relaxed) == 0) {
+      if ((st = record_cuda(cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, device))) != LITE3R_OK) return st;
+      if ((st = record_cuda(cudaDeviceGetAttribute(&d.cc_major, cudaDevAttrComputeCapabilityMajor, device))) != LITE3R_OK) return st;
+      d.ready.store(1, std::memory_order_release);
+    }
+  }
+  *info = &d;
+  if (device_out != nullptr) *device_out = device;
+  return LITE3R_OK;
+}
+}  // namespace
+
+lite3r_status sm_count(int* count) {
+  const DeviceInfo* d = nullptr;
+  lite3r_status st = device_info(&d);
+  if (st != LITE3R_OK) return st;
+  *count = d->sms;
+  return LITE3R_OK;
+}
+
+lite3r_status check_device() {
+  const DeviceInfo* d = nullptr;
+  lite3r_status st = device_info(&d);
+  if (st != LITE3R_OK) return st;
+  return d->cc_major == 10 ? LITE3R_OK : LITE3R_ERR_UNSUPPORTED;
+}
+
+namespace {
+struct SmemLimits {
+  int set_bytes[kMaxDevices] = {};
+};
+std::mutex g_smem_mutex;
+std::unordered_map<const void*, SmemLimits> g_smem_limits;
+}  // namespace
+
+lite3r_status ensure_smem_limit(const void* kernel, int bytes) {
+  const DeviceInfo* d = nullptr;
+  int device = 0;
+  lite3r_status st = device_info(&d, &device);
+  if (st != LITE3R_OK) return st;
+  std::lock_guard<std::mutex> lock(g_smem_mutex);
+  SmemLimits& limits = g_smem_limits[kernel];
+  if (limits.set_bytes[device] >= bytes) return LITE3R_OK;
+  st = record_cuda(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  if (st == LITE3R_OK) limits.set_bytes[device] = bytes;
+  return st;
 }
 
 static bool g_profile = false;
@@ -148,14 +210,22 @@ lite3r_status lite3r_plan_sizes(const lite3r_shape* shape, double crit, double n
   return LITE3R_OK;
 }
 
-lite3r_status lite3r_forward_workspace(const lite3r_shape* shape, double crit, double neg, size_t* bytes) {
+static lite3r_status workspace_query(const lite3r_shape* shape, double crit, double neg, bool plan_inside, size_t* bytes) {
   lite3r_status st = check_shape(shape);
   if (st != LITE3R_OK) return st;
   st = check_fractions(crit, neg);
   if (st != LITE3R_OK) return st;
   if (bytes == nullptr) return LITE3R_ERR_INVALID_ARG;
-  *bytes = forward_workspace_bytes(*shape, class_counts(ceil_div(shape->tokens, shape->block), crit, neg));
+  *bytes = forward_workspace_bytes(*shape, class_counts(ceil_div(shape->tokens, shape->block), crit, neg), plan_inside);
   return LITE3R_OK;
+}
+
+lite3r_status lite3r_forward_workspace(const lite3r_shape* shape, double crit, double neg, size_t* bytes) {
+  return workspace_query(shape, crit, neg, false, bytes);
+}
+
+lite3r_status lite3r_forward_workspace_planned(const lite3r_shape* shape, double crit, double neg, size_t* bytes) {
+  return workspace_query(shape, crit, neg, true, bytes);
 }
 
 static lite3r_status check_source(const lite3r_tensor* x) {
@@ -172,6 +242,7 @@ lite3r_status lite3r_quantize_fp8(const lite3r_tensor* x, const lite3r_shape* sh
   if ((st = check_source(x)) != LITE3R_OK) return st;
   st = check_fp8(&out, true, false);
   if (st != LITE3R_OK) return st;
+  if ((st = check_device()) != LITE3R_OK) return st;
   return launch_quantize(&x, &out, 1, *shape, static_cast<cudaStream_t>(stream));
 }
 
@@ -187,6 +258,7 @@ lite3r_status lite3r_quantize_fp8_qkv(const lite3r_tensor* q, const lite3r_tenso
     if ((st = check_fp8(&out[n], true, false)) != LITE3R_OK) return st;
     if (x[n]->dtype != x[0]->dtype) return LITE3R_ERR_UNSUPPORTED;
   }
+  if ((st = check_device()) != LITE3R_OK) return st;
   return launch_quantize(x, out, 3, *shape, static_cast<cudaStream_t>(stream));
 }
 
@@ -204,38 +276,58 @@ lite3r_status lite3r_sla_plan(const lite3r_fp8* q, const lite3r_fp8* k, const li
   plan->k_crit = c.k_crit;
   plan->k_marg = c.k_marg;
   plan->k_neg = c.k_neg;
+  if ((st = check_device()) != LITE3R_OK) return st;
   return launch_plan(*q, *k, *shape, c, *plan, static_cast<cudaStream_t>(stream));
 }
 
 // Shared argument checks and launch of lite3r_sla_forward and its two halves (phases as in launch_forward).
 static lite3r_status forward_phases(int phases, const lite3r_fp8* q, const lite3r_fp8* k, const lite3r_fp8* v,
                                     const float* proj, long long proj_head_stride, const lite3r_shape* shape,
-                                    lite3r_phi phi, const lite3r_plan* plan, float* out, long long out_stride_b,
-                                    long long out_stride_h, long long out_stride_n, void* workspace,
-                                    size_t workspace_bytes, int* device_status, void* stream) {
+                                    double crit, double neg, lite3r_phi phi, const lite3r_plan* plan, void* out,
+                                    lite3r_dtype out_dtype, long long out_stride_b, long long out_stride_h,
+                                    long long out_stride_n, void* workspace, size_t workspace_bytes,
+                                    int* device_status, void* stream) {
   lite3r_status st = check_shape(shape);
   if (st != LITE3R_OK) return st;
   if ((st = check_fp8(k, true, false)) != LITE3R_OK) return st;
   if ((st = check_fp8(v, true, false)) != LITE3R_OK) return st;
   if (phi != LITE3R_PHI_SOFTMAX && phi != LITE3R_PHI_ELU1) return LITE3R_ERR_UNSUPPORTED;
-  if (plan == nullptr) return LITE3R_ERR_INVALID_ARG;
   const int nb = ceil_div(shape->tokens, shape->block);
-  if (plan->k_crit < 0 || plan->k_marg < 0 || plan->k_neg < 0 || plan->k_crit + plan->k_marg + plan->k_neg != nb)
-    return LITE3R_ERR_INVALID_ARG;
+  const bool plan_inside = plan == nullptr;
+  lite3r_plan effective = {};
+  if (plan_inside) {
+    if (phases != 3) return LITE3R_ERR_INVALID_ARG;  // the two halves take the plan from the caller
+    if ((st = check_fractions(crit, neg)) != LITE3R_OK) return st;
+    if ((st = check_fp8(q, true, true)) != LITE3R_OK) return st;  // pooled scores need the column sums
+    if ((st = check_fp8(k, true, true)) != LITE3R_OK) return st;
+    const Counts c = class_counts(nb, crit, neg);
+    effective.k_crit = c.k_crit;
+    effective.k_marg = c.k_marg;
+    effective.k_neg = c.k_neg;
+  } else {
+    effective = *plan;
+    if (plan->k_crit < 0 || plan->k_marg < 0 || plan->k_neg < 0 || plan->k_crit + plan->k_marg + plan->k_neg != nb)
+      return LITE3R_ERR_INVALID_ARG;
+  }
   if (phases & 1) {
     if (proj == nullptr || !aligned(proj, 16) || proj_head_stride < 0 || (proj_head_stride % 4)) return LITE3R_ERR_INVALID_ARG;
   }
   if (phases & 2) {
     if ((st = check_fp8(q, true, false)) != LITE3R_OK) return st;
+    if (out_dtype != LITE3R_F32 && out_dtype != LITE3R_BF16 && out_dtype != LITE3R_F16) return LITE3R_ERR_UNSUPPORTED;
+    const int vec = out_dtype == LITE3R_F32 ? 4 : 8;  // elements per 16-byte store
     if (out == nullptr || !aligned(out, 16)) return LITE3R_ERR_INVALID_ARG;
     if (out_stride_n < kHeadDim || out_stride_b < 0 || out_stride_h < 0) return LITE3R_ERR_INVALID_ARG;
-    if ((out_stride_b % 4) || (out_stride_h % 4) || (out_stride_n % 4)) return LITE3R_ERR_INVALID_ARG;
-    if (plan->cls == nullptr) return LITE3R_ERR_INVALID_ARG;
-    if (plan->k_crit > 0 && plan->crit_idx == nullptr) return LITE3R_ERR_INVALID_ARG;
+    if ((out_stride_b % vec) || (out_stride_h % vec) || (out_stride_n % vec)) return LITE3R_ERR_INVALID_ARG;
+    if (!plan_inside) {
+      if (plan->cls == nullptr) return LITE3R_ERR_INVALID_ARG;
+      if (plan->k_crit > 0 && plan->crit_idx == nullptr) return LITE3R_ERR_INVALID_ARG;
+    }
   }
-  const Counts c{plan->k_crit, plan->k_marg, plan->k_neg};
+  const Counts c{effective.k_crit, effective.k_marg, effective.k_neg};
   if (workspace == nullptr || !aligned(workspace, 256)) return LITE3R_ERR_INVALID_ARG;
-  if (workspace_bytes < forward_workspace_bytes(*shape, c)) return LITE3R_ERR_WORKSPACE;
+  if (workspace_bytes < forward_workspace_bytes(*shape, c, plan_inside)) return LITE3R_ERR_WORKSPACE;
+  if ((st = check_device()) != LITE3R_OK) return st;
   ForwardArgs a = {};
   if (q != nullptr) a.q = *q;
   a.k = *k;
@@ -244,9 +336,12 @@ static lite3r_status forward_phases(int phases, const lite3r_fp8* q, const lite3
   a.proj_head_stride = proj_head_stride;
   a.s = *shape;
   a.phi = static_cast<int>(phi);
-  a.plan = *plan;
+  a.plan = effective;
+  a.plan_inside = plan_inside ? 1 : 0;
+  a.crit = crit;
+  a.neg = neg;
   a.out = out;
-  a.out_dtype = LITE3R_F32;
+  a.out_dtype = static_cast<int>(out_dtype);
   a.out_stride_b = out_stride_b;
   a.out_stride_h = out_stride_h;
   a.out_stride_n = out_stride_n;
@@ -257,12 +352,12 @@ static lite3r_status forward_phases(int phases, const lite3r_fp8* q, const lite3
 }
 
 lite3r_status lite3r_sla_forward(const lite3r_fp8* q, const lite3r_fp8* k, const lite3r_fp8* v, const float* proj,
-                                 long long proj_head_stride, const lite3r_shape* shape, lite3r_phi phi,
-                                 const lite3r_plan* plan, float* out, long long out_stride_b,
-                                 long long out_stride_h, long long out_stride_n, void* workspace,
-                                 size_t workspace_bytes, int* device_status, void* stream) {
-  return forward_phases(3, q, k, v, proj, proj_head_stride, shape, phi, plan, out, out_stride_b, out_stride_h,
-                        out_stride_n, workspace, workspace_bytes, device_status, stream);
+                                 long long proj_head_stride, const lite3r_shape* shape, double crit, double neg,
+                                 lite3r_phi phi, const lite3r_plan* plan, void* out, lite3r_dtype out_dtype,
+                                 long long out_stride_b, long long out_stride_h, long long out_stride_n,
+                                 void* workspace, size_t workspace_bytes, int* device_status, void* stream) {
+  return forward_phases(3, q, k, v, proj, proj_head_stride, shape, crit, neg, phi, plan, out, out_dtype, out_stride_b,
+                        out_stride_h, out_stride_n, workspace, workspace_bytes, device_status, stream);
 }
 
 lite3r_status lite3r_sla_forward_begin(const lite3r_fp8* k, const lite3r_fp8* v, const float* proj,
@@ -273,17 +368,29 @@ lite3r_status lite3r_sla_forward_begin(const lite3r_fp8* k, const lite3r_fp8* v,
   counts.k_crit = k_crit;
   counts.k_marg = k_marg;
   counts.k_neg = k_neg;
-  return forward_phases(1, nullptr, k, v, proj, proj_head_stride, shape, phi, &counts, nullptr, 0, 0, 0, workspace,
-                        workspace_bytes, device_status, stream);
+  return forward_phases(1, nullptr, k, v, proj, proj_head_stride, shape, 0.0, 0.0, phi, &counts, nullptr, LITE3R_F32,
+                        0, 0, 0, workspace, workspace_bytes, device_status, stream);
 }
 
 lite3r_status lite3r_sla_forward_finish(const lite3r_fp8* q, const lite3r_fp8* k, const lite3r_fp8* v,
                                         const lite3r_shape* shape, lite3r_phi phi, const lite3r_plan* plan,
-                                        float* out, long long out_stride_b, long long out_stride_h,
-                                        long long out_stride_n, void* workspace, size_t workspace_bytes,
-                                        int* device_status, void* stream) {
-  return forward_phases(2, q, k, v, nullptr, 0, shape, phi, plan, out, out_stride_b, out_stride_h, out_stride_n,
-                        workspace, workspace_bytes, device_status, stream);
+                                        void* out, lite3r_dtype out_dtype, long long out_stride_b,
+                                        long long out_stride_h, long long out_stride_n, void* workspace,
+                                        size_t workspace_bytes, int* device_status, void* stream) {
+  if (plan == nullptr) return LITE3R_ERR_INVALID_ARG;
+  return forward_phases(2, q, k, v, nullptr, 0, shape, 0.0, 0.0, phi, plan, out, out_dtype, out_stride_b,
+                        out_stride_h, out_stride_n, workspace, workspace_bytes, device_status, stream);
+}
+
+lite3r_status lite3r_workspace_layout(const lite3r_shape* shape, double crit, double neg, int plan_inside,
+                                      size_t* offsets) {
+  lite3r_status st = check_shape(shape);
+  if (st != LITE3R_OK) return st;
+  if ((st = check_fractions(crit, neg)) != LITE3R_OK) return st;
+  if (offsets == nullptr) return LITE3R_ERR_INVALID_ARG;
+  forward_workspace_offsets(*shape, class_counts(ceil_div(shape->tokens, shape->block), crit, neg), plan_inside != 0,
+                            offsets);
+  return LITE3R_OK;
 }
 
 lite3r_status lite3r_selftest_wait_expiry(int* device_status, unsigned long long limit_ns, void* stream) {

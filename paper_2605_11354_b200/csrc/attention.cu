@@ -704,12 +704,31 @@ lite3r_status launch(const AttentionLaunch& a, cudaStream_t stream) {
   const lite3r_shape& s = a.shape;
   const int nb = ceil_div(s.tokens, BS);
   const uint64_t tiles = static_cast<uint64_t>(s.batch) * s.heads * nb;
-  alignas(64) CUtensorMap map_q, map_k, map_v, map_g;
+  // The four tensor maps depend on the buffers and the shape only; a caller that runs the same buffers again (the
+  // usual serving loop) reuses the encoded maps of its previous call (one entry per calling thread).
+  struct MapCache {
+    alignas(64) CUtensorMap q, k, v, g;
+    const void* key[4] = {nullptr, nullptr, nullptr, nullptr};
+    uint64_t tiles = 0;
+    int block = 0;
+  };
+  thread_local MapCache cache;
   lite3r_status st;
-  if ((st = make_tensor_map_2d(&map_q, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.q_codes, 64, tiles * BS, 64, 64, CU_TENSOR_MAP_SWIZZLE_64B)) != LITE3R_OK) return st;
-  if ((st = make_tensor_map_2d(&map_k, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.k_codes, 64, tiles * BS, 64, 64, CU_TENSOR_MAP_SWIZZLE_64B)) != LITE3R_OK) return st;
-  if ((st = make_tensor_map_2d(&map_v, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, a.v16, 64, tiles * BS, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B)) != LITE3R_OK) return st;
-  if ((st = make_tensor_map_2d(&map_g, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.g16, 64, tiles * 64, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B)) != LITE3R_OK) return st;
+  if (cache.key[0] != a.q_codes || cache.key[1] != a.k_codes || cache.key[2] != a.v16 || cache.key[3] != a.g16 ||
+      cache.tiles != tiles || cache.block != BS) {
+    cache.key[0] = nullptr;  // stays invalid if an encode below fails
+    if ((st = make_tensor_map_2d(&cache.q, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.q_codes, 64, tiles * BS, 64, 64, CU_TENSOR_MAP_SWIZZLE_64B)) != LITE3R_OK) return st;
+    if ((st = make_tensor_map_2d(&cache.k, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.k_codes, 64, tiles * BS, 64, 64, CU_TENSOR_MAP_SWIZZLE_64B)) != LITE3R_OK) return st;
+    if ((st = make_tensor_map_2d(&cache.v, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, a.v16, 64, tiles * BS, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B)) != LITE3R_OK) return st;
+    if ((st = make_tensor_map_2d(&cache.g, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.g16, 64, tiles * 64, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B)) != LITE3R_OK) return st;
+    cache.key[0] = a.q_codes;
+    cache.key[1] = a.k_codes;
+    cache.key[2] = a.v16;
+    cache.key[3] = a.g16;
+    cache.tiles = tiles;
+    cache.block = BS;
+  }
+  const CUtensorMap &map_q = cache.q, &map_k = cache.k, &map_v = cache.v, &map_g = cache.g;
   AttnParams p;
   p.q_scales = a.q_scales;
   p.k_scales = a.k_scales;
@@ -727,8 +746,7 @@ lite3r_status launch(const AttentionLaunch& a, cudaStream_t stream) {
   p.phi = a.phi;
   p.out_dtype = a.out_dtype;
   p.status = a.device_status;
-  st = record_cuda(cudaFuncSetAttribute(attention_kernel<BS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        static_cast<int>(kSmemBytes)));
+  st = ensure_dynamic_smem(attention_kernel<BS>, static_cast<int>(kSmemBytes));
   if (st != LITE3R_OK) return st;
   const int ctas = s.batch * s.heads * (BS == 64 ? (nb + 1) / 2 : nb);
   attention_kernel<BS><<<ctas, kThreads, kSmemBytes, stream>>>(map_q, map_k, map_v, map_g, p);

@@ -25,8 +25,20 @@ lite3r_status after_launch();
 // profiling is enabled.
 void profile_mark(int idx, cudaStream_t stream);
 
-// Number of SMs of the current device.
+// Number of SMs of the current device (looked up once per device).
 lite3r_status sm_count(int* count);
+// LITE3R_OK when the current device is a compute-capability 10.x part (the kernels are sm_100a code), else
+// LITE3R_ERR_UNSUPPORTED (looked up once per device).
+lite3r_status check_device();
+
+// Sets a kernel's dynamic shared-memory limit, but only when this launch needs more than any earlier launch of that
+// kernel on that device asked for (the limits already set are remembered per kernel and device; guarded by a mutex so
+// that concurrent callers cannot leave a smaller limit behind).
+lite3r_status ensure_smem_limit(const void* kernel, int bytes);
+template <typename K>
+lite3r_status ensure_dynamic_smem(K* kernel, int bytes) {
+  return ensure_smem_limit(reinterpret_cast<const void*>(kernel), bytes);
+}
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
@@ -83,6 +95,8 @@ struct ForwardArgs {
   void* out;
   int out_dtype;
   long long out_stride_b, out_stride_h, out_stride_n;
+  int plan_inside;      // 1: the plan is built in the workspace from q/k column sums and the fractions below
+  double crit, neg;
   void* workspace;
   size_t workspace_bytes;
   int* device_status;
@@ -122,7 +136,9 @@ lite3r_status make_tensor_map_2d(CUtensorMap* map, CUtensorMapDataType type, int
                                  CUtensorMapSwizzle swizzle);
 
 lite3r_status launch_wait_expiry_probe(int* status, unsigned long long limit_ns, cudaStream_t stream);
-size_t forward_workspace_bytes(const lite3r_shape& s, const Counts& c);
+size_t forward_workspace_bytes(const lite3r_shape& s, const Counts& c, bool plan_inside = false);
+// byte offsets of the workspace's parts: summaries, aggregates, zeta, fp16 V, class bytes, critical lists
+void forward_workspace_offsets(const lite3r_shape& s, const Counts& c, bool plan_inside, size_t* offsets);
 // phases: 1 = the plan-independent first part, 2 = the rest, 3 = the whole forward
 lite3r_status launch_forward(const ForwardArgs& a, int phases, cudaStream_t stream);
 

@@ -60,10 +60,13 @@ struct Workspace {
   __nv_bfloat16* g16;  // [tiles][64][64] aggregated summaries, [e][d]
   float* zeta;         // [tiles][64]
   __half* v16;         // [tiles*Bs][64]  dequantised V as fp16
+  signed char* cls;    // [tiles][Nb]     block classes, only when the plan is built inside the workspace
+  int* crit_idx;       // [tiles][k_crit] critical lists, likewise
   size_t bytes;
+  size_t offsets[6];
 };
 
-Workspace carve(void* base, const lite3r_shape& s) {
+Workspace carve(void* base, const lite3r_shape& s, int k_crit = 0, bool plan_inside = false) {
   const size_t tiles = static_cast<size_t>(s.batch) * s.heads * ceil_div(s.tokens, s.block);
   char* p = static_cast<char*>(base);
   size_t off = 0;
@@ -73,10 +76,24 @@ Workspace carve(void* base, const lite3r_shape& s) {
     off += align_up(bytes, 1024);
     return r;
   };
+  w.offsets[0] = off;
   w.hws = reinterpret_cast<__nv_bfloat16*>(take(tiles * kSummaryRow * sizeof(__nv_bfloat16)));
+  w.offsets[1] = off;
   w.g16 = reinterpret_cast<__nv_bfloat16*>(take(tiles * kHeadDim * kHeadDim * sizeof(__nv_bfloat16)));
+  w.offsets[2] = off;
   w.zeta = reinterpret_cast<float*>(take(tiles * kHeadDim * sizeof(float)));
+  w.offsets[3] = off;
   w.v16 = reinterpret_cast<__half*>(take(tiles * s.block * kHeadDim * sizeof(__half)));
+  w.cls = nullptr;
+  w.crit_idx = nullptr;
+  w.offsets[4] = w.offsets[5] = off;
+  if (plan_inside) {
+    const size_t nb = ceil_div(s.tokens, s.block);
+    w.offsets[4] = off;
+    w.cls = reinterpret_cast<signed char*>(take(tiles * nb + 16));  // the class bytes are read in aligned 32-bit words
+    w.offsets[5] = off;
+    w.crit_idx = reinterpret_cast<int*>(take(tiles * static_cast<size_t>(k_crit) * sizeof(int) + 16));
+  }
   w.bytes = off;
   return w;
 }
@@ -87,8 +104,16 @@ lite3r_status run_forward(const ForwardArgs& a, int phases, cudaStream_t stream)
   const lite3r_shape& s = a.s;
   const int nb = ceil_div(s.tokens, BS);
   const int rows = s.batch * s.heads * nb;
-  const Workspace w = carve(a.workspace, s);
+  const Workspace w = carve(a.workspace, s, a.plan.k_crit, a.plan_inside != 0);
   lite3r_status st = LITE3R_OK;
+  lite3r_plan plan = a.plan;
+  if (a.plan_inside) {  // the block plan is built first, into the tail of the workspace
+    plan.cls = w.cls;
+    plan.crit_idx = w.crit_idx;
+    plan.marg_idx = nullptr;
+    const Counts c{plan.k_crit, plan.k_marg, plan.k_neg};
+    if ((st = launch_plan(a.q, a.k, s, c, plan, stream)) != LITE3R_OK) return st;
+  }
   if (phases & 1) profile_mark(0, stream);
   // With a linear branch the summary kernel reads every V row anyway and writes the fp16 operand on the way; the
   // stand-alone pass runs only when there is no linear branch.
@@ -112,7 +137,7 @@ lite3r_status run_forward(const ForwardArgs& a, int phases, cudaStream_t stream)
   if (!(phases & 2)) return st;
   if (a.plan.k_marg > 0) {
     profile_mark(4, stream);
-    if ((st = launch_aggregate(w.hws, a.plan.cls, s, nb, w.g16, w.zeta, a.device_status, stream)) != LITE3R_OK) return st;
+    if ((st = launch_aggregate(w.hws, plan.cls, s, nb, w.g16, w.zeta, a.device_status, stream)) != LITE3R_OK) return st;
     profile_mark(5, stream);
   }
   AttentionLaunch att;
@@ -125,7 +150,7 @@ lite3r_status run_forward(const ForwardArgs& a, int phases, cudaStream_t stream)
   att.v16 = w.v16;
   att.g16 = w.g16;
   att.zeta = w.zeta;
-  att.crit_idx = a.plan.crit_idx;
+  att.crit_idx = plan.crit_idx;
   att.k_crit = a.plan.k_crit;
   att.k_marg = a.plan.k_marg;
   att.phi = a.phi;
@@ -150,9 +175,13 @@ lite3r_status launch_wait_expiry_probe(int* status, unsigned long long limit_ns,
   return after_launch();
 }
 
-size_t forward_workspace_bytes(const lite3r_shape& s, const Counts& c) {
-  (void)c;
-  return carve(nullptr, s).bytes;
+size_t forward_workspace_bytes(const lite3r_shape& s, const Counts& c, bool plan_inside) {
+  return carve(nullptr, s, c.k_crit, plan_inside).bytes;
+}
+
+void forward_workspace_offsets(const lite3r_shape& s, const Counts& c, bool plan_inside, size_t* offsets) {
+  const Workspace w = carve(nullptr, s, c.k_crit, plan_inside);
+  for (int i = 0; i < 6; ++i) offsets[i] = w.offsets[i];
 }
 
 lite3r_status launch_forward(const ForwardArgs& a, int phases, cudaStream_t stream) {

@@ -4,8 +4,10 @@
 // another runtime's pre-planned arena, a real-time loop that must not touch the allocator, or a process whose memory
 // pool has already been sized to the last byte.  For them the
 // forward's scratch (per-key-block summaries and per-query-block aggregates) lives in a fixed array that is part of
-// the loaded library image: every GPU that loads the library reserves LITE3R_STATIC_SCRATCH_BYTES for it until the
-// process exits.  The paper has no counterpart; this is a deployment convenience of the library.
+// the loaded library image.  CUDA loads a module's device code lazily by default, so the array takes its
+// LITE3R_STATIC_SCRATCH_BYTES of device memory when this file's module is first touched on a device -- the first
+// call of the entry point there -- and keeps them until the process exits; every later call allocates nothing.
+// The paper has no counterpart; this is a deployment convenience of the library.
 #include <mutex>
 
 #include "common.cuh"
@@ -44,21 +46,24 @@ lite3r_status scratch_address(void** ptr) {
 extern "C" lite3r_status lite3r_sla_forward_static_scratch(const lite3r_fp8* q, const lite3r_fp8* k,
                                                            const lite3r_fp8* v, const float* proj,
                                                            long long proj_head_stride, const lite3r_shape* shape,
-                                                           lite3r_phi phi, const lite3r_plan* plan, float* out,
-                                                           long long out_stride_b, long long out_stride_h,
-                                                           long long out_stride_n, int* device_status, void* stream) {
+                                                           lite3r_phi phi, const lite3r_plan* plan, void* out,
+                                                           lite3r_dtype out_dtype, long long out_stride_b,
+                                                           long long out_stride_h, long long out_stride_n,
+                                                           int* device_status, void* stream) {
   using namespace lite3r;
   if (shape == nullptr || plan == nullptr) return LITE3R_ERR_INVALID_ARG;
-  // Size check first, on the host, so an oversized problem is refused before anything is looked up or enqueued.
+  // The array's address is resolved first, before any other check: under lazy module loading this look-up is what
+  // loads the module that holds the array (and makes the driver set its 32 MiB aside), so even a call that is then
+  // refused for its size serves as the warm-up that start-up code should make once per device.
+  void* scratch = nullptr;
+  lite3r_status st = scratch_address(&scratch);
+  if (st != LITE3R_OK) return st;
   size_t need = 0;
-  lite3r_status st = lite3r_forward_workspace(shape, 0.0, 0.0, &need);
+  st = lite3r_forward_workspace(shape, 0.0, 0.0, &need);  // validates the shape
   if (st != LITE3R_OK) return st;
   need = forward_workspace_bytes(*shape, Counts{plan->k_crit, plan->k_marg, plan->k_neg});
   if (need > static_cast<size_t>(LITE3R_STATIC_SCRATCH_BYTES)) return LITE3R_ERR_WORKSPACE;
-  void* scratch = nullptr;
-  st = scratch_address(&scratch);
-  if (st != LITE3R_OK) return st;
-  return lite3r_sla_forward(q, k, v, proj, proj_head_stride, shape, phi, plan, out, out_stride_b, out_stride_h,
-                            out_stride_n, scratch, static_cast<size_t>(LITE3R_STATIC_SCRATCH_BYTES), device_status,
-                            stream);
+  return lite3r_sla_forward(q, k, v, proj, proj_head_stride, shape, 0.0, 0.0, phi, plan, out, out_dtype, out_stride_b,
+                            out_stride_h, out_stride_n, scratch, static_cast<size_t>(LITE3R_STATIC_SCRATCH_BYTES),
+                            device_status, stream);
 }

@@ -496,8 +496,7 @@ template <int R>
 lite3r_status launch_rows(const lite3r_fp8& q, const lite3r_fp8& k, const lite3r_shape& s, const Counts& c,
                           const lite3r_plan& plan, int nb, cudaStream_t stream) {
   const size_t smem = plan_smem_bytes(nb, R);
-  lite3r_status st = record_cuda(
-      cudaFuncSetAttribute(plan_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  lite3r_status st = ensure_dynamic_smem(plan_kernel<R>, static_cast<int>(smem));
   if (st != LITE3R_OK) return st;
   const int row_tiles = ceil_div(nb, R);
   plan_kernel<R><<<s.batch * s.heads * row_tiles, R * 32, smem, stream>>>(q.colsum, k.colsum, k.scales, s.tokens,

@@ -9,6 +9,8 @@
 // sums of the code values as exact integers (units of 2^-9), which is all the block plan needs.  HBM traffic: 2
 // (bf16) or 4 (fp32) bytes read and 1 byte written per element; the instruction count per element decides how
 // close the kernel gets to that, hence the packed fp32x2 arithmetic.
+#include <atomic>
+
 #include "common.cuh"
 #include "sm100.cuh"
 
@@ -262,12 +264,17 @@ lite3r_status launch(const QuantBatch& batch, const lite3r_shape& s, cudaStream_
   int sms = 0;
   lite3r_status st = sm_count(&sms);
   if (st != LITE3R_OK) return st;
-  st = record_cuda(cudaFuncSetAttribute(quantize_kernel<BS, SrcT, kThreads>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem));
+  st = ensure_dynamic_smem(quantize_kernel<BS, SrcT, kThreads>, kSmem);
   if (st != LITE3R_OK) return st;
-  int per_sm = 0;
-  st = record_cuda(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, quantize_kernel<BS, SrcT, kThreads>, kThreads, kSmem));
-  if (st != LITE3R_OK) return st;
-  if (per_sm < 1) per_sm = 1;
+  // resident CTAs per SM: a property of the kernel and the part (every supported device is the same part), asked once
+  static std::atomic<int> per_sm_cached{0};
+  int per_sm = per_sm_cached.load(std::memory_order_relaxed);
+  if (per_sm == 0) {
+    st = record_cuda(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, quantize_kernel<BS, SrcT, kThreads>, kThreads, kSmem));
+    if (st != LITE3R_OK) return st;
+    if (per_sm < 1) per_sm = 1;
+    per_sm_cached.store(per_sm, std::memory_order_relaxed);
+  }
   const long long all = static_cast<long long>(tiles) * batch.count;
   const int grid = static_cast<int>(all < static_cast<long long>(sms) * per_sm ? all : static_cast<long long>(sms) * per_sm);
   quantize_kernel<BS, SrcT, kThreads><<<grid, kThreads, kSmem, stream>>>(batch, s.heads, s.tokens, nb, tiles);

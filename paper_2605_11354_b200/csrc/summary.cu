@@ -393,8 +393,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) summary_kernel(const Sum
 
 template <int BS>
 lite3r_status launch(const SummaryParams& p, int sm_count, cudaStream_t stream) {
-  lite3r_status st = record_cuda(cudaFuncSetAttribute(summary_kernel<BS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                      static_cast<int>(kSmemBytes)));
+  lite3r_status st = ensure_dynamic_smem(summary_kernel<BS>, static_cast<int>(kSmemBytes));
   if (st != LITE3R_OK) return st;
   const int grid = p.rounds < sm_count * kCtasPerSm ? p.rounds : sm_count * kCtasPerSm;
   summary_kernel<BS><<<grid, kThreads, kSmemBytes, stream>>>(p);

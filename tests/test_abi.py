@@ -52,7 +52,23 @@ def test_size_queries():
     shape = lt.Shape(4, 16, 21984, 64, 128)
     codes, scales, colsum = lt.lite3r_fp8_sizes(shape)
     assert codes == 4 * 16 * 172 * 128 * 64 and scales == 4 * 16 * 172 * 4 and colsum == 4 * 16 * 172 * 64 * 4
-    assert lt.lite3r_forward_workspace(shape, 0.08, 0.7) > 0
+    plain = lt.lite3r_forward_workspace(shape, 0.08, 0.7)
+    planned = lt.lite3r_forward_workspace_planned(shape, 0.08, 0.7)
+    tiles = 4 * 16 * 172
+    # with the plan inside, the class bytes and the critical lists (14 of 172 blocks) come on top
+    assert plain > 0 and planned >= plain + tiles * 172 + tiles * 14 * 4
+    off = lt.lite3r_workspace_layout(shape, 0.08, 0.7, plan_inside=True)
+    assert off[0] == 0 and list(off) == sorted(off) and off[4] == plain and off[5] >= off[4] + tiles * 172
+    assert off[1] - off[0] >= tiles * 4160 * 2 and off[2] - off[1] >= tiles * 64 * 64 * 2
+    assert off[3] - off[2] >= tiles * 64 * 4 and off[4] - off[3] >= tiles * 128 * 64 * 2
+    assert lt.lite3r_workspace_layout(shape, 0.08, 0.7)[:4] == off[:4]
+
+
+def test_static_scratch_tile_limits():
+    """The 32 MiB array holds 1344 tiles at block 64 and 1012 at block 128 (what the header says)."""
+    for block, fits in ((64, 1344), (128, 1012)):
+        assert lt.lite3r_forward_workspace(lt.Shape(1, 1, fits * block, 64, block), 0.1, 0.6) <= lt.STATIC_SCRATCH_BYTES
+        assert lt.lite3r_forward_workspace(lt.Shape(1, 1, (fits + 1) * block, 64, block), 0.1, 0.6) > lt.STATIC_SCRATCH_BYTES
 
 
 @pytest.mark.parametrize("shape,status", [
@@ -74,6 +90,9 @@ def test_bad_fractions_and_null_pointers_are_rejected(built_library):
     f = lt.Fp8(None, None, None)
     p = lt.Plan(None, None, None, 0, 0, 0)
     assert built_library.lite3r_sla_plan(C.byref(f), C.byref(f), C.byref(shape), 0.5, 0.2, C.byref(p), None) == 1
-    assert built_library.lite3r_sla_forward(C.byref(f), C.byref(f), C.byref(f), None, 0, C.byref(shape), 0, C.byref(p),
-                                            None, 0, 0, 64, None, 0, None, None) == 1
+    assert built_library.lite3r_sla_forward(C.byref(f), C.byref(f), C.byref(f), None, 0, C.byref(shape), 0.5, 0.2, 0,
+                                            C.byref(p), None, 0, 0, 0, 64, None, 0, None, None) == 1
+    # no plan: the fractions are validated instead, and q / k must then carry column sums
+    assert built_library.lite3r_sla_forward(C.byref(f), C.byref(f), C.byref(f), None, 0, C.byref(shape), 1.5, 0.2, 0,
+                                            None, None, 0, 0, 0, 64, None, 0, None, None) == 1
     assert built_library.lite3r_status_string(3) == b"workspace too small"

@@ -301,3 +301,174 @@ def test_device_waits_are_bounded():
     assert 1.0 <= t0.elapsed_time(t1) < 200.0
     wl = wk.WORKLOADS["tiny"]
     full_parity(wl, wk.make_inputs(wl))
+
+
+# ------------------------------------------------------------------------------------------------ boundary options
+def bf16_round(x: np.ndarray) -> np.ndarray:
+    return wk.round_to_bf16(x.astype(np.float32)).astype(np.float64)
+
+
+@pytest.mark.parametrize("dtype,block", [(torch.bfloat16, 64), (torch.float16, 64), (torch.bfloat16, 128)])
+def test_sixteen_bit_output(dtype, block):
+    """out_dtype bf16 / fp16: the stored values are the fp32 result rounded to nearest even.  Checked two ways: bit for
+    bit against the fp32 run's values cast by torch, and against the oracle within the fp32 tolerance plus half an
+    ulp of the output type (bf16: 2^-9 relative, fp16: 2^-12)."""
+    wl = small_workload(f"out16-{block}", tokens=1100, block=block, heads=3, batch=2)
+    inputs = wk.make_inputs(wl)
+    eng, out32 = pu.run_gpu(inputs, wl)
+    proj = torch.from_numpy(inputs["proj"]).cuda()
+    buf = torch.full((wl.batch, wl.heads, wl.tokens, 64), float("nan"), dtype=dtype, device="cuda")
+    lt.lite3r_sla_forward(eng.q8, eng.k8, eng.v8, proj, eng.shape, eng.phi, eng.plan, buf, eng.workspace, eng.status)
+    torch.cuda.synchronize()
+    assert int(eng.status.item()) == 0
+    assert torch.equal(buf, out32.to(dtype))
+    ref = oracle_subset(inputs, wl, list(range(wl.heads)), cls=eng.plan.cls.cpu().numpy())
+    got = buf.float().cpu().numpy().astype(np.float64)
+    half_ulp = 2.0 ** -9 if dtype == torch.bfloat16 else 2.0 ** -12
+    err = np.abs(got - ref["out"])
+    assert (err <= pu.MAX_ABS_TOL + half_ulp * np.abs(ref["out"])).all()
+    rel, _ = pu.output_errors(got, ref["out"])
+    assert rel <= pu.REL_L2_TOL + half_ulp  # rounding alone is at most half an ulp relative on every element
+
+
+def test_token_major_sixteen_bit_output():
+    wl = small_workload("out16-strides", tokens=450, batch=2, heads=3)
+    inputs = wk.make_inputs(wl)
+    eng, out = pu.run_gpu(inputs, wl)
+    proj = torch.from_numpy(inputs["proj"]).cuda()
+    buf = torch.full((wl.batch, wl.tokens, wl.heads, 64), float("nan"), dtype=torch.bfloat16, device="cuda")
+    view = buf.permute(0, 2, 1, 3)
+    lt.lite3r_sla_forward(eng.q8, eng.k8, eng.v8, proj, eng.shape, eng.phi, eng.plan, view, eng.workspace, eng.status)
+    torch.cuda.synchronize()
+    assert torch.equal(view, out.to(torch.bfloat16))
+
+
+@pytest.mark.parametrize("block,crit,neg", [(64, 0.25, 0.4), (128, 0.1, 0.5), (64, 0.0, 0.3), (64, 1.0, 0.0)])
+def test_forward_builds_its_own_plan(block, crit, neg):
+    """plan == NULL: lite3r_sla_forward classifies the blocks itself (inside its workspace) from the fractions; the
+    result is bit-identical to lite3r_sla_plan followed by the forward, and the plan it left in the workspace is the
+    one lite3r_sla_plan writes."""
+    wl = small_workload(f"selfplan-{block}", tokens=1500, block=block, heads=2, batch=2, crit=crit, neg=neg)
+    inputs = wk.make_inputs(wl)
+    eng, expected = pu.run_gpu(inputs, wl)
+    inside = lt.SlaForward(wl.batch, wl.heads, wl.tokens, wl.block, crit, neg, plan_inside=True)
+    q, k, v = (pu.to_device(inputs[n], wl.src_dtype) for n in ("q", "k", "v"))
+    proj = torch.from_numpy(inputs["proj"]).cuda()
+    inside.workspace.fill_(0xEE)
+    out = inside.run(q, k, v, proj)
+    torch.cuda.synchronize()
+    assert int(inside.status.item()) == 0
+    assert torch.equal(out, expected)
+    off = lt.lite3r_workspace_layout(inside.shape, crit, neg, plan_inside=True)
+    nb, tiles = wl.n_blocks, wl.batch * wl.heads * wl.n_blocks
+    cls = inside.workspace[off[4]:off[4] + tiles * nb].view(torch.int8).view(wl.batch, wl.heads, nb, nb)
+    assert torch.equal(cls, eng.plan.cls)
+    if eng.plan.k_crit:
+        lists = inside.workspace[off[5]:off[5] + tiles * eng.plan.k_crit * 4].view(torch.int32)
+        assert torch.equal(lists.view(wl.batch, wl.heads, nb, eng.plan.k_crit), eng.plan.crit_idx)
+
+
+# ------------------------------------------------------------------------------------------------ memory safety
+@pytest.mark.parametrize("tokens,block,batch,heads,crit,neg", [(7, 64, 1, 1, 0.5, 0.2), (1000, 64, 1, 2, 0.25, 0.4),
+                                                                (1000, 128, 2, 1, 0.25, 0.4), (1374, 64, 3, 2, 0.25, 0.5),
+                                                                (200, 64, 1, 1, 1.0, 0.0), (200, 128, 1, 1, 0.0, 0.0)])
+def test_no_write_outside_the_buffers(tokens, block, batch, heads, crit, neg):
+    """Every buffer the library writes (codes, scales, column sums, classes, both index lists, workspace, output) sits
+    between two bands of a known byte pattern; after quantise + plan + forward the bands must be untouched.  Stands
+    in for a memory checker: a kernel that writes a few bytes past a buffer fails here."""
+    wl = small_workload("bands", tokens=tokens, block=block, batch=batch, heads=heads, crit=crit, neg=neg)
+    inputs = wk.make_inputs(wl)
+    shape = lt.Shape(batch, heads, tokens, 64, block)
+    band = 4096
+    guarded = []
+
+    def banded(nbytes, dtype, shp):
+        raw = torch.full((nbytes + 2 * band + 256,), 0xA5, dtype=torch.uint8, device="cuda")
+        start = band + (-(raw.data_ptr() + band)) % 256
+        guarded.append((raw, start, nbytes))
+        return raw[start:start + nbytes].view(dtype).view(shp)
+
+    codes_b, scales_b, colsum_b = lt.lite3r_fp8_sizes(shape)
+    nb = wl.n_blocks
+    fp8 = []
+    for _ in range(3):
+        fp8.append(lt.Fp8Tensor(banded(codes_b, torch.uint8, (batch, heads, nb * block, 64)),
+                                banded(scales_b, torch.float32, (batch, heads, nb)),
+                                banded(colsum_b, torch.int32, (batch, heads, nb, 64))))
+    cls_b, crit_b, marg_b, kc, km, kn = lt.lite3r_plan_sizes(shape, crit, neg)
+    plan = lt.PlanBuffers(banded(cls_b, torch.int8, (batch, heads, nb, nb)),
+                          banded(max(crit_b, 4), torch.int32, (-1,))[:batch * heads * nb * kc].view(batch, heads, nb, kc),
+                          banded(max(marg_b, 4), torch.int32, (-1,))[:batch * heads * nb * km].view(batch, heads, nb, km),
+                          kc, km, kn)
+    ws = banded(lt.lite3r_forward_workspace(shape, crit, neg), torch.uint8, (-1,))
+    out = banded(batch * heads * tokens * 64 * 4, torch.float32, (batch, heads, tokens, 64))
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    q, k, v = (pu.to_device(inputs[n], wl.src_dtype) for n in ("q", "k", "v"))
+    proj = torch.from_numpy(inputs["proj"]).cuda()
+    lt.lite3r_quantize_fp8_qkv(q, k, v, shape, *fp8)
+    lt.lite3r_sla_plan(fp8[0], fp8[1], shape, crit, neg, plan)
+    lt.lite3r_sla_forward(fp8[0], fp8[1], fp8[2], proj, shape, lt.PHI_SOFTMAX, plan, out, ws, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for raw, start, nbytes in guarded:
+        assert bool((raw[:start] == 0xA5).all()) and bool((raw[start + nbytes:] == 0xA5).all())
+    # and the run is the ordinary one
+    eng, expected = pu.run_gpu(inputs, wl, crit=crit, neg=neg)
+    assert torch.equal(out, expected)
+
+
+# ------------------------------------------------------------------------------------------------ intermediates
+@pytest.mark.parametrize("block,phi", [(64, "softmax"), (128, "softmax"), (64, "elu1")])
+def test_workspace_intermediates_against_the_oracle(block, phi):
+    """The linear branch's intermediates as the kernels leave them in the workspace: per-key-block summaries
+    ((H_j W)^T | z_j), their sums over the marginal blocks (G_i^T W-folded | zeta_i) and the fp16 copy of V, against
+    the oracle's kv_summaries (times W) at the precision they are stored in (bf16: 2^-9 relative per element)."""
+    wl = small_workload(f"ws-{block}-{phi}", tokens=1000, block=block, heads=2, batch=1)
+    inputs = wk.make_inputs(wl)
+    eng, _ = pu.run_gpu(inputs, wl, phi=phi)
+    ref = oracle_subset(inputs, wl, [0, 1], phi=phi, cls=eng.plan.cls.cpu().numpy(), query_blocks=[])
+    Hs, zs = orc.kv_summaries(ref["khat"], ref["vhat"], block, phi)
+    W = inputs["proj"].astype(np.float64)
+    HW = np.einsum("bhjde,hef->bhjdf", Hs, W)  # H_j W, [d][f]
+    off = lt.lite3r_workspace_layout(eng.shape, wl.crit, wl.neg)
+    nb, tiles = wl.n_blocks, wl.heads * wl.n_blocks
+    ws = eng.workspace
+    hws = ws[off[0]:off[0] + tiles * 4160 * 2].view(torch.bfloat16).float().cpu().numpy().reshape(1, wl.heads, nb, 4160)
+    got_hw_t = hws[..., :4096].reshape(1, wl.heads, nb, 64, 64)  # [f][d]
+    got_z = hws[..., 4096:]
+
+    def close(got, want, rel, what):
+        scale = np.abs(want).max()
+        err = np.abs(got - want).max()
+        assert err <= rel * scale, (what, err, scale)
+
+    close(got_hw_t, np.swapaxes(HW, -1, -2), 6e-3, "summaries")  # fp16 operands, bf16 storage
+    close(got_z, zs, 4e-3, "normalisers")
+    cls = eng.plan.cls.cpu().numpy()
+    marg = (cls == 1).astype(np.float64)
+    G = np.einsum("bhij,bhjdf->bhidf", marg, HW)
+    zeta = np.einsum("bhij,bhjd->bhid", marg, zs)
+    g16 = ws[off[1]:off[1] + tiles * 4096 * 2].view(torch.bfloat16).float().cpu().numpy().reshape(1, wl.heads, nb, 64, 64)
+    zt = ws[off[2]:off[2] + tiles * 64 * 4].view(torch.float32).cpu().numpy().reshape(1, wl.heads, nb, 64)
+    close(g16, np.swapaxes(G, -1, -2), 8e-3, "aggregates")
+    close(zt, zeta, 4e-3, "zeta")
+    v16 = ws[off[3]:off[3] + tiles * block * 64 * 2].view(torch.float16).float().cpu().numpy()
+    v16 = v16.reshape(1, wl.heads, nb * block, 64)[:, :, :wl.tokens]
+    assert np.abs(v16 - ref["vhat"]).max() <= 2.0 ** -11 * np.abs(ref["vhat"]).max()
+
+
+@pytest.mark.parametrize("phi,vscale,kscale", [("softmax", 300.0, 1.0), ("elu1", 100.0, 3.0), ("softmax", 1e-3, 20.0)])
+def test_large_and_small_magnitudes(phi, vscale, kscale):
+    """Values far from unit scale (V in the hundreds, K several times larger, V tiny): inside the documented range the
+    fp16 / bf16 intermediates neither overflow nor lose the result; checked against the oracle with the tolerance
+    scaled by the output's magnitude."""
+    wl = small_workload(f"mag-{phi}", tokens=900, heads=2, src_dtype="f32")
+    inputs = wk.make_inputs(wl)
+    inputs["v"] = (inputs["v"] * np.float32(vscale)).astype(np.float32)
+    inputs["k"] = (inputs["k"] * np.float32(kscale)).astype(np.float32)
+    eng, out = pu.run_gpu(inputs, wl, phi=phi)
+    ref = oracle_subset(inputs, wl, [0, 1], phi=phi, cls=eng.plan.cls.cpu().numpy())
+    got = out.cpu().numpy()
+    assert np.isfinite(got).all()
+    rel, mx = pu.output_errors(got, ref["out"])
+    assert rel <= pu.REL_L2_TOL and mx <= pu.MAX_ABS_TOL * max(1.0, vscale)
