@@ -190,6 +190,87 @@ def build_roofline(wl, plan, stage_ms, peaks, peak_kind, fp8_probe=None):
             "stage_ms": stage_ms, "kernels": table}
 
 
+# ------------------------------------------------------------------------------------------------ every configuration
+PER_CONFIG = (("tiny", None), ("vggt8", None), ("vggt32", None), ("da3l", None), ("frame32", None),
+              ("stress100", (0.02, 0.60)), ("stress100", (0.05, 0.60)), ("stress100", (0.10, 0.60)),
+              ("stress100", (0.25, 0.60)), ("stress100", (1.00, 0.00)))
+
+
+def measure_config(lt, wl, crit, neg, dev, proj, device, flush, peaks, reps=5):
+    """Step and stage times of one configuration (outside the headline's timed region): whole step with L2 flushed
+    before every run and back to back (L2 as the previous run left it), quantiser / plan / forward stages from CUDA
+    events, the forward again with bf16 output, and each kernel against its bound."""
+    from dataclasses import replace
+    wl = replace(wl, crit=crit, neg=neg)
+    eng = lt.SlaForward(wl.batch, wl.heads, wl.tokens, wl.block, crit, neg, device=device)
+
+    def timed_once(fn, flushed):
+        if flushed:
+            flush.fill_(1)
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        start.record()
+        fn()
+        end.record()
+        end.synchronize()
+        return start.elapsed_time(end)
+
+    run = lambda: eng.run(dev["q"], dev["k"], dev["v"], proj, overlap=True)  # noqa: E731
+    for _ in range(3):
+        run()
+    torch.cuda.synchronize(device)
+    cold = statistics.median(timed_once(run, True) for _ in range(reps))
+    warm = statistics.median(timed_once(run, False) for _ in range(reps))
+    lt.profile_enable(True)
+    stages = []
+    for _ in range(reps):
+        timed_once(lambda: eng.run(dev["q"], dev["k"], dev["v"], proj), True)
+        stages.append(lt.profile_stage_ms())
+    lt.profile_enable(False)
+    quant = statistics.median(timed_once(lambda: eng.quantize(dev["q"], dev["k"], dev["v"]), True) for _ in range(reps))
+    plan = statistics.median(timed_once(eng.make_plan, True) for _ in range(reps))
+    fwd32 = statistics.median(timed_once(lambda: eng.forward(proj), True) for _ in range(reps))
+    out16 = torch.empty(eng.out.shape, dtype=torch.bfloat16, device=device)
+    fwd16 = statistics.median(timed_once(lambda: eng.forward(proj, out=out16), True) for _ in range(reps))
+    assert int(eng.status.item()) == 0
+    stage = {"quantize_qkv": quant, "plan": plan, "prep": statistics.median(s[0] for s in stages),
+             "summary": statistics.median(s[1] for s in stages), "aggregation": statistics.median(s[2] for s in stages),
+             "attention": statistics.median(s[3] for s in stages)}
+    table = build_roofline(wl, eng.plan, stage, peaks, "measured")["kernels"]
+    res = {"workload": wl.name, "crit": crit, "neg": neg, "k_crit": eng.plan.k_crit, "k_marg": eng.plan.k_marg,
+           "ms_l2_flushed": cold, "ms_l2_warm": warm, "ms_quantize": quant, "ms_plan": plan, "ms_forward": fwd32,
+           "ms_forward_bf16_out": fwd16, "dense_equiv_tflops": wl.dense_equiv_flops / cold / 1e9,
+           "stage_ms": stage, "roofline_frac": {k: round(v["frac"], 4) for k, v in table.items()},
+           "attention_tflops_executed": table["attention"]["achieved"] if "attention" in table else None}
+    del eng, out16
+    return res
+
+
+def per_config_table(lt, device, flush, peaks):
+    """One entry per benchmark configuration (the five of the contract, the frame-attention shape and the sparsity
+    sweep of the stress configuration)."""
+    rows, cached, cached_name = [], None, None
+    for name, fractions in PER_CONFIG:
+        try:
+            wl = wk.WORKLOADS[name]
+            if cached_name != name:
+                cached = None
+                torch.cuda.empty_cache()
+                inputs = wk.make_inputs(wl)
+                dev = {}
+                for n in ("q", "k", "v"):
+                    if wl.src_dtype == "bf16":
+                        dev[n] = torch.from_numpy(wk.bf16_bits(inputs[n]).view(np.int16)).to(device).view(torch.bfloat16)
+                    else:
+                        dev[n] = torch.from_numpy(inputs[n]).to(device)
+                cached, cached_name = (dev, torch.from_numpy(inputs["proj"]).to(device)), name
+                del inputs
+            crit, neg = fractions if fractions is not None else (wl.crit, wl.neg)
+            rows.append(measure_config(lt, wl, crit, neg, cached[0], cached[1], device, flush, peaks))
+        except Exception as exc:  # noqa: BLE001 - a failed configuration is reported, the others still run
+            rows.append({"workload": name, "error": f"{type(exc).__name__}: {exc}"})
+    return rows
+
+
 # ------------------------------------------------------------------------------------------------ CPU oracle timing
 def time_oracle(wl, inputs, n_heads, budget_blocks):
     """One bounded sample of the step on the host cores: quantiser and plan for the first `n_heads` heads of every
@@ -417,6 +498,12 @@ def run_ours(args, wl):
             "e2e": {"value": e2e_flops / 1e12, "unit": UNIT, "h2d_bytes_per_step": in_bytes,
                     "d2h_bytes_per_step": out_bytes},
             "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline}
+    if world == 1 and not args.no_per_config:
+        del dev, eng
+        clocks_all = ClockSampler(local_rank)
+        clocks_all.start()
+        line["per_config"] = per_config_table(lt, device, flush, peaks)
+        line["per_config_clocks"] = clocks_all.stop()
     if world == 1 and not args.no_cpu_baseline:
         sec, sample = time_oracle(wl, inputs, wl.heads, args.oracle_blocks)
         line["cpu_baseline"] = {"value": flops / sec / 1e12, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
@@ -434,6 +521,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--oracle-blocks", type=int, default=512)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true", help="skip the table over all configurations")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     wl = wk.WORKLOADS[args.workload]

@@ -56,3 +56,14 @@ def test_roofline_headline_is_the_largest_stage():
     assert "prep" not in r["kernels"]  # a stage that did not run has no entry
     assert r["kernels"]["quantize_qkv"]["bound"] == "hbm" and r["kernels"]["quantize_qkv"]["peak"] == 6500.0
     assert abs(r["frac_of_fp8_gemm_probe"] - r["achieved"] / 3200.0) < 1e-12
+
+
+def test_per_config_table_covers_every_configuration():
+    """The table bench.py adds to its line (`per_config`) has one entry per contract configuration, the frame-attention
+    shape and all five points of the stress sweep."""
+    names = [n for n, _ in bench.PER_CONFIG]
+    for wl in ("tiny", "vggt8", "vggt32", "da3l", "stress100", "frame32"):
+        assert wl in names and wl in wk.WORKLOADS
+    sweep = [f for n, f in bench.PER_CONFIG if n == "stress100"]
+    assert tuple(sweep) == tuple(wk.STRESS_SWEEP)
+    assert all(f is None for n, f in bench.PER_CONFIG if n != "stress100")
