@@ -15,6 +15,8 @@ Conventions
 * The quantiser's three operations (scale, divide, clamp) run in fp32 because
   the paper's quantiser is an fp32 program whose integer result must be
   reproduced bit for bit; everything after the codes is fp64.
+* The FP8 linear layer in front of the attention (per-token / per-output-row scaled e4m3 operands, Algorithm 2 in its
+  deployed form) follows the same rule: scale, divide and clamp in fp32, the product in fp64.
 * Pins (checked in tests/test_oracle_pins.py): the e4m3 codec against the
   closed-form format definition and torch's float8_e4m3fn cast; crit=1 against
   dense softmax attention; crit=0,neg=0 against the global linear-attention
@@ -277,3 +279,46 @@ def sla_forward_from_source(q, k, v, proj, block, crit, neg, phi="softmax", cls=
     out = sla_forward(qhat, khat, vhat, proj, cls, block, phi, query_blocks)
     return {"q_codes": qc, "q_scales": qs, "k_codes": kc, "k_scales": ks, "v_codes": vc, "v_scales": vs,
             "qhat": qhat, "khat": khat, "vhat": vhat, "scores": scores, "cls": cls, "out": out}
+
+
+# --------------------------------------------------------------------------- FP8 linear layer (Algorithm 2, deployed form)
+def quantize_fp8_rows(x: np.ndarray):
+    """Scaled FP8 quantisation with one scale per row of a matrix [R, C]: per token for activations, per output
+    row for weights (appendix "Per-Tensor Dynamic Scaling").  scale_i = (max_j |x_ij| + 1e-8) / 448, codes =
+    e4m3(clamp(x / scale, -448, 448)); the three steps in fp32 as in quantize_fp8_blocks.
+    Returns (codes uint8 [R, C], scales fp32 [R])."""
+    x = np.asarray(x, dtype=np.float32)
+    amax = np.abs(x).max(axis=1).astype(np.float32)
+    scales = ((amax + np.float32(SCALE_EPS)) / np.float32(FP8_MAX)).astype(np.float32)
+    y = (x / scales[:, None]).astype(np.float32)
+    y = np.minimum(np.maximum(y, np.float32(-FP8_MAX)), np.float32(FP8_MAX))
+    return e4m3_encode_rne(y), scales
+
+
+def dequantize_rows(codes: np.ndarray, scales: np.ndarray) -> np.ndarray:
+    """value(code) * scale of its row, fp64 (exact)."""
+    return e4m3_decode(codes) * scales.astype(np.float64)[:, None]
+
+
+def linear_fp8(x_codes, x_scales, w_codes, w_scales, bias=None) -> np.ndarray:
+    """y = x_q W_q^T + b (the linear transformation of Algorithm 2) on the quantised operands: x_q [N, d_in] with
+    per-token scales, W_q [d_out, d_in] with per-output-row scales.  fp64 [N, d_out]."""
+    y = dequantize_rows(x_codes, x_scales) @ dequantize_rows(w_codes, w_scales).T
+    if bias is not None:
+        y = y + np.asarray(bias, dtype=np.float64)[None, :]
+    return y
+
+
+def qkv_project_fp8(x, w_qkv, heads: int, bias=None):
+    """The qkv projection of an attention block as an FP8 linear layer (Eq. 2: W_q = Q_fp8(W), X_q = Q_fp8(X),
+    Y = Linear(X_q, W_q)): x [B, N, d_model], w_qkv [3 * heads * D, d_model] with the output rows ordered
+    (q | k | v) x head x D.  Returns (q, k, v) fp64 [B, heads, N, D] and the quantised operands."""
+    x = np.asarray(x, dtype=np.float32)
+    B, N, dm = x.shape
+    xc, xs = quantize_fp8_rows(x.reshape(B * N, dm))
+    wc, ws = quantize_fp8_rows(w_qkv)
+    y = linear_fp8(xc, xs, wc, ws, bias)
+    D = w_qkv.shape[0] // (3 * heads)
+    y = y.reshape(B, N, 3, heads, D)
+    q, k, v = (np.ascontiguousarray(y[:, :, i].transpose(0, 2, 1, 3)) for i in range(3))
+    return q, k, v, {"x_codes": xc, "x_scales": xs, "w_codes": wc, "w_scales": ws}

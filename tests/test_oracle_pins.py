@@ -427,3 +427,77 @@ def test_from_source_composition_against_independent_pieces(phi):
     # and the brute force with the fractions swapped is a different answer (the test would notice the swap)
     swapped = brute_force(qh, kh, vh, w.astype(np.float64), block, neg, crit, phi)
     assert not np.allclose(res["out"], swapped, rtol=1e-3, atol=1e-3)
+
+
+# ------------------------------------------------------------------ FP8 linear layer (Algorithm 2)
+def test_row_quantizer_against_torch_cast():
+    g = rng(31)
+    x = (g.standard_normal((37, 48)) * g.uniform(0.01, 30.0, size=(37, 1))).astype(np.float32)
+    x[5] = 0.0
+    x[6, 3] = 1.0e4
+    codes, scales = orc.quantize_fp8_rows(x)
+    for i in range(x.shape[0]):
+        s = np.float32(np.float32(np.float32(np.abs(x[i]).max()) + np.float32(1e-8)) / np.float32(448.0))
+        assert scales[i] == s
+        ref = torch.from_numpy((x[i] / s).astype(np.float32)).clamp(-448, 448).to(torch.float8_e4m3fn)
+        assert np.array_equal(codes[i], ref.view(torch.uint8).numpy())
+    assert not codes[5].any() and codes[6, 3] == 0x7E
+    # every non-zero row reaches +-448, and a power-of-two factor per row only moves the scale
+    assert (np.abs(orc.e4m3_decode(codes[np.abs(x).max(axis=1) > 0])).max(axis=1) == 448).all()
+    factor = np.float32(2.0) ** g.integers(-3, 6, size=(37, 1)).astype(np.float32)
+    c2, s2 = orc.quantize_fp8_rows(x * factor)
+    keep = np.abs(x).max(axis=1) >= 0.25  # the 1e-8 guard is absorbed from there on
+    assert np.array_equal(c2[keep], codes[keep]) and np.array_equal(s2[keep], (scales * factor[:, 0])[keep])
+
+
+def test_fp8_linear_against_torch_matmul_and_scalar_loops():
+    g = rng(32)
+    N, din, dout = 23, 40, 17
+    x = g.standard_normal((N, din)).astype(np.float32) * 3
+    w = (g.standard_normal((dout, din)) / math.sqrt(din)).astype(np.float32)
+    b = g.standard_normal(dout).astype(np.float32)
+    xc, xs = orc.quantize_fp8_rows(x)
+    wc, ws = orc.quantize_fp8_rows(w)
+    y = orc.linear_fp8(xc, xs, wc, ws, b)
+    # library routine on operands dequantised through torch's float8 view
+    xq = torch.from_numpy(xc).view(torch.float8_e4m3fn).to(torch.float64) * torch.from_numpy(xs.astype(np.float64))[:, None]
+    wq = torch.from_numpy(wc).view(torch.float8_e4m3fn).to(torch.float64) * torch.from_numpy(ws.astype(np.float64))[:, None]
+    ref = torch.nn.functional.linear(xq, wq, torch.from_numpy(b.astype(np.float64))).numpy()
+    assert np.allclose(y, ref, rtol=1e-13, atol=1e-13)
+    # scalar loops, scales applied outside the integer-like sum as a kernel would
+    tab = orc.e4m3_value_table()
+    for (n, o) in ((0, 0), (22, 16), (7, 3)):
+        acc = sum(float(tab[xc[n, k]]) * float(tab[wc[o, k]]) for k in range(din))
+        assert np.isclose(y[n, o], acc * float(xs[n]) * float(ws[o]) + float(b[o]), rtol=1e-12)
+    # not symmetric in its operands, and the quantised product stays close to the unquantised one
+    assert y.shape == (N, dout)
+    exact = x.astype(np.float64) @ w.astype(np.float64).T + b
+    assert np.abs(y - exact).max() < 0.08 * np.abs(exact).max()
+    assert np.allclose(orc.linear_fp8(xc, xs, wc, ws), y - b[None, :], rtol=1e-12, atol=1e-12)
+
+
+def test_qkv_projection_layout_and_identity_weight():
+    """Output rows are ordered (q | k | v) x head x D; with a weight that copies input channels, each head's q / k /
+    v is the per-token-quantised input slice times the (exactly representable) weight."""
+    g = rng(33)
+    B, N, H, D = 2, 19, 3, 4
+    dm = H * D
+    x = g.standard_normal((B, N, dm)).astype(np.float32)
+    w = np.zeros((3 * H * D, dm), dtype=np.float32)
+    for part, gain in enumerate((1.0, 2.0, -0.5)):
+        for o in range(H * D):
+            w[part * H * D + o, o] = gain
+    q, k, v, ops = orc.qkv_project_fp8(x, w, H)
+    assert q.shape == (B, H, N, D)
+    xq = orc.dequantize_rows(ops["x_codes"], ops["x_scales"]).reshape(B, N, H, D).transpose(0, 2, 1, 3)
+    # a weight row with a single entry g dequantises to sign(g) * 448 * scale_row (its code is +-448), g up to fp32 rounding
+    gq = [math.copysign(448.0 * float(ops["w_scales"][part * H * D]), gain) for part, gain in enumerate((1.0, 2.0, -0.5))]
+    assert all(abs(a / b - 1.0) < 1e-6 for a, b in zip(gq, (1.0, 2.0, -0.5)))
+    assert np.allclose(q, gq[0] * xq, rtol=1e-12, atol=0) and np.allclose(k, gq[1] * xq, rtol=1e-12, atol=0)
+    assert np.allclose(v, gq[2] * xq, rtol=1e-12, atol=0)
+    # a general weight: equals the plain linear layer reshaped
+    w2 = (g.standard_normal((3 * H * D, dm)) / 3).astype(np.float32)
+    q2, k2, v2, ops2 = orc.qkv_project_fp8(x, w2, H)
+    y = orc.linear_fp8(ops2["x_codes"], ops2["x_scales"], ops2["w_codes"], ops2["w_scales"])
+    assert np.array_equal(k2[1, 2, 5], y[1 * N + 5, H * D + 2 * D:H * D + 3 * D])
+    assert np.array_equal(v2[0, 0, 18], y[18, 2 * H * D:2 * H * D + D])
