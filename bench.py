@@ -245,6 +245,56 @@ def measure_config(lt, wl, crit, neg, dev, proj, device, flush, peaks, reps=5):
     return res
 
 
+def measure_projection(lt, wl, device, flush, peaks, reps=5):
+    """The qkv projection in front of the attention as an FP8 GEMM whose epilogue is the block quantiser (Algorithm 2
+    in its deployed form): per-token quantiser of the activations, the fused GEMM, and the step it makes possible
+    (projection + plan + forward, no separate pass over Q, K, V)."""
+    d_model = wl.heads * wl.head_dim
+    g = torch.Generator(device="cpu").manual_seed(wl.cfg_id)
+    x = torch.randn((wl.batch * wl.tokens, d_model), generator=g).to(torch.bfloat16).to(device)
+    w = (torch.randn((3 * d_model, d_model), generator=g) / d_model ** 0.5).to(device)
+    proj = (torch.randn((wl.heads, 64, 64), generator=g) / 8).to(device)
+    wc, ws = lt.lite3r_quantize_rows_fp8(w)  # weights are quantised once, offline
+    eng = lt.SlaForward(wl.batch, wl.heads, wl.tokens, wl.block, wl.crit, wl.neg, device=device)
+    state = {}
+
+    def timed_once(fn):
+        flush.fill_(1)
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        start.record()
+        fn()
+        end.record()
+        end.synchronize()
+        return start.elapsed_time(end)
+
+    def rowq():
+        state["xc"], state["xs"] = lt.lite3r_quantize_rows_fp8(x)
+
+    def gemm():
+        lt.lite3r_qkv_project_fp8(state["xc"], state["xs"], wc, ws, None, eng.shape, eng.q8, eng.k8, eng.v8, eng.status)
+
+    def step():
+        rowq()
+        gemm()
+        eng.make_plan()
+        eng.forward(proj)
+
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize(device)
+    t_rowq = statistics.median(timed_once(rowq) for _ in range(reps))
+    t_gemm = statistics.median(timed_once(gemm) for _ in range(reps))
+    t_step = statistics.median(timed_once(step) for _ in range(reps))
+    assert int(eng.status.item()) == 0
+    flops = 2.0 * wl.batch * wl.tokens * d_model * 3 * d_model
+    fp8_peak = peaks["bf16_tflops"] * FP8_OVER_BF16
+    rowq_bytes = wl.batch * wl.tokens * d_model * 3 + wl.batch * wl.tokens * 4
+    return {"workload": wl.name + "+qkv_projection", "d_model": d_model, "ms_quantize_rows": t_rowq,
+            "ms_qkv_gemm_fused_quantiser": t_gemm, "ms_step_from_activations": t_step,
+            "gemm_tflops": flops / t_gemm / 1e9, "gemm_frac_of_fp8_peak": flops / t_gemm / 1e9 / fp8_peak,
+            "quantize_rows_frac_of_hbm": rowq_bytes / (t_rowq * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+
+
 def per_config_table(lt, device, flush, peaks):
     """One entry per benchmark configuration (the five of the contract, the frame-attention shape and the sparsity
     sweep of the stress configuration)."""
@@ -266,6 +316,8 @@ def per_config_table(lt, device, flush, peaks):
                 del inputs
             crit, neg = fractions if fractions is not None else (wl.crit, wl.neg)
             rows.append(measure_config(lt, wl, crit, neg, cached[0], cached[1], device, flush, peaks))
+            if name in ("vggt8", "vggt32"):
+                rows.append(measure_projection(lt, wl, device, flush, peaks))
         except Exception as exc:  # noqa: BLE001 - a failed configuration is reported, the others still run
             rows.append({"workload": name, "error": f"{type(exc).__name__}: {exc}"})
     return rows

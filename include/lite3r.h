@@ -209,6 +209,43 @@ LITE3R_API lite3r_status lite3r_sla_forward_static_scratch(const lite3r_fp8* q, 
                                                 long long out_stride_h, long long out_stride_n, int* device_status,
                                                 void* stream);
 
+/* ---- The FP8 linear layer in front of the attention (paper Sec. 3.4 Eq. 2; appendix "Per-Tensor Dynamic Scaling" and
+ * Algorithm 2 "FP8 fake-quantised linear" in its deployed form: the operands really are e4m3, nothing is faked). ---- */
+
+/* Scaled FP8 quantisation with one scale per row of a matrix [rows, cols] (appendix "Per-Tensor Dynamic Scaling"):
+ * per token for an activation matrix, per output row for a weight matrix.  In fp32, as for the block quantiser:
+ *   scale_i = (max_j |x_ij| + 1e-8) / 448;  code_ij = e4m3_round_to_nearest_even(clamp(x_ij / scale_i, -448, 448)).
+ * x: DEVICE, fp32 or bf16, 16-byte aligned, row_stride in elements (a multiple of 8, >= cols); cols a multiple of 16.
+ * codes: DEVICE uint8 [rows, cols] contiguous; scales: DEVICE fp32 [rows]. */
+LITE3R_API lite3r_status lite3r_quantize_rows_fp8(const void* x, lite3r_dtype dtype, long long row_stride, int rows, int cols,
+                                       unsigned char* codes, float* scales, void* stream);
+
+/* y = x_q W_q^T + b (the linear transformation of Algorithm 2) on quantised operands, e4m3 x e4m3 with fp32
+ * accumulation on the tensor cores:  y[n][o] = x_scales[n] * w_scales[o] * sum_k value(x_codes[n][k]) value(w_codes[o][k]) + bias[o].
+ * x_codes: DEVICE uint8 [rows, d_in]; w_codes: DEVICE uint8 [d_out, d_in] (the layout of an nn.Linear weight);
+ * bias: DEVICE fp32 [d_out] or NULL.  d_in must be a multiple of 128 and d_out of 64 (else LITE3R_ERR_UNSUPPORTED).
+ * y: DEVICE [rows, d_out] of y_dtype (fp32, bf16 or fp16), row pitch y_stride elements (a multiple of 8), 16-byte
+ * aligned.  device_status as for lite3r_sla_forward (cleared by the call). */
+LITE3R_API lite3r_status lite3r_linear_fp8(const unsigned char* x_codes, const float* x_scales, const unsigned char* w_codes,
+                                const float* w_scales, const float* bias, int rows, int d_in, int d_out, void* y,
+                                lite3r_dtype y_dtype, long long y_stride, int* device_status, void* stream);
+
+/* The qkv projection of an attention block as that FP8 linear layer (Eq. 2), with the block quantiser of
+ * lite3r_quantize_fp8 fused into its epilogue: Q, K and V never exist in 16 or 32 bits in memory, they leave the
+ * kernel as the lite3r_fp8 tensors lite3r_sla_plan / lite3r_sla_forward take.
+ * x_codes: [B * N, d_model] (token-major; row b * N + n); w_codes: [3 * H * 64, d_model] with the output rows ordered
+ * (q | k | v) x head x 64; bias [3 * H * 64] or NULL; shape gives B, H, N and the block size; H must be even.
+ * Each output value is formed in fp32 (accumulator x (x_scale * w_scale) + bias) and each (b, h, token-block) tile of
+ * it is then quantised by the rule of lite3r_quantize_fp8 (tile maximum over the valid tokens, scale, codes, column
+ * sums when colsum is not NULL; v_out.colsum may be NULL).  Because the fp32 accumulation order of the tensor cores is
+ * not that of an fp64 evaluation, a value may fall on the other side of an e4m3 rounding boundary than a reference
+ * computed in higher precision would put it: scales agree to within a few fp32 ulps and codes except for a small
+ * fraction that differ by one code step. */
+LITE3R_API lite3r_status lite3r_qkv_project_fp8(const unsigned char* x_codes, const float* x_scales, const unsigned char* w_codes,
+                                     const float* w_scales, const float* bias, const lite3r_shape* shape, int d_model,
+                                     lite3r_fp8 q_out, lite3r_fp8 k_out, lite3r_fp8 v_out, int* device_status,
+                                     void* stream);
+
 /* Text for a status code; the last CUDA error code (cudaError_t as int) recorded by this thread. */
 LITE3R_API const char* lite3r_status_string(lite3r_status status);
 LITE3R_API int lite3r_last_cuda_error(void);

@@ -48,7 +48,7 @@ EXPORTS = ("lite3r_fp8_sizes", "lite3r_plan_sizes", "lite3r_forward_workspace", 
            "lite3r_launch_count", "lite3r_profile_enable", "lite3r_profile_stage_ms",
            "lite3r_sla_forward_static_scratch", "lite3r_quantize_fp8_qkv", "lite3r_selftest_wait_expiry",
            "lite3r_sla_forward_begin", "lite3r_sla_forward_finish", "lite3r_forward_workspace_planned",
-           "lite3r_workspace_layout")
+           "lite3r_workspace_layout", "lite3r_quantize_rows_fp8", "lite3r_linear_fp8", "lite3r_qkv_project_fp8")
 STATIC_SCRATCH_BYTES = 32 << 20  # LITE3R_STATIC_SCRATCH_BYTES
 
 
@@ -92,6 +92,15 @@ def lib() -> C.CDLL:
                                             C.POINTER(Plan), C.c_void_p, C.c_int, C.c_longlong, C.c_longlong,
                                             C.c_longlong, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
     L.lite3r_sla_forward_finish.restype = C.c_int
+    L.lite3r_quantize_rows_fp8.argtypes = [C.c_void_p, C.c_int, C.c_longlong, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
+                                           C.c_void_p]
+    L.lite3r_quantize_rows_fp8.restype = C.c_int
+    L.lite3r_linear_fp8.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
+                                    C.c_void_p, C.c_int, C.c_longlong, C.c_void_p, C.c_void_p]
+    L.lite3r_linear_fp8.restype = C.c_int
+    L.lite3r_qkv_project_fp8.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(Shape),
+                                         C.c_int, Fp8, Fp8, Fp8, C.c_void_p, C.c_void_p]
+    L.lite3r_qkv_project_fp8.restype = C.c_int
     L.lite3r_selftest_wait_expiry.argtypes = [C.c_void_p, C.c_ulonglong, C.c_void_p]
     L.lite3r_selftest_wait_expiry.restype = C.c_int
     L.lite3r_status_string.argtypes = [C.c_int]
@@ -333,6 +342,46 @@ def lite3r_sla_forward_static_scratch(q: Fp8Tensor, k: Fp8Tensor, v: Fp8Tensor, 
         out.data_ptr(), out_dtype, out.stride(0), out.stride(1), out.stride(2),
         device_status.data_ptr() if device_status is not None else None, _stream_ptr(stream)),
         "lite3r_sla_forward_static_scratch")
+
+
+# ----------------------------------------------------------------------------- FP8 linear layer in front of the attention
+def lite3r_quantize_rows_fp8(x: torch.Tensor, stream=None):
+    """Per-row scaled e4m3 quantisation of a CUDA matrix [rows, cols] (fp32 or bf16, contiguous columns):
+    per token for activations, per output row for weights.  Returns (codes uint8 [rows, cols], scales fp32 [rows])."""
+    if not x.is_cuda or x.dim() != 2 or x.stride(1) != 1:
+        raise Lite3rError("lite3r_quantize_rows_fp8: x must be a CUDA matrix with contiguous columns")
+    dtype = {torch.float32: F32, torch.bfloat16: BF16}.get(x.dtype)
+    if dtype is None:
+        raise Lite3rError("lite3r_quantize_rows_fp8: dtype must be float32 or bfloat16")
+    codes = torch.empty(x.shape, dtype=torch.uint8, device=x.device)
+    scales = torch.empty(x.shape[0], dtype=torch.float32, device=x.device)
+    _check(lib().lite3r_quantize_rows_fp8(x.data_ptr(), dtype, x.stride(0), x.shape[0], x.shape[1], codes.data_ptr(),
+                                          scales.data_ptr(), _stream_ptr(stream)), "lite3r_quantize_rows_fp8")
+    return codes, scales
+
+
+def lite3r_linear_fp8(x_codes, x_scales, w_codes, w_scales, bias, y: torch.Tensor, device_status=None, stream=None):
+    """y = x_q W_q^T + b on e4m3 operands ([rows, d_in] x [d_out, d_in]); y: CUDA [rows, d_out] fp32 / bf16 / fp16."""
+    if y.dtype not in OUT_DTYPES or not y.is_cuda or y.dim() != 2 or y.stride(1) != 1:
+        raise Lite3rError("lite3r_linear_fp8: y must be a CUDA float32 / bfloat16 / float16 matrix")
+    rows, d_in = x_codes.shape
+    d_out = w_codes.shape[0]
+    _check(lib().lite3r_linear_fp8(x_codes.data_ptr(), x_scales.data_ptr(), w_codes.data_ptr(), w_scales.data_ptr(),
+                                   bias.data_ptr() if bias is not None else None, rows, d_in, d_out, y.data_ptr(),
+                                   OUT_DTYPES[y.dtype], y.stride(0),
+                                   device_status.data_ptr() if device_status is not None else None,
+                                   _stream_ptr(stream)), "lite3r_linear_fp8")
+
+
+def lite3r_qkv_project_fp8(x_codes, x_scales, w_codes, w_scales, bias, shape: Shape, q_out: Fp8Tensor, k_out: Fp8Tensor,
+                           v_out: Fp8Tensor, device_status=None, stream=None):
+    """qkv projection on e4m3 operands with the block quantiser fused into its epilogue: fills the three Fp8Tensors
+    the attention calls take.  x_codes [B*N, d_model], w_codes [3*H*64, d_model] ordered (q | k | v) x head x 64."""
+    _check(lib().lite3r_qkv_project_fp8(x_codes.data_ptr(), x_scales.data_ptr(), w_codes.data_ptr(), w_scales.data_ptr(),
+                                        bias.data_ptr() if bias is not None else None, C.byref(shape),
+                                        x_codes.shape[1], q_out.c_struct(), k_out.c_struct(), v_out.c_struct(),
+                                        device_status.data_ptr() if device_status is not None else None,
+                                        _stream_ptr(stream)), "lite3r_qkv_project_fp8")
 
 
 # ----------------------------------------------------------------------------- whole path

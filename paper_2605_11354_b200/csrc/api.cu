@@ -393,6 +393,61 @@ lite3r_status lite3r_workspace_layout(const lite3r_shape* shape, double crit, do
   return LITE3R_OK;
 }
 
+lite3r_status lite3r_quantize_rows_fp8(const void* x, lite3r_dtype dtype, long long row_stride, int rows, int cols,
+                                       unsigned char* codes, float* scales, void* stream) {
+  if (x == nullptr || codes == nullptr || scales == nullptr || rows <= 0 || cols <= 0) return LITE3R_ERR_INVALID_ARG;
+  if (dtype != LITE3R_F32 && dtype != LITE3R_BF16) return LITE3R_ERR_UNSUPPORTED;
+  if ((cols % 16) || row_stride < cols || (row_stride % 8) || !aligned(x, 16) || !aligned(codes, 16) || !aligned(scales, 4))
+    return LITE3R_ERR_INVALID_ARG;
+  lite3r_status st = check_device();
+  if (st != LITE3R_OK) return st;
+  return launch_rowquant(x, static_cast<int>(dtype), row_stride, rows, cols, codes, scales, static_cast<cudaStream_t>(stream));
+}
+
+static lite3r_status check_linear_operands(const unsigned char* x_codes, const float* x_scales, const unsigned char* w_codes,
+                                           const float* w_scales, const float* bias, long long rows, int d_in, int d_out) {
+  if (x_codes == nullptr || x_scales == nullptr || w_codes == nullptr || w_scales == nullptr) return LITE3R_ERR_INVALID_ARG;
+  if (rows <= 0 || rows > 0x7FFFFFFFLL - 256 || d_in <= 0 || d_out <= 0) return LITE3R_ERR_INVALID_ARG;
+  if ((d_in % 128) || (d_out % 64)) return LITE3R_ERR_UNSUPPORTED;
+  if (!aligned(x_codes, 16) || !aligned(w_codes, 16) || !aligned(x_scales, 4) || !aligned(w_scales, 4) ||
+      (bias != nullptr && !aligned(bias, 4)))
+    return LITE3R_ERR_INVALID_ARG;
+  return LITE3R_OK;
+}
+
+lite3r_status lite3r_linear_fp8(const unsigned char* x_codes, const float* x_scales, const unsigned char* w_codes,
+                                const float* w_scales, const float* bias, int rows, int d_in, int d_out, void* y,
+                                lite3r_dtype y_dtype, long long y_stride, int* device_status, void* stream) {
+  lite3r_status st = check_linear_operands(x_codes, x_scales, w_codes, w_scales, bias, rows, d_in, d_out);
+  if (st != LITE3R_OK) return st;
+  if (y_dtype != LITE3R_F32 && y_dtype != LITE3R_BF16 && y_dtype != LITE3R_F16) return LITE3R_ERR_UNSUPPORTED;
+  if (y == nullptr || !aligned(y, 16) || y_stride < d_out || (y_stride % 8)) return LITE3R_ERR_INVALID_ARG;
+  if ((st = check_device()) != LITE3R_OK) return st;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  if (device_status != nullptr && (st = record_cuda(cudaMemsetAsync(device_status, 0, sizeof(int), cs))) != LITE3R_OK) return st;
+  return launch_linear_fp8(x_codes, x_scales, w_codes, w_scales, bias, rows, d_in, d_out, y, static_cast<int>(y_dtype),
+                           y_stride, device_status, cs);
+}
+
+lite3r_status lite3r_qkv_project_fp8(const unsigned char* x_codes, const float* x_scales, const unsigned char* w_codes,
+                                     const float* w_scales, const float* bias, const lite3r_shape* shape, int d_model,
+                                     lite3r_fp8 q_out, lite3r_fp8 k_out, lite3r_fp8 v_out, int* device_status,
+                                     void* stream) {
+  lite3r_status st = check_shape(shape);
+  if (st != LITE3R_OK) return st;
+  if (shape->heads % 2) return LITE3R_ERR_UNSUPPORTED;  // an output tile of 128 columns is two whole heads
+  const long long rows = static_cast<long long>(shape->batch) * shape->tokens;
+  st = check_linear_operands(x_codes, x_scales, w_codes, w_scales, bias, rows, d_model, 3 * shape->heads * kHeadDim);
+  if (st != LITE3R_OK) return st;
+  const lite3r_fp8 out[3] = {q_out, k_out, v_out};
+  for (int i = 0; i < 3; ++i)
+    if ((st = check_fp8(&out[i], true, false)) != LITE3R_OK) return st;
+  if ((st = check_device()) != LITE3R_OK) return st;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  if (device_status != nullptr && (st = record_cuda(cudaMemsetAsync(device_status, 0, sizeof(int), cs))) != LITE3R_OK) return st;
+  return launch_qkv_project(x_codes, x_scales, w_codes, w_scales, bias, *shape, d_model, out, device_status, cs);
+}
+
 lite3r_status lite3r_selftest_wait_expiry(int* device_status, unsigned long long limit_ns, void* stream) {
   if (device_status == nullptr || limit_ns == 0 || limit_ns > 1000000000ull) return LITE3R_ERR_INVALID_ARG;
   return launch_wait_expiry_probe(device_status, limit_ns, static_cast<cudaStream_t>(stream));

@@ -135,6 +135,16 @@ lite3r_status make_tensor_map_2d(CUtensorMap* map, CUtensorMapDataType type, int
                                  uint64_t inner, uint64_t rows, uint32_t box_inner, uint32_t box_rows,
                                  CUtensorMapSwizzle swizzle);
 
+// The FP8 linear layer in front of the attention (linear.cu).
+lite3r_status launch_rowquant(const void* x, int dtype, long long row_stride, int rows, int cols, uint8_t* codes,
+                              float* scales, cudaStream_t stream);
+lite3r_status launch_linear_fp8(const uint8_t* x_codes, const float* x_scales, const uint8_t* w_codes,
+                                const float* w_scales, const float* bias, int rows, int d_in, int d_out, void* y,
+                                int y_dtype, long long y_stride, int* device_status, cudaStream_t stream);
+lite3r_status launch_qkv_project(const uint8_t* x_codes, const float* x_scales, const uint8_t* w_codes,
+                                 const float* w_scales, const float* bias, const lite3r_shape& s, int d_model,
+                                 const lite3r_fp8* out, int* device_status, cudaStream_t stream);
+
 lite3r_status launch_wait_expiry_probe(int* status, unsigned long long limit_ns, cudaStream_t stream);
 size_t forward_workspace_bytes(const lite3r_shape& s, const Counts& c, bool plan_inside = false);
 // byte offsets of the workspace's parts: summaries, aggregates, zeta, fp16 V, class bytes, critical lists
