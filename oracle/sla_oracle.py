@@ -322,3 +322,21 @@ def qkv_project_fp8(x, w_qkv, heads: int, bias=None):
     y = y.reshape(B, N, 3, heads, D)
     q, k, v = (np.ascontiguousarray(y[:, :, i].transpose(0, 2, 1, 3)) for i in range(3))
     return q, k, v, {"x_codes": xc, "x_scales": xs, "w_codes": wc, "w_scales": ws}
+
+
+# --------------------------------------------------------------------------- training side of proj_lin (Sec. 3.3, Eq. 3)
+def mse_distill(student: np.ndarray, teacher: np.ndarray):
+    """One module's term of the partial attention distillation loss (Eq. 3): MSE(A_student, stopgrad(A_teacher)) =
+    mean over all elements of (A_s - A_t)^2, and its gradient with respect to the student output,
+    2 (A_s - A_t) / numel.  fp64."""
+    s = np.asarray(student, dtype=np.float64)
+    t = np.asarray(teacher, dtype=np.float64)
+    d = s - t
+    return float((d * d).mean()), 2.0 * d / d.size
+
+
+def proj_lin_backward(o_lin: np.ndarray, d_out: np.ndarray) -> np.ndarray:
+    """Gradient of a loss with respect to the linear-branch projection W (the only trained tensor, Sec. 3.3
+    "selective freezing"): the output is O = O_sparse + O_lin W_h per head (Algorithm 1's last step), so
+    dL/dW_h = sum over batch and tokens of O_lin[b,h,t,:]^T dO[b,h,t,:].  o_lin, d_out: [B,H,N,D]; returns [H,D,D]."""
+    return np.einsum("bhtd,bhte->hde", np.asarray(o_lin, dtype=np.float64), np.asarray(d_out, dtype=np.float64))

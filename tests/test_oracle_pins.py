@@ -501,3 +501,43 @@ def test_qkv_projection_layout_and_identity_weight():
     y = orc.linear_fp8(ops2["x_codes"], ops2["x_scales"], ops2["w_codes"], ops2["w_scales"])
     assert np.array_equal(k2[1, 2, 5], y[1 * N + 5, H * D + 2 * D:H * D + 3 * D])
     assert np.array_equal(v2[0, 0, 18], y[18, 2 * H * D:2 * H * D + D])
+
+
+# ------------------------------------------------------------------ training side of proj_lin (Eq. 3, selective freezing)
+def test_mse_distill_against_torch_autograd():
+    g = rng(41)
+    a = torch.from_numpy(g.standard_normal((2, 3, 17, 8))).requires_grad_(True)
+    t = torch.from_numpy(g.standard_normal((2, 3, 17, 8)))
+    loss = torch.nn.functional.mse_loss(a, t)
+    loss.backward()
+    mine_loss, mine_grad = orc.mse_distill(a.detach().numpy(), t.numpy())
+    assert np.isclose(mine_loss, float(loss), rtol=1e-14)
+    assert np.allclose(mine_grad, a.grad.numpy(), rtol=1e-13, atol=0)
+    assert orc.mse_distill(t.numpy(), t.numpy())[0] == 0.0
+
+
+def test_proj_lin_gradient_by_finite_differences():
+    """dW = O_lin^T dO pinned against what it must be the derivative of: the distillation loss of the whole SLA
+    forward as a function of W, differentiated numerically (central differences) on a small problem.  The loss is
+    quadratic in W, so central differences are exact up to round-off."""
+    q, k, v, w = small_problem(42, H=2, N=70, D=4, block=16)
+    qh, kh, vh = quantized(q, k, v, 16)
+    cls = orc.classify(orc.pooled_scores(qh, kh, 16), 0.25, 0.25)
+    teacher = rng(43).standard_normal(qh.shape)
+    w = w.astype(np.float64)
+    out, o_sp, o_li = orc.sla_forward(qh, kh, vh, w, cls, 16, parts=True)
+    loss, d_out = orc.mse_distill(out, teacher)
+    dw = orc.proj_lin_backward(o_li, d_out)
+    assert dw.shape == w.shape
+    eps = 1e-4
+    for (h, i, j) in ((0, 0, 0), (1, 3, 2), (0, 2, 3), (1, 1, 1)):
+        wp, wm = w.copy(), w.copy()
+        wp[h, i, j] += eps
+        wm[h, i, j] -= eps
+        lp = orc.mse_distill(orc.sla_forward(qh, kh, vh, wp, cls, 16), teacher)[0]
+        lm = orc.mse_distill(orc.sla_forward(qh, kh, vh, wm, cls, 16), teacher)[0]
+        assert np.isclose((lp - lm) / (2 * eps), dw[h, i, j], rtol=1e-7, atol=1e-12), (h, i, j)
+    # against the library routine and a transposed-operand mistake
+    ref = torch.einsum("bhtd,bhte->hde", torch.from_numpy(o_li), torch.from_numpy(d_out)).numpy()
+    assert np.allclose(dw, ref, rtol=1e-13, atol=1e-15)
+    assert not np.allclose(dw, np.swapaxes(dw, 1, 2), rtol=1e-3, atol=1e-9)
