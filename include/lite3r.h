@@ -246,6 +246,41 @@ LITE3R_API lite3r_status lite3r_qkv_project_fp8(const unsigned char* x_codes, co
                                      lite3r_fp8 q_out, lite3r_fp8 k_out, lite3r_fp8 v_out, int* device_status,
                                      void* stream);
 
+/* ---- Training side of the linear-branch projection, the only tensor the method trains (Sec. 3.3 "selective
+ * freezing": gradients are applied only to the linear-branch projection layers; Sec. 3.5 Eq. 3). ---- */
+
+/* Bytes of scratch that cover lite3r_sla_linear_branch, lite3r_mse_distill and lite3r_proj_lin_backward for `shape`
+ * and these fractions.  Host-only. */
+LITE3R_API lite3r_status lite3r_train_workspace(const lite3r_shape* shape, double crit, double neg, size_t* bytes);
+
+/* The linear branch alone, before the projection: O_lin = (phi(q_hat) G_i) / (phi(q_hat) . zeta_i) over the marginal
+ * blocks of the given plan (Algorithm 1's feature map, KV summary, normaliser and linear output; zero where a query
+ * block has no marginal block).  The forward proper never forms it (the projection is folded into the summaries);
+ * the backward of the projection needs it.  Arguments as for lite3r_sla_forward with a plan; out may be fp32, bf16
+ * or fp16 (lite3r_proj_lin_backward takes bf16, contiguous [B, H, N, 64]).  workspace: lite3r_train_workspace() bytes. */
+LITE3R_API lite3r_status lite3r_sla_linear_branch(const lite3r_fp8* q, const lite3r_fp8* k, const lite3r_fp8* v,
+                                       const lite3r_shape* shape, lite3r_phi phi, const lite3r_plan* plan, void* out,
+                                       lite3r_dtype out_dtype, long long out_stride_b, long long out_stride_h,
+                                       long long out_stride_n, void* workspace, size_t workspace_bytes,
+                                       int* device_status, void* stream);
+
+/* One module's term of the partial attention distillation loss (Eq. 3):
+ *   *loss = mean over all `count` elements of (student - teacher)^2   (the teacher is a constant: stop-gradient),
+ *   grad  = 2 (student - teacher) / count, the gradient with respect to the student's attention output, as bf16.
+ * student, teacher: DEVICE, contiguous, fp32 or bf16 (same dtype), 16-byte aligned; count a multiple of 8.
+ * grad: DEVICE bf16 [count] or NULL; loss: DEVICE double.  The sum is accumulated in fp64 in a fixed order.
+ * workspace: DEVICE, 256-byte aligned, at least 16 KiB. */
+LITE3R_API lite3r_status lite3r_mse_distill(const void* student, const void* teacher, lite3r_dtype dtype, long long count,
+                                 void* grad, double* loss, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Gradient of the loss with respect to the projection: the output is out = sparse + O_lin @ proj[h] (Algorithm 1's
+ * last step), hence  d_proj[h] = sum over batch and tokens of O_lin[b,h,t,:]^T d_out[b,h,t,:]   ([d_in][d_out] like proj).
+ * o_lin, d_out: DEVICE bf16, contiguous [B, H, N, 64]; d_proj: DEVICE fp32 [H, 64, 64] (overwritten).
+ * A contraction over the tokens on the tensor cores (bf16 operands, fp32 accumulation), partial sums added in a fixed
+ * order.  workspace: lite3r_train_workspace() bytes. */
+LITE3R_API lite3r_status lite3r_proj_lin_backward(const void* o_lin, const void* d_out, const lite3r_shape* shape, float* d_proj,
+                                       void* workspace, size_t workspace_bytes, int* device_status, void* stream);
+
 /* Text for a status code; the last CUDA error code (cudaError_t as int) recorded by this thread. */
 LITE3R_API const char* lite3r_status_string(lite3r_status status);
 LITE3R_API int lite3r_last_cuda_error(void);

@@ -48,7 +48,8 @@ EXPORTS = ("lite3r_fp8_sizes", "lite3r_plan_sizes", "lite3r_forward_workspace", 
            "lite3r_launch_count", "lite3r_profile_enable", "lite3r_profile_stage_ms",
            "lite3r_sla_forward_static_scratch", "lite3r_quantize_fp8_qkv", "lite3r_selftest_wait_expiry",
            "lite3r_sla_forward_begin", "lite3r_sla_forward_finish", "lite3r_forward_workspace_planned",
-           "lite3r_workspace_layout", "lite3r_quantize_rows_fp8", "lite3r_linear_fp8", "lite3r_qkv_project_fp8")
+           "lite3r_workspace_layout", "lite3r_quantize_rows_fp8", "lite3r_linear_fp8", "lite3r_qkv_project_fp8",
+           "lite3r_train_workspace", "lite3r_sla_linear_branch", "lite3r_mse_distill", "lite3r_proj_lin_backward")
 STATIC_SCRATCH_BYTES = 32 << 20  # LITE3R_STATIC_SCRATCH_BYTES
 
 
@@ -101,6 +102,18 @@ def lib() -> C.CDLL:
     L.lite3r_qkv_project_fp8.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(Shape),
                                          C.c_int, Fp8, Fp8, Fp8, C.c_void_p, C.c_void_p]
     L.lite3r_qkv_project_fp8.restype = C.c_int
+    L.lite3r_train_workspace.argtypes = [C.POINTER(Shape), C.c_double, C.c_double, sz]
+    L.lite3r_train_workspace.restype = C.c_int
+    L.lite3r_sla_linear_branch.argtypes = [C.POINTER(Fp8), C.POINTER(Fp8), C.POINTER(Fp8), C.POINTER(Shape), C.c_int,
+                                           C.POINTER(Plan), C.c_void_p, C.c_int, C.c_longlong, C.c_longlong,
+                                           C.c_longlong, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+    L.lite3r_sla_linear_branch.restype = C.c_int
+    L.lite3r_mse_distill.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_longlong, C.c_void_p, C.c_void_p, C.c_void_p,
+                                     C.c_size_t, C.c_void_p]
+    L.lite3r_mse_distill.restype = C.c_int
+    L.lite3r_proj_lin_backward.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(Shape), C.c_void_p, C.c_void_p, C.c_size_t,
+                                           C.c_void_p, C.c_void_p]
+    L.lite3r_proj_lin_backward.restype = C.c_int
     L.lite3r_selftest_wait_expiry.argtypes = [C.c_void_p, C.c_ulonglong, C.c_void_p]
     L.lite3r_selftest_wait_expiry.restype = C.c_int
     L.lite3r_status_string.argtypes = [C.c_int]
@@ -382,6 +395,51 @@ def lite3r_qkv_project_fp8(x_codes, x_scales, w_codes, w_scales, bias, shape: Sh
                                         x_codes.shape[1], q_out.c_struct(), k_out.c_struct(), v_out.c_struct(),
                                         device_status.data_ptr() if device_status is not None else None,
                                         _stream_ptr(stream)), "lite3r_qkv_project_fp8")
+
+
+# ----------------------------------------------------------------------------- training side of the projection
+def lite3r_train_workspace(shape: Shape, crit: float, neg: float) -> int:
+    a = C.c_size_t()
+    _check(lib().lite3r_train_workspace(C.byref(shape), crit, neg, C.byref(a)), "lite3r_train_workspace")
+    return a.value
+
+
+def lite3r_sla_linear_branch(q: Fp8Tensor, k: Fp8Tensor, v: Fp8Tensor, shape: Shape, phi: int, plan: PlanBuffers,
+                             out: torch.Tensor, workspace: torch.Tensor, device_status=None, stream=None) -> None:
+    """O_lin (the linear branch before the projection) into `out` (CUDA fp32 / bf16 / fp16 [B,H,N,D])."""
+    out_dtype = _check_out(out, "lite3r_sla_linear_branch")
+    p = plan.c_struct()
+    qs, ks, vs = q.c_struct(), k.c_struct(), v.c_struct()
+    _check(lib().lite3r_sla_linear_branch(C.byref(qs), C.byref(ks), C.byref(vs), C.byref(shape), phi, C.byref(p),
+                                          out.data_ptr(), out_dtype, out.stride(0), out.stride(1), out.stride(2),
+                                          workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                          device_status.data_ptr() if device_status is not None else None,
+                                          _stream_ptr(stream)), "lite3r_sla_linear_branch")
+
+
+def lite3r_mse_distill(student: torch.Tensor, teacher: torch.Tensor, grad, loss: torch.Tensor, workspace: torch.Tensor,
+                       stream=None) -> None:
+    """loss (CUDA float64 [1]) = MSE(student, teacher); grad (CUDA bf16, same shape, or None) = its gradient."""
+    if student.dtype != teacher.dtype or student.dtype not in (torch.float32, torch.bfloat16):
+        raise Lite3rError("lite3r_mse_distill: student and teacher must both be float32 or bfloat16")
+    if not (student.is_contiguous() and teacher.is_contiguous()) or student.shape != teacher.shape:
+        raise Lite3rError("lite3r_mse_distill: contiguous tensors of one shape")
+    _check(lib().lite3r_mse_distill(student.data_ptr(), teacher.data_ptr(), OUT_DTYPES[student.dtype], student.numel(),
+                                    grad.data_ptr() if grad is not None else None, loss.data_ptr(), workspace.data_ptr(),
+                                    workspace.numel() * workspace.element_size(), _stream_ptr(stream)),
+           "lite3r_mse_distill")
+
+
+def lite3r_proj_lin_backward(o_lin: torch.Tensor, d_out: torch.Tensor, shape: Shape, d_proj: torch.Tensor,
+                             workspace: torch.Tensor, device_status=None, stream=None) -> None:
+    """d_proj (CUDA fp32 [H,64,64]) = sum over batch and tokens of o_lin^T d_out (both CUDA bf16 contiguous [B,H,N,64])."""
+    for t in (o_lin, d_out):
+        if t.dtype != torch.bfloat16 or not t.is_contiguous():
+            raise Lite3rError("lite3r_proj_lin_backward: o_lin and d_out must be contiguous bfloat16")
+    _check(lib().lite3r_proj_lin_backward(o_lin.data_ptr(), d_out.data_ptr(), C.byref(shape), d_proj.data_ptr(),
+                                          workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                          device_status.data_ptr() if device_status is not None else None,
+                                          _stream_ptr(stream)), "lite3r_proj_lin_backward")
 
 
 # ----------------------------------------------------------------------------- whole path

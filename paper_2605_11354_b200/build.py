@@ -14,7 +14,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 INCLUDE = os.path.join(os.path.dirname(PKG_DIR), "include")
 LIB_PATH = os.path.join(PKG_DIR, "liblite3r.so")
-SOURCES = ("api.cu", "quantize.cu", "plan.cu", "forward.cu", "summary.cu", "attention.cu", "aggregate.cu", "noalloc.cu", "linear.cu")
+SOURCES = ("api.cu", "quantize.cu", "plan.cu", "forward.cu", "summary.cu", "attention.cu", "aggregate.cu", "noalloc.cu", "linear.cu", "train.cu")
 NVCC_FLAGS = ("-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr")
 

@@ -1,4 +1,5 @@
 // C-ABI entry points of the lite3r library: argument validation, size queries and dispatch.
+#include <algorithm>
 #include <atomic>
 #include <cmath>
 #include <mutex>
@@ -127,6 +128,21 @@ lite3r_status make_tensor_map_2d(CUtensorMap* map, CUtensorMapDataType type, int
   const cuuint32_t box[2] = {box_inner, box_rows};
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = fn(map, type, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? LITE3R_OK : LITE3R_ERR_CUDA;
+}
+
+lite3r_status make_tensor_map_3d(CUtensorMap* map, CUtensorMapDataType type, int elem_bytes, const void* base,
+                                 uint64_t inner, uint64_t rows, uint64_t planes, uint32_t box_inner, uint32_t box_rows,
+                                 CUtensorMapSwizzle swizzle) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return LITE3R_ERR_CUDA;
+  const cuuint64_t dims[3] = {inner, rows, planes};
+  const cuuint64_t strides[2] = {inner * static_cast<cuuint64_t>(elem_bytes),
+                                 inner * rows * static_cast<cuuint64_t>(elem_bytes)};
+  const cuuint32_t box[3] = {box_inner, box_rows, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = fn(map, type, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                         swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? LITE3R_OK : LITE3R_ERR_CUDA;
 }
@@ -286,7 +302,7 @@ static lite3r_status forward_phases(int phases, const lite3r_fp8* q, const lite3
                                     double crit, double neg, lite3r_phi phi, const lite3r_plan* plan, void* out,
                                     lite3r_dtype out_dtype, long long out_stride_b, long long out_stride_h,
                                     long long out_stride_n, void* workspace, size_t workspace_bytes,
-                                    int* device_status, void* stream) {
+                                    int* device_status, void* stream, int linear_only = 0) {
   lite3r_status st = check_shape(shape);
   if (st != LITE3R_OK) return st;
   if ((st = check_fp8(k, true, false)) != LITE3R_OK) return st;
@@ -338,6 +354,7 @@ static lite3r_status forward_phases(int phases, const lite3r_fp8* q, const lite3
   a.phi = static_cast<int>(phi);
   a.plan = effective;
   a.plan_inside = plan_inside ? 1 : 0;
+  a.linear_only = linear_only;
   a.crit = crit;
   a.neg = neg;
   a.out = out;
@@ -380,6 +397,62 @@ lite3r_status lite3r_sla_forward_finish(const lite3r_fp8* q, const lite3r_fp8* k
   if (plan == nullptr) return LITE3R_ERR_INVALID_ARG;
   return forward_phases(2, q, k, v, nullptr, 0, shape, 0.0, 0.0, phi, plan, out, out_dtype, out_stride_b,
                         out_stride_h, out_stride_n, workspace, workspace_bytes, device_status, stream);
+}
+
+lite3r_status lite3r_train_workspace(const lite3r_shape* shape, double crit, double neg, size_t* bytes) {
+  size_t fwd = 0;
+  lite3r_status st = workspace_query(shape, crit, neg, false, &fwd);
+  if (st != LITE3R_OK) return st;
+  *bytes = std::max(fwd + kHeadDim * kHeadDim * sizeof(float), train_workspace_bytes(*shape));
+  return LITE3R_OK;
+}
+
+lite3r_status lite3r_sla_linear_branch(const lite3r_fp8* q, const lite3r_fp8* k, const lite3r_fp8* v,
+                                       const lite3r_shape* shape, lite3r_phi phi, const lite3r_plan* plan, void* out,
+                                       lite3r_dtype out_dtype, long long out_stride_b, long long out_stride_h,
+                                       long long out_stride_n, void* workspace, size_t workspace_bytes,
+                                       int* device_status, void* stream) {
+  lite3r_status st = check_shape(shape);
+  if (st != LITE3R_OK) return st;
+  if (plan == nullptr || workspace == nullptr || !aligned(workspace, 256)) return LITE3R_ERR_INVALID_ARG;
+  const size_t fwd = forward_workspace_bytes(*shape, Counts{plan->k_crit, plan->k_marg, plan->k_neg});
+  if (workspace_bytes < fwd + kHeadDim * kHeadDim * sizeof(float)) return LITE3R_ERR_WORKSPACE;
+  if ((st = check_device()) != LITE3R_OK) return st;
+  // the projection is left out by running the forward with the identity in its place (exact in every format used)
+  float* identity = reinterpret_cast<float*>(static_cast<char*>(workspace) + fwd);
+  if ((st = launch_fill_identity(identity, static_cast<cudaStream_t>(stream))) != LITE3R_OK) return st;
+  return forward_phases(3, q, k, v, identity, 0, shape, 0.0, 0.0, phi, plan, out, out_dtype, out_stride_b, out_stride_h,
+                        out_stride_n, workspace, fwd, device_status, stream, 1);
+}
+
+lite3r_status lite3r_mse_distill(const void* student, const void* teacher, lite3r_dtype dtype, long long count,
+                                 void* grad, double* loss, void* workspace, size_t workspace_bytes, void* stream) {
+  if (student == nullptr || teacher == nullptr || loss == nullptr || workspace == nullptr || count <= 0)
+    return LITE3R_ERR_INVALID_ARG;
+  if (dtype != LITE3R_F32 && dtype != LITE3R_BF16) return LITE3R_ERR_UNSUPPORTED;
+  if ((count % 8) || !aligned(student, 16) || !aligned(teacher, 16) || (grad != nullptr && !aligned(grad, 16)) ||
+      !aligned(loss, 8) || !aligned(workspace, 256))
+    return LITE3R_ERR_INVALID_ARG;
+  if (workspace_bytes < 2048 * sizeof(double)) return LITE3R_ERR_WORKSPACE;
+  lite3r_status st = check_device();
+  if (st != LITE3R_OK) return st;
+  return launch_mse_distill(student, teacher, static_cast<int>(dtype), static_cast<size_t>(count),
+                            static_cast<__nv_bfloat16*>(grad), loss, static_cast<double*>(workspace),
+                            static_cast<cudaStream_t>(stream));
+}
+
+lite3r_status lite3r_proj_lin_backward(const void* o_lin, const void* d_out, const lite3r_shape* shape, float* d_proj,
+                                       void* workspace, size_t workspace_bytes, int* device_status, void* stream) {
+  lite3r_status st = check_shape(shape);
+  if (st != LITE3R_OK) return st;
+  if (o_lin == nullptr || d_out == nullptr || d_proj == nullptr || workspace == nullptr) return LITE3R_ERR_INVALID_ARG;
+  if (!aligned(o_lin, 16) || !aligned(d_out, 16) || !aligned(d_proj, 16) || !aligned(workspace, 256)) return LITE3R_ERR_INVALID_ARG;
+  if (workspace_bytes < train_workspace_bytes(*shape)) return LITE3R_ERR_WORKSPACE;
+  if ((st = check_device()) != LITE3R_OK) return st;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  if (device_status != nullptr && (st = record_cuda(cudaMemsetAsync(device_status, 0, sizeof(int), cs))) != LITE3R_OK) return st;
+  return launch_proj_lin_backward(static_cast<const __nv_bfloat16*>(o_lin), static_cast<const __nv_bfloat16*>(d_out), *shape,
+                                  d_proj, static_cast<float*>(workspace), device_status, cs);
 }
 
 lite3r_status lite3r_workspace_layout(const lite3r_shape* shape, double crit, double neg, int plan_inside,

@@ -95,6 +95,7 @@ struct ForwardArgs {
   void* out;
   int out_dtype;
   long long out_stride_b, out_stride_h, out_stride_n;
+  int linear_only;      // 1: the sparse branch is left out (the output is the linear branch through proj alone)
   int plan_inside;      // 1: the plan is built in the workspace from q/k column sums and the fractions below
   double crit, neg;
   void* workspace;
@@ -144,6 +145,20 @@ lite3r_status launch_linear_fp8(const uint8_t* x_codes, const float* x_scales, c
 lite3r_status launch_qkv_project(const uint8_t* x_codes, const float* x_scales, const uint8_t* w_codes,
                                  const float* w_scales, const float* bias, const lite3r_shape& s, int d_model,
                                  const lite3r_fp8* out, int* device_status, cudaStream_t stream);
+
+// The same for a 3-D tensor [planes][rows][inner] with a box of box_inner x box_rows x 1 (rows past the end of a plane
+// are zero-filled, so a tile never runs into the next plane).
+lite3r_status make_tensor_map_3d(CUtensorMap* map, CUtensorMapDataType type, int elem_bytes, const void* base,
+                                 uint64_t inner, uint64_t rows, uint64_t planes, uint32_t box_inner, uint32_t box_rows,
+                                 CUtensorMapSwizzle swizzle);
+
+// Training side of the linear-branch projection (train.cu).
+size_t train_workspace_bytes(const lite3r_shape& s);
+lite3r_status launch_fill_identity(float* dst, cudaStream_t stream);
+lite3r_status launch_mse_distill(const void* student, const void* teacher, int dtype, size_t count, __nv_bfloat16* grad,
+                                 double* loss, double* partials, cudaStream_t stream);
+lite3r_status launch_proj_lin_backward(const __nv_bfloat16* o_lin, const __nv_bfloat16* d_out, const lite3r_shape& s,
+                                       float* d_w, float* partials, int* device_status, cudaStream_t stream);
 
 lite3r_status launch_wait_expiry_probe(int* status, unsigned long long limit_ns, cudaStream_t stream);
 size_t forward_workspace_bytes(const lite3r_shape& s, const Counts& c, bool plan_inside = false);

@@ -118,7 +118,7 @@ lite3r_status run_forward(const ForwardArgs& a, int phases, cudaStream_t stream)
   // With a linear branch the summary kernel reads every V row anyway and writes the fp16 operand on the way; the
   // stand-alone pass runs only when there is no linear branch.
   const bool v16_from_summary = a.plan.k_marg > 0;
-  if ((phases & 1) && a.plan.k_crit > 0 && !v16_from_summary) {
+  if ((phases & 1) && a.plan.k_crit > 0 && !v16_from_summary && !a.linear_only) {
     const size_t words = static_cast<size_t>(rows) * BS * kHeadDim / 16;  // 16 codes per thread and pass
     int sms = 0;
     if ((st = sm_count(&sms)) != LITE3R_OK) return st;
@@ -151,7 +151,7 @@ lite3r_status run_forward(const ForwardArgs& a, int phases, cudaStream_t stream)
   att.g16 = w.g16;
   att.zeta = w.zeta;
   att.crit_idx = plan.crit_idx;
-  att.k_crit = a.plan.k_crit;
+  att.k_crit = a.linear_only ? 0 : a.plan.k_crit;
   att.k_marg = a.plan.k_marg;
   att.phi = a.phi;
   att.out = a.out;

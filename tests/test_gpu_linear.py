@@ -135,3 +135,31 @@ def test_fused_qkv_projection_against_the_oracle(block, tokens, batch, heads, d_
     ref_out = orc.sla_forward(qh, kh, vh, proj.cpu().numpy(), eng.plan.cls.cpu().numpy(), block)
     rel, mx = pu.output_errors(out.cpu().numpy(), ref_out)
     assert rel <= pu.REL_L2_TOL and mx <= pu.MAX_ABS_TOL * max(1.0, float(np.abs(ref_out).max()))
+
+
+def test_attention_output_requantised_for_the_out_projection():
+    """The step after the attention: its output, written token-major in bf16 ([B, N, H*64] seen as [B, H, N, 64]), is
+    quantised per token for the attention block's output projection and multiplied by the e4m3 weight (Algorithm 2
+    again).  Codes and scales are bit-exact for the bf16 values the forward stored; the product matches the oracle."""
+    from test_gpu_parity import small_workload
+    wl = small_workload("requant", tokens=500, heads=4, batch=2)
+    inputs = wk.make_inputs(wl)
+    eng, _ = pu.run_gpu(inputs, wl)
+    proj = torch.from_numpy(inputs["proj"]).cuda()
+    buf = torch.empty((wl.batch, wl.tokens, wl.heads, 64), dtype=torch.bfloat16, device="cuda")
+    eng.forward(proj, out=buf.permute(0, 2, 1, 3))
+    a = buf.view(wl.batch * wl.tokens, wl.heads * 64)
+    ac, asc = lt.lite3r_quantize_rows_fp8(a)
+    g = np.random.default_rng(11)
+    w = (g.standard_normal((256, 256)) / 16).astype(np.float32)
+    wc, ws = lt.lite3r_quantize_rows_fp8(torch.from_numpy(w).cuda())
+    y = torch.empty((a.shape[0], 256), device="cuda")
+    lt.lite3r_linear_fp8(ac, asc, wc, ws, None, y, eng.status)
+    torch.cuda.synchronize()
+    assert int(eng.status.item()) == 0
+    a_np = a.float().cpu().numpy()
+    rc, rs = orc.quantize_fp8_rows(a_np)
+    assert np.array_equal(ac.cpu().numpy(), rc) and np.array_equal(asc.cpu().numpy(), rs)
+    rwc, rws = orc.quantize_fp8_rows(w)
+    ref = orc.linear_fp8(rc, rs, rwc, rws)
+    assert np.abs(y.cpu().numpy() - ref).max() <= 1e-5 * np.abs(ref).max()
