@@ -472,3 +472,27 @@ def test_large_and_small_magnitudes(phi, vscale, kscale):
     assert np.isfinite(got).all()
     rel, mx = pu.output_errors(got, ref["out"])
     assert rel <= pu.REL_L2_TOL and mx <= pu.MAX_ABS_TOL * max(1.0, vscale)
+
+
+def test_step_replayed_as_a_cuda_graph():
+    """SlaForward.run_graph (one captured step) gives the bits of the stream-ordered run, on replay after replay and
+    after new values were written into the captured source tensors."""
+    wl = small_workload("graph", tokens=3 * 1374, heads=4, batch=2)
+    inputs = wk.make_inputs(wl)
+    eng, expected = pu.run_gpu(inputs, wl)
+    expected = expected.clone()
+    q, k, v = (pu.to_device(inputs[n], wl.src_dtype) for n in ("q", "k", "v"))
+    proj = torch.from_numpy(inputs["proj"]).cuda()
+    for _ in range(3):
+        eng.out.fill_(float("nan"))
+        out = eng.run_graph(q, k, v, proj)
+        torch.cuda.synchronize()
+        assert int(eng.status.item()) == 0 and torch.equal(out, expected)
+    other = wk.make_inputs(small_workload("graph2", tokens=3 * 1374, heads=4, batch=2, cfg_id=92))
+    for n, t in (("q", q), ("k", k), ("v", v)):
+        t.copy_(pu.to_device(other[n], wl.src_dtype))
+    out = eng.run_graph(q, k, v, proj).clone()
+    torch.cuda.synchronize()
+    ref = eng.run(q, k, v, proj)
+    torch.cuda.synchronize()
+    assert torch.equal(out, ref) and not torch.equal(out, expected)
