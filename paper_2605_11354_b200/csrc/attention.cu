@@ -537,24 +537,31 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         ok = mbar_wait_far(&bars->k_free[u % kStages], (u / kStages) & 1, abort_flag, p.status, 310);
       const uint8_t* qrow = smem + kOffQ + p_row * 64;
       const int qswz = (p_row >> 1) & 3;
-      float mxq[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      // phi = softmax over the components: any common shift of the exponents cancels in the ratio numerator /
+      // denominator.  448 * scale bounds every component of the block, so it serves as the shift without a pass over
+      // the row; only when exponents could then leave the fp32 range (block magnitudes in the hundreds) is the row's
+      // own maximum looked up.
+      const bool phi_softmax = p.phi == LITE3R_PHI_SOFTMAX;
+      const float cq = sq * kLog2e;
+      float shift = 448.f * cq;
+      if (phi_softmax && 896.f * cq > 100.f) {
+        float mxq[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll 1
-      for (int c4 = 0; c4 < 4; ++c4) {  // row maximum over the 64 components
-        const uint4 raw = *reinterpret_cast<const uint4*>(qrow + ((c4 ^ qswz) << 4));
-        const uint32_t words[4] = {raw.x, raw.y, raw.z, raw.w};
+        for (int c4 = 0; c4 < 4; ++c4) {  // row maximum over the 64 components
+          const uint4 raw = *reinterpret_cast<const uint4*>(qrow + ((c4 ^ qswz) << 4));
+          const uint32_t words[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-        for (int xw = 0; xw < 4; ++xw) {
-          float fv[4];
-          e4m3x4_to_float(words[xw], fv);
+          for (int xw = 0; xw < 4; ++xw) {
+            float fv[4];
+            e4m3x4_to_float(words[xw], fv);
 #pragma unroll
-          for (int y = 0; y < 4; ++y) mxq[y] = fmaxf(mxq[y], fv[y]);
+            for (int y = 0; y < 4; ++y) mxq[y] = fmaxf(mxq[y], fv[y]);
+          }
         }
+        shift = fmaxf(fmaxf(mxq[0], mxq[1]), fmaxf(mxq[2], mxq[3])) * cq;  // sq > 0 commutes with max
       }
-      const float mx = fmaxf(fmaxf(mxq[0], mxq[1]), fmaxf(mxq[2], mxq[3]));
-      const float cq = sq * kLog2e, shift = mx * cq;  // sq > 0 commutes with max
       uint8_t* const phirow = smem + kOffPhi + p_row * 128;
       float den4[4] = {0.f, 0.f, 0.f, 0.f};
-      const bool phi_softmax = p.phi == LITE3R_PHI_SOFTMAX;
 #pragma unroll 1
       for (int cc = 0; cc < 2; ++cc) {  // this warpgroup's two chunks of 16 components
         const int c4 = 2 * w + cc;
