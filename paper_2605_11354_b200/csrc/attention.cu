@@ -60,7 +60,8 @@ constexpr uint32_t kOffV = kOffK + kStages * kKStage;
 constexpr uint32_t kOffZeta = kOffV + kStages * kVStage;  // zeta_i of the linear branch (256 B per query block)
 constexpr uint32_t kOffRef = kOffZeta + 512;              // per row: {reference maximum, number of steps published}
 constexpr uint32_t kOffX = kOffRef + 1024;                // epilogue exchange between the warpgroups (2 x 128 x 8 B)
-constexpr uint32_t kOffBar = kOffX + 2048;
+constexpr uint32_t kOffScal = kOffX + 2048;               // per step and query block: {exponent factor, valid keys}, ring of 8
+constexpr uint32_t kOffBar = kOffScal + 128;
 constexpr uint32_t kSmemBytes = kOffBar + 512;  // two CTAs per SM: 2 * (110592 + 1024 reserved) <= 232448
 // after the main loop the rings are reused: aggregated summaries G_i in K stages 0-1 (16 KB), the phi(Q) operand in
 // K stages 2-3 (16 KB), the output rows in the V ring (32 KB)
@@ -241,37 +242,57 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   setmaxnreg_dec<kCtrlRegs>();
   if (warp == 0) {
     // ------------------------------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      tma_prefetch_desc(&map_q);
-      tma_prefetch_desc(&map_k);
-      tma_prefetch_desc(&map_v);
-      mbar_arrive_expect_tx(&bars->q_full, kQBytes);
-      if (kPair) {
-        tma_load_2d(smem + kOffQ, &map_q, &bars->q_full, 0, static_cast<int>((bh_rows + i_q[0]) * 64));
-        tma_load_2d(smem + kOffQ + 4096, &map_q, &bars->q_full, 0, static_cast<int>((bh_rows + i_q[1]) * 64));
-      } else {
-        tma_load_2d(smem + kOffQ, &map_q, &bars->q_full, 0, static_cast<int>((bh_rows + i_q[0]) * 128));
-        tma_load_2d(smem + kOffQ + 4096, &map_q, &bars->q_full, 0, static_cast<int>((bh_rows + i_q[0]) * 128 + 64));
-      }
-      if (p.k_marg > 0) {  // the denominators of the linear branch have a place of their own: fetched right away
-        mbar_arrive_expect_tx(&bars->z_full, kHalves * 256);
-        for (int hf = 0; hf < kHalves; ++hf)
-          bulk_load(smem + kOffZeta + hf * 256, p.zeta + (bh_rows + i_q[hf]) * kHeadDim, 256, &bars->z_full);
+    // All 32 lanes run the loops and the waits, so that control flow, step counters and addresses are the same in every
+    // lane (the compiler can then keep them in the warp's uniform registers, which is where TMA and tcgen05
+    // instructions take their operands from); one elected lane issues.
+    {
+      const bool leader = elect_one();
+      if (leader) {
+        tma_prefetch_desc(&map_q);
+        tma_prefetch_desc(&map_k);
+        tma_prefetch_desc(&map_v);
+        mbar_arrive_expect_tx(&bars->q_full, kQBytes);
+        if (kPair) {
+          tma_load_2d(smem + kOffQ, &map_q, &bars->q_full, 0, static_cast<int>((bh_rows + i_q[0]) * 64));
+          tma_load_2d(smem + kOffQ + 4096, &map_q, &bars->q_full, 0, static_cast<int>((bh_rows + i_q[1]) * 64));
+        } else {
+          tma_load_2d(smem + kOffQ, &map_q, &bars->q_full, 0, static_cast<int>((bh_rows + i_q[0]) * 128));
+          tma_load_2d(smem + kOffQ + 4096, &map_q, &bars->q_full, 0, static_cast<int>((bh_rows + i_q[0]) * 128 + 64));
+        }
+        if (p.k_marg > 0) {  // the denominators of the linear branch have a place of their own: fetched right away
+          mbar_arrive_expect_tx(&bars->z_full, kHalves * 256);
+          for (int hf = 0; hf < kHalves; ++hf)
+            bulk_load(smem + kOffZeta + hf * 256, p.zeta + (bh_rows + i_q[hf]) * kHeadDim, 256, &bars->z_full);
+        }
       }
       const int* list0 = p.crit_idx + (bh_rows + i_q[0]) * p.k_crit;
       const int* list1 = p.crit_idx + (bh_rows + i_q[1]) * p.k_crit;
-      // tile row (in the code tensors) of step t for query block hf
-      auto tile_row = [&](int t, int hf) {
-        if (kPair) return static_cast<int>((bh_rows + ldg_pinned((hf ? list1 : list0) + t)) * 64);
-        return static_cast<int>((bh_rows + ldg_pinned(list0 + t / 2)) * 128 + (t & 1) * 64);
+      const float sq0 = __ldg(p.q_scales + bh_rows + i_q[0]) * (kLog2e * 0.125f);
+      const float sq1 = __ldg(p.q_scales + bh_rows + i_q[1]) * (kLog2e * 0.125f);
+      // key block of step t for query block hf
+      auto key_block = [&](int t, int hf) {
+        if (kPair) return ldg_pinned((hf ? list1 : list0) + t);
+        return ldg_pinned(list0 + t / 2);
+      };
+      // tile row (in the code tensors) of a step in key block j
+      auto tile_row = [&](int t, int j) {
+        if (kPair) return static_cast<int>((bh_rows + j) * 64);
+        return static_cast<int>((bh_rows + j) * 128 + (t & 1) * 64);
       };
       // The K cursor runs one step ahead of the V cursor (a K stage is free after the Q K^T of four steps earlier,
       // a V stage only after that step's P V, and Q K^T of step t is issued before P V of step t-1).  The events the
-      // two cursors wait for alternate in time in exactly this order, so blocking waits lose nothing.  The tile rows
-      // of each cursor's next step are fetched one step ahead.
-      int rk[2] = {0, 0}, rv[2] = {0, 0};
+      // two cursors wait for alternate in time in exactly this order, so blocking waits lose nothing.  The key block
+      // of the K cursor's next step and its scale are fetched one step ahead.  Together with the K tile of a step
+      // the producer leaves the step's scalars for the softmax threads: the factor that turns a raw score into a
+      // base-2 exponent and the number of valid keys (ring of eight: the slot of step t is rewritten for step t+8,
+      // when the softmax threads of step t+2 have long released the scores, which they read after the scalars).
+      int jk[2] = {0, 0}, jv[2] = {0, 0};
+      float sk[2] = {0.f, 0.f};
       if (steps > 0) {
-        for (int hf = 0; hf < kHalves; ++hf) rk[hf] = rv[hf] = tile_row(0, hf);
+        for (int hf = 0; hf < kHalves; ++hf) {
+          jk[hf] = jv[hf] = key_block(0, hf);
+          sk[hf] = ldg_pinned(p.k_scales + bh_rows + jk[hf]);
+        }
       }
       bool ok = true;
       for (int i = 0; ok && i <= steps; ++i) {
@@ -279,25 +300,38 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         if (tk < steps) {
           const int st = tk % kStages;
           if (tk >= kStages)
-            ok = mbar_wait(&bars->k_free[st], ((tk - kStages) / kStages) & 1, abort_flag, p.status, 101, kBackoffNs);
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars->k_free[st], ((tk - kStages) / kStages) & 1, abort_flag, p.status, 101, kBackoffNs));
           if (!ok) break;
-          mbar_arrive_expect_tx(&bars->k_full[st], kKTx);
-          for (int hf = 0; hf < kHalves; ++hf)
-            tma_load_2d(smem + kOffK + st * kKStage + hf * 4096, &map_k, &bars->k_full[st], 0, rk[hf]);
+          if (leader) {
+            for (int hf = 0; hf < kHalves; ++hf) {
+              int valid = p.tokens - jk[hf] * BS - (kPair ? 0 : (tk & 1) * kStepKeys);
+              valid = max(0, min(kStepKeys, valid));
+              sts_volatile_v2(smem_u32(smem + kOffScal) + (tk & 7) * 16 + hf * 8,
+                              __float_as_uint((hf ? sq1 : sq0) * sk[hf]), static_cast<uint32_t>(valid));
+            }
+            mbar_arrive_expect_tx(&bars->k_full[st], kKTx);
+            for (int hf = 0; hf < kHalves; ++hf)
+              tma_load_2d(smem + kOffK + st * kKStage + hf * 4096, &map_k, &bars->k_full[st], 0, tile_row(tk, jk[hf]));
+          }
           if (tk + 1 < steps) {
-            for (int hf = 0; hf < kHalves; ++hf) rk[hf] = tile_row(tk + 1, hf);
+            for (int hf = 0; hf < kHalves; ++hf) {
+              jk[hf] = key_block(tk + 1, hf);
+              sk[hf] = ldg_pinned(p.k_scales + bh_rows + jk[hf]);
+            }
           }
         }
         if (tv >= 0) {
           const int st = tv % kStages;
           if (tv >= kStages)
-            ok = mbar_wait(&bars->pv_done[st], ((tv - kStages) / kStages) & 1, abort_flag, p.status, 102, kBackoffNs);
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars->pv_done[st], ((tv - kStages) / kStages) & 1, abort_flag, p.status, 102, kBackoffNs));
           if (!ok) break;
-          mbar_arrive_expect_tx(&bars->v_full[st], kVTx);
-          for (int hf = 0; hf < kHalves; ++hf)
-            tma_load_2d(smem + kOffV + st * kVStage + hf * 8192, &map_v, &bars->v_full[st], 0, rv[hf]);
+          if (leader) {
+            mbar_arrive_expect_tx(&bars->v_full[st], kVTx);
+            for (int hf = 0; hf < kHalves; ++hf)
+              tma_load_2d(smem + kOffV + st * kVStage + hf * 8192, &map_v, &bars->v_full[st], 0, tile_row(tv, jv[hf]));
+          }
           if (tv + 1 < steps) {
-            for (int hf = 0; hf < kHalves; ++hf) rv[hf] = tile_row(tv + 1, hf);
+            for (int hf = 0; hf < kHalves; ++hf) jv[hf] = key_block(tv + 1, hf);
           }
         }
       }
@@ -305,8 +339,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         // The aggregated summaries go to K stages 0 and 1, which are free once the last Q K^T products have
         // completed: well before the last P V products, so this load is off the tail's critical path.
         for (int u = max(0, steps - kStages); u < steps && ok; ++u)
-          ok = mbar_wait(&bars->k_free[u % kStages], (u / kStages) & 1, abort_flag, p.status, 103, kBackoffNs);
-        if (ok) {
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars->k_free[u % kStages], (u / kStages) & 1, abort_flag, p.status, 103, kBackoffNs));
+        if (ok && leader) {
           mbar_arrive_expect_tx(&bars->g_full, kHalves * 8192);
           for (int hf = 0; hf < kHalves; ++hf)
             tma_load_2d(smem + kOffG + hf * 8192, &map_g, &bars->g_full, 0, static_cast<int>((bh_rows + i_q[hf]) * 64));
@@ -316,15 +350,17 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   } else if (warp == 1) {
     // ------------------------------------------------------------------------------------------ Q K^T issuer
     // One thread issues a small tcgen05.mma about every 55 clocks and pays some 100 clocks per barrier it looks
-    // at, so the two products of a step have an issuing thread each (this warp and the next); a single issuer for
+    // at, so the two products of a step have an issuing warp each (this one and the next); a single issuer for
     // both was measured to be the bottleneck of the whole kernel.  Operand descriptors are built once and advanced by
-    // adding byte offsets (in 16-byte units) to their address field.
-    if (lane == 0) {
+    // adding byte offsets (in 16-byte units) to their address field.  As in the producer, all lanes run the loop
+    // and one elected lane issues.
+    {
+      const bool leader = elect_one();
       constexpr uint32_t idesc_qk = instr_desc(0, kM, 64, 0, 0);   // e4m3 x e4m3, both K-major
       constexpr uint32_t idesc_lin = instr_desc(1, kM, 64, 0, 0);  // bf16 x bf16, both K-major
       const uint32_t q_addr = smem_u32(smem + kOffQ);
       const uint64_t k_desc0 = smem_desc(smem_u32(smem + kOffK), 16, 512, kSwizzle64);
-      bool ok = mbar_wait(&bars->q_full, 0, abort_flag, p.status, 201, kBackoffNs);
+      bool ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars->q_full, 0, abort_flag, p.status, 201, kBackoffNs));
       uint64_t q_desc[2][kHalves];
 #pragma unroll
       for (int kk = 0; kk < 2; ++kk)
@@ -338,41 +374,48 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         ok = mbar_wait(&bars->k_full[st], (t / kStages) & 1, abort_flag, p.status, 202, kBackoffNs);
         if (ok && t >= 2)
           ok = mbar_wait(&bars->s_empty[t & 1], ((t - 2) >> 1) & 1, abort_flag, p.status, 203, kBackoffNs);
+        ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
         const uint32_t s_tmem = tmem + kColS + (t & 1) * 64;
         const uint64_t k_desc = k_desc0 + static_cast<uint64_t>((st * kKStage) >> 4);
         tc_fence_after();
+        if (leader) {
 #pragma unroll
-        for (int kk = 0; kk < 2; ++kk) {
+          for (int kk = 0; kk < 2; ++kk) {
 #pragma unroll
-          for (int hf = 0; hf < kHalves; ++hf)
-            mma_f8(s_tmem + ((hf * 16u) << 16), q_desc[kk][hf], k_desc + ((hf * 4096 + kk * 32) >> 4), idesc_qk, kk);
+            for (int hf = 0; hf < kHalves; ++hf)
+              mma_f8(s_tmem + ((hf * 16u) << 16), q_desc[kk][hf], k_desc + ((hf * 4096 + kk * 32) >> 4), idesc_qk, kk);
+          }
+          mma_commit(&bars->qk_done[t & 1]);
+          mma_commit(&bars->k_free[st]);
         }
-        mma_commit(&bars->qk_done[t & 1]);
-        mma_commit(&bars->k_free[st]);
       }
       if (ok && p.k_marg > 0) {
         ok = mbar_wait(&bars->g_full, 0, abort_flag, p.status, 206, kBackoffNs) &&
              mbar_wait(&bars->phi_full, 0, abort_flag, p.status, 207, kBackoffNs);
+        ok = __all_sync(0xFFFFFFFFu, ok);
         if (ok) {
           tc_fence_after();
           const uint32_t phi_addr = smem_u32(smem + kOffPhi), g_addr = smem_u32(smem + kOffG);
+          if (leader) {
 #pragma unroll
-          for (int kk = 0; kk < 4; ++kk) {
+            for (int kk = 0; kk < 4; ++kk) {
 #pragma unroll
-            for (int hf = 0; hf < kHalves; ++hf) {
-              const uint64_t a = smem_desc(phi_addr + (kPair ? hf * 8192 : 0) + kk * 32, 16, 1024, kSwizzle128);
-              const uint64_t bd = smem_desc(g_addr + hf * 8192 + kk * 32, 16, 1024, kSwizzle128);
-              mma_f16(tmem + kColL + ((hf * 16u) << 16), a, bd, idesc_lin, kk);
+              for (int hf = 0; hf < kHalves; ++hf) {
+                const uint64_t a = smem_desc(phi_addr + (kPair ? hf * 8192 : 0) + kk * 32, 16, 1024, kSwizzle128);
+                const uint64_t bd = smem_desc(g_addr + hf * 8192 + kk * 32, 16, 1024, kSwizzle128);
+                mma_f16(tmem + kColL + ((hf * 16u) << 16), a, bd, idesc_lin, kk);
+              }
             }
+            mma_commit(&bars->l_full);
           }
-          mma_commit(&bars->l_full);
         }
       }
     }
   } else if (warp == 2) {
     // ------------------------------------------------------------------------------------------ P V issuer
-    if (lane == 0) {
+    {
+      const bool leader = elect_one();
       constexpr uint32_t idesc_pv = instr_desc(0, kM, 64, 0, 1);  // f16 x f16, P from TMEM, V MN-major
       const uint64_t v_desc0 = smem_desc(smem_u32(smem + kOffV), 8192, 1024, kSwizzle128);
       const uint32_t o_tmem = tmem + kColO;
@@ -381,18 +424,21 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const int st = t % kStages;
         ok = mbar_wait(&bars->v_full[st], (t / kStages) & 1, abort_flag, p.status, 205, kBackoffNs) &&
              mbar_wait(&bars->p_full[t & 1], (t >> 1) & 1, abort_flag, p.status, 204, kBackoffNs);
+        ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
         const uint32_t p_tmem = tmem + kColP + (t & 1) * 32;
         const uint64_t v_desc = v_desc0 + static_cast<uint64_t>((st * kVStage) >> 4);
         tc_fence_after();
+        if (leader) {
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
+          for (int kk = 0; kk < 4; ++kk) {
 #pragma unroll
-          for (int hf = 0; hf < kHalves; ++hf)
-            mma_f16_ts(o_tmem + ((hf * 16u) << 16), p_tmem + ((hf * 16u) << 16) + kk * 8,
-                       v_desc + ((hf * 8192 + kk * 2048) >> 4), idesc_pv, (t > 0 || kk > 0) ? 1u : 0u);
+            for (int hf = 0; hf < kHalves; ++hf)
+              mma_f16_ts(o_tmem + ((hf * 16u) << 16), p_tmem + ((hf * 16u) << 16) + kk * 8,
+                         v_desc + ((hf * 8192 + kk * 2048) >> 4), idesc_pv, (t > 0 || kk > 0) ? 1u : 0u);
+          }
+          mma_commit(&bars->pv_done[st]);
         }
-        mma_commit(&bars->pv_done[st]);
       }
     }
   }
@@ -409,8 +455,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const uint32_t lane_addr = tmem + ((static_cast<uint32_t>(quarter) * 32u) << 16);
     const uint32_t s_addr = lane_addr + kColS + w * 64, p_addr = lane_addr + kColP + w * 32, o_addr = lane_addr + kColO;
     const float sq = __ldg(p.q_scales + q_tile);
-    const float qk_scale = sq * (kLog2e * 0.125f);
-    const int* list = p.crit_idx + q_tile * p.k_crit;
+    const uint32_t scal_slot = smem_u32(smem + kOffScal) + hf * 8;
     const uint32_t ref_slot = smem_u32(smem + kOffRef) + p_row * 8;
 
     float m_seen = kNoMax, l = 0.f;  // reference this warpgroup's row sum is relative to; the row sum
@@ -425,23 +470,19 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       return true;
     };
 
-    // per-step scalars: the key-block index is fetched two of the warpgroup's steps ahead and its scale one ahead, so
-    // that no load in the loop waits for the address produced by another load of the same iteration
-    int j_cur = w < steps ? ldg_pinned(list + w / kStepsPerBlock) : 0;
-    int j_nxt = w + 2 < steps ? ldg_pinned(list + (w + 2) / kStepsPerBlock) : 0;
-    float sk_cur = w < steps ? ldg_pinned(p.k_scales + bh_rows + j_cur) : 0.f;
+    // barrier of the P V product two steps back (the one that frees P[w]): its stage alternates between w and w + 2,
+    // its parity flips every second iteration; both are carried along instead of being recomputed from t
+    uint64_t* const pv_bar0 = &bars->pv_done[w];
+    uint32_t pv_off = 0, pv_par = 0, pv_flip = 0, qk_par = 0;
 
     for (int t = w; t < steps; t += 2) {
-      const int j = j_cur;
-      const float c = qk_scale * sk_cur;
-      j_cur = j_nxt;
-      if (t + 2 < steps) sk_cur = ldg_pinned(p.k_scales + bh_rows + j_nxt);
-      if (t + 4 < steps) j_nxt = ldg_pinned(list + (t + 4) / kStepsPerBlock);
-      int valid = p.tokens - j * BS - (kPair ? 0 : (t & 1) * kStepKeys);
-      valid = max(0, min(kStepKeys, valid));
-
-      if (!(ok = mbar_wait_far(&bars->qk_done[w], (t >> 1) & 1, abort_flag, p.status, 301))) break;
+      if (!(ok = mbar_wait_far(&bars->qk_done[w], qk_par, abort_flag, p.status, 301))) break;
+      qk_par ^= 1u;
       tc_fence_after();
+      // the step's scalars, left by the producer before it requested the K tile
+      const uint2 scal = lds_volatile_v2(scal_slot + (t & 7) * 16);
+      const float c = __uint_as_float(scal.x);
+      const int valid = static_cast<int>(scal.y);
       uint32_t xa[32];
       float mx4[4];
       {
@@ -487,8 +528,12 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       sts_volatile_v2(ref_slot, __float_as_uint(m_ref), static_cast<uint32_t>(t + 1));
 
       // P[w] is free once the P V product of step t-2 has completed (long ago in the steady state)
-      if (t >= 2 && !(ok = mbar_wait_far(&bars->pv_done[(t - 2) % kStages], ((t - 2) / kStages) & 1, abort_flag, p.status, 302)))
-        break;
+      if (t >= 2) {
+        if (!(ok = mbar_wait_far(pv_bar0 + pv_off, pv_par, abort_flag, p.status, 302))) break;
+        pv_off ^= 2u;
+        pv_par ^= pv_flip;
+        pv_flip ^= 1u;
+      }
       tc_fence_after();
       {
         // the second half of the row is read again instead of being held across the first half's exponentials;
