@@ -36,7 +36,8 @@ namespace {
 
 using namespace sm100;
 
-constexpr int kStages = 4;  // K and V rings
+constexpr int kStages = 4;   // K ring; also the number of P V completion barriers (step t uses number t % 4)
+constexpr int kVStages = 3;  // V ring
 constexpr int kSetThreads = 128;                 // one softmax warpgroup
 constexpr int kSoftmaxThreads = 2 * kSetThreads;
 constexpr int kCtrlWarps = 4;
@@ -57,23 +58,23 @@ constexpr uint32_t kQBytes = 8192, kKStage = 8192, kVStage = 16384;
 constexpr uint32_t kOffQ = 0;
 constexpr uint32_t kOffK = kOffQ + kQBytes;
 constexpr uint32_t kOffV = kOffK + kStages * kKStage;
-constexpr uint32_t kOffZeta = kOffV + kStages * kVStage;  // zeta_i of the linear branch (256 B per query block)
+constexpr uint32_t kOffPhi = kOffV + kVStages * kVStage;  // phi(Q) as bf16 A operand of the linear product (16 KB)
+constexpr uint32_t kOffZeta = kOffPhi + 16384;            // zeta_i of the linear branch (256 B per query block)
 constexpr uint32_t kOffRef = kOffZeta + 512;              // per row: {reference maximum, number of steps published}
 constexpr uint32_t kOffX = kOffRef + 1024;                // epilogue exchange between the warpgroups (2 x 128 x 8 B)
 constexpr uint32_t kOffScal = kOffX + 2048;               // per step and query block: {exponent factor, valid keys}, ring of 8
 constexpr uint32_t kOffBar = kOffScal + 128;
 constexpr uint32_t kSmemBytes = kOffBar + 512;  // two CTAs per SM: 2 * (110592 + 1024 reserved) <= 232448
-// after the main loop the rings are reused: aggregated summaries G_i in K stages 0-1 (16 KB), the phi(Q) operand in
-// K stages 2-3 (16 KB), the output rows in the V ring (32 KB)
+// after the main loop the rings are reused: aggregated summaries G_i in K stages 0-1 (16 KB), the output rows in the
+// V ring (32 KB)
 constexpr uint32_t kOffG = kOffK;
-constexpr uint32_t kOffPhi = kOffK + 2 * kKStage;
 constexpr uint32_t kOffOut = kOffV;
 
 struct Bars {
   uint64_t q_full, z_full, g_full, phi_full, l_full, x_full;
-  uint64_t k_full[kStages], v_full[kStages];  // TMA -> issuer
+  uint64_t k_full[kStages], v_full[kVStages];  // TMA -> issuer
   uint64_t k_free[kStages];                   // Q K^T of the step in this stage complete -> producer
-  uint64_t pv_done[kStages];                  // P V of the step in this stage complete -> producer, softmax
+  uint64_t pv_done[kStages];                  // P V of step t (number t % 4) complete -> producer, softmax
   uint64_t qk_done[2];                        // S buffer written -> softmax
   uint64_t s_empty[2], p_full[2];             // softmax -> issuer
   uint32_t tmem_base;
@@ -212,9 +213,9 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     mbar_init(&bars->g_full, 1);
     mbar_init(&bars->phi_full, kSoftmaxThreads);
     mbar_init(&bars->l_full, 1);
+    for (int s = 0; s < kVStages; ++s) mbar_init(&bars->v_full[s], 1);
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&bars->k_full[s], 1);
-      mbar_init(&bars->v_full[s], 1);
       mbar_init(&bars->k_free[s], 1);
       mbar_init(&bars->pv_done[s], 1);
     }
@@ -265,14 +266,20 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             bulk_load(smem + kOffZeta + hf * 256, p.zeta + (bh_rows + i_q[hf]) * kHeadDim, 256, &bars->z_full);
         }
       }
-      const int* list0 = p.crit_idx + (bh_rows + i_q[0]) * p.k_crit;
-      const int* list1 = p.crit_idx + (bh_rows + i_q[1]) * p.k_crit;
       const float sq0 = __ldg(p.q_scales + bh_rows + i_q[0]) * (kLog2e * 0.125f);
       const float sq1 = __ldg(p.q_scales + bh_rows + i_q[1]) * (kLog2e * 0.125f);
-      // key block of step t for query block hf
-      auto key_block = [&](int t, int hf) {
-        if (kPair) return ldg_pinned((hf ? list1 : list0) + t);
-        return ldg_pinned(list0 + t / 2);
+      // Key blocks and their scales are fetched 32 steps at a time, lane l holding those of step 32 c + l, and handed
+      // to the issuing lane by a shuffle: no global load (let alone two dependent ones) sits in the per-step path.
+      int jl[2] = {0, 0};
+      float sl[2] = {0.f, 0.f};
+      auto refill = [&](int first) {
+        const int tt = first + lane;
+        if (tt < steps) {
+          for (int hf = 0; hf < kHalves; ++hf) {
+            jl[hf] = ldg_pinned(p.crit_idx + (bh_rows + i_q[hf]) * p.k_crit + (kPair ? tt : tt / 2));
+            sl[hf] = ldg_pinned(p.k_scales + bh_rows + jl[hf]);
+          }
+        }
       };
       // tile row (in the code tensors) of a step in key block j
       auto tile_row = [&](int t, int j) {
@@ -280,24 +287,25 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         return static_cast<int>((bh_rows + j) * 128 + (t & 1) * 64);
       };
       // The K cursor runs one step ahead of the V cursor (a K stage is free after the Q K^T of four steps earlier,
-      // a V stage only after that step's P V, and Q K^T of step t is issued before P V of step t-1).  The events the
-      // two cursors wait for alternate in time in exactly this order, so blocking waits lose nothing.  The key block
-      // of the K cursor's next step and its scale are fetched one step ahead.  Together with the K tile of a step
-      // the producer leaves the step's scalars for the softmax threads: the factor that turns a raw score into a
-      // base-2 exponent and the number of valid keys (ring of eight: the slot of step t is rewritten for step t+8,
-      // when the softmax threads of step t+2 have long released the scores, which they read after the scalars).
-      int jk[2] = {0, 0}, jv[2] = {0, 0};
-      float sk[2] = {0.f, 0.f};
-      if (steps > 0) {
-        for (int hf = 0; hf < kHalves; ++hf) {
-          jk[hf] = jv[hf] = key_block(0, hf);
-          sk[hf] = ldg_pinned(p.k_scales + bh_rows + jk[hf]);
-        }
-      }
+      // a V stage only after the P V of three steps earlier, and Q K^T of step t is issued before P V of step t-1).
+      // The events the two cursors wait for alternate in time in exactly this order, so blocking waits lose nothing.
+      // Together with the K tile of a step the producer leaves the step's scalars for the softmax threads: the
+      // factor that turns a raw score into a base-2 exponent and the number of valid keys (ring of eight: the slot of
+      // step t is rewritten for step t+8, when the softmax threads of step t+2 have long released the scores, which
+      // they read after the scalars).
       bool ok = true;
+      int sv = 0;              // V stage of the V cursor's step (tv % 3)
+      int jv[2] = {0, 0};      // key blocks of the V cursor's step (those of the K cursor one iteration earlier)
       for (int i = 0; ok && i <= steps; ++i) {
         const int tk = i, tv = i - 1;
+        int jk[2] = {0, 0};
         if (tk < steps) {
+          if ((tk & 31) == 0) refill(tk);
+          float sk[2];
+          for (int hf = 0; hf < kHalves; ++hf) {
+            jk[hf] = __shfl_sync(0xFFFFFFFFu, jl[hf], tk & 31);
+            sk[hf] = __shfl_sync(0xFFFFFFFFu, sl[hf], tk & 31);
+          }
           const int st = tk % kStages;
           if (tk >= kStages)
             ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars->k_free[st], ((tk - kStages) / kStages) & 1, abort_flag, p.status, 101, kBackoffNs));
@@ -313,27 +321,21 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             for (int hf = 0; hf < kHalves; ++hf)
               tma_load_2d(smem + kOffK + st * kKStage + hf * 4096, &map_k, &bars->k_full[st], 0, tile_row(tk, jk[hf]));
           }
-          if (tk + 1 < steps) {
-            for (int hf = 0; hf < kHalves; ++hf) {
-              jk[hf] = key_block(tk + 1, hf);
-              sk[hf] = ldg_pinned(p.k_scales + bh_rows + jk[hf]);
-            }
-          }
         }
         if (tv >= 0) {
-          const int st = tv % kStages;
-          if (tv >= kStages)
-            ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars->pv_done[st], ((tv - kStages) / kStages) & 1, abort_flag, p.status, 102, kBackoffNs));
+          // the stage of step tv held step tv - 3 before
+          if (tv >= kVStages)
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars->pv_done[(tv - kVStages) % kStages], ((tv - kVStages) / kStages) & 1,
+                                                   abort_flag, p.status, 102, kBackoffNs));
           if (!ok) break;
           if (leader) {
-            mbar_arrive_expect_tx(&bars->v_full[st], kVTx);
+            mbar_arrive_expect_tx(&bars->v_full[sv], kVTx);
             for (int hf = 0; hf < kHalves; ++hf)
-              tma_load_2d(smem + kOffV + st * kVStage + hf * 8192, &map_v, &bars->v_full[st], 0, tile_row(tv, jv[hf]));
+              tma_load_2d(smem + kOffV + sv * kVStage + hf * 8192, &map_v, &bars->v_full[sv], 0, tile_row(tv, jv[hf]));
           }
-          if (tv + 1 < steps) {
-            for (int hf = 0; hf < kHalves; ++hf) jv[hf] = key_block(tv + 1, hf);
-          }
+          if (++sv == kVStages) sv = 0;
         }
+        for (int hf = 0; hf < kHalves; ++hf) jv[hf] = jk[hf];
       }
       if (ok && p.k_marg > 0) {
         // The aggregated summaries go to K stages 0 and 1, which are free once the last Q K^T products have
@@ -391,8 +393,14 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
       }
       if (ok && p.k_marg > 0) {
+        // the linear product lands in score buffer 0: the scores of the last even step must have been read (the loop
+        // above has only waited for those of steps up to steps - 3)
         ok = mbar_wait(&bars->g_full, 0, abort_flag, p.status, 206, kBackoffNs) &&
              mbar_wait(&bars->phi_full, 0, abort_flag, p.status, 207, kBackoffNs);
+        if (ok && steps > 0) {
+          const int t_even = (steps - 1) & ~1;
+          ok = mbar_wait(&bars->s_empty[0], (t_even >> 1) & 1, abort_flag, p.status, 208, kBackoffNs);
+        }
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (ok) {
           tc_fence_after();
@@ -420,14 +428,15 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       const uint64_t v_desc0 = smem_desc(smem_u32(smem + kOffV), 8192, 1024, kSwizzle128);
       const uint32_t o_tmem = tmem + kColO;
       bool ok = true;
+      int sv = 0;
+      uint32_t v_par = 0;  // V stage of step t (t % 3) and the parity of its barrier ((t / 3) & 1)
       for (int t = 0; ok && t < steps; ++t) {  // O += P[t&1] V(t)
-        const int st = t % kStages;
-        ok = mbar_wait(&bars->v_full[st], (t / kStages) & 1, abort_flag, p.status, 205, kBackoffNs) &&
+        ok = mbar_wait(&bars->v_full[sv], v_par, abort_flag, p.status, 205, kBackoffNs) &&
              mbar_wait(&bars->p_full[t & 1], (t >> 1) & 1, abort_flag, p.status, 204, kBackoffNs);
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
         const uint32_t p_tmem = tmem + kColP + (t & 1) * 32;
-        const uint64_t v_desc = v_desc0 + static_cast<uint64_t>((st * kVStage) >> 4);
+        const uint64_t v_desc = v_desc0 + static_cast<uint64_t>((sv * kVStage) >> 4);
         tc_fence_after();
         if (leader) {
 #pragma unroll
@@ -437,7 +446,11 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               mma_f16_ts(o_tmem + ((hf * 16u) << 16), p_tmem + ((hf * 16u) << 16) + kk * 8,
                          v_desc + ((hf * 8192 + kk * 2048) >> 4), idesc_pv, (t > 0 || kk > 0) ? 1u : 0u);
           }
-          mma_commit(&bars->pv_done[st]);
+          mma_commit(&bars->pv_done[t % kStages]);
+        }
+        if (++sv == kVStages) {
+          sv = 0;
+          v_par ^= 1u;
         }
       }
     }
@@ -469,6 +482,86 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       m = __uint_as_float(v.x);
       return true;
     };
+
+    // linear branch, first part: this thread's 32 columns (warpgroup w -> columns 32 w ..) of phi(q) as bf16 A operand
+    // of the linear product, partial denominator phi(q) . zeta_i on the side.  It needs the Q tile and zeta_i only, so
+    // it is computed while the first key tiles are on their way and the softmax threads would be idle; the operand
+    // has a shared-memory region of its own and the linear product can then be issued as soon as the aggregated
+    // summaries have arrived and the last scores have been read.
+    // The query row comes from the Q tile in shared memory (64-byte rows, 64B swizzle: 16-byte chunk c of row r sits at
+    // chunk c ^ ((r >> 1) & 3)).
+    // The loops over 16-column chunks here and in the epilogue are deliberately NOT unrolled: the kernel's code has to
+    // stay within the instruction cache of an SM, which its fully unrolled form exceeded several times over (the
+    // kernel was then bound by instruction fetch from the GPC-level cache, not by any arithmetic unit).
+    float den = 0.f;
+    const int swz = p_row & 7;
+    if (p.k_marg > 0) {
+      ok = mbar_wait_far(&bars->q_full, 0, abort_flag, p.status, 307) && mbar_wait_far(&bars->z_full, 0, abort_flag, p.status, 308);
+      const uint8_t* qrow = smem + kOffQ + p_row * 64;
+      const int qswz = (p_row >> 1) & 3;
+      // phi = softmax over the components: any common shift of the exponents cancels in the ratio numerator /
+      // denominator.  448 * scale bounds every component of the block, so it serves as the shift without a pass over
+      // the row; only when exponents could then leave the fp32 range (block magnitudes in the hundreds) is the row's
+      // own maximum looked up.
+      const bool phi_softmax = p.phi == LITE3R_PHI_SOFTMAX;
+      const float cq = sq * kLog2e;
+      float shift = 448.f * cq;
+      if (phi_softmax && 896.f * cq > 100.f) {
+        float mxq[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll 1
+        for (int c4 = 0; c4 < 4; ++c4) {  // row maximum over the 64 components
+          const uint4 raw = *reinterpret_cast<const uint4*>(qrow + ((c4 ^ qswz) << 4));
+          const uint32_t words[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+          for (int xw = 0; xw < 4; ++xw) {
+            float fv[4];
+            e4m3x4_to_float(words[xw], fv);
+#pragma unroll
+            for (int y = 0; y < 4; ++y) mxq[y] = fmaxf(mxq[y], fv[y]);
+          }
+        }
+        shift = fmaxf(fmaxf(mxq[0], mxq[1]), fmaxf(mxq[2], mxq[3])) * cq;  // sq > 0 commutes with max
+      }
+      uint8_t* const phirow = smem + kOffPhi + p_row * 128;
+      float den4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+      for (int cc = 0; cc < 2; ++cc) {  // this warpgroup's two chunks of 16 components
+        const int c4 = 2 * w + cc;
+        const uint4 raw = *reinterpret_cast<const uint4*>(qrow + ((c4 ^ qswz) << 4));
+        const uint32_t words[4] = {raw.x, raw.y, raw.z, raw.w};
+        const float4* zeta = reinterpret_cast<const float4*>(smem + kOffZeta + hf * 256 + c4 * 64);
+        uint32_t pk8[8];
+#pragma unroll
+        for (int xw = 0; xw < 4; ++xw) {
+          float fv[4];
+          e4m3x4_to_float(words[xw], fv);
+          const float4 z = zeta[xw];
+          const float zz[4] = {z.x, z.y, z.z, z.w};
+#pragma unroll
+          for (int y = 0; y < 4; y += 2) {
+            float e0, e1;
+            if (phi_softmax) {  // the softmax normaliser cancels in the ratio
+              e0 = ex2(fmaf(fv[y], cq, -shift));
+              e1 = ex2(fmaf(fv[y + 1], cq, -shift));
+            } else {
+              e0 = fv[y] > 0.f ? fmaf(fv[y], sq, 1.f) : ex2(fv[y] * cq);
+              e1 = fv[y + 1] > 0.f ? fmaf(fv[y + 1], sq, 1.f) : ex2(fv[y + 1] * cq);
+            }
+            const uint32_t pk = pack_bf162(e0, e1);
+            pk8[xw * 2 + (y >> 1)] = pk;
+            // the denominator uses the same rounded values as the MMA's numerator
+            den4[y] = fmaf(__uint_as_float(pk << 16), zz[y], den4[y]);
+            den4[y + 1] = fmaf(__uint_as_float(pk & 0xFFFF0000u), zz[y + 1], den4[y + 1]);
+          }
+        }
+        *reinterpret_cast<uint4*>(phirow + (((c4 * 2) ^ swz) << 4)) = make_uint4(pk8[0], pk8[1], pk8[2], pk8[3]);
+        *reinterpret_cast<uint4*>(phirow + (((c4 * 2 + 1) ^ swz) << 4)) = make_uint4(pk8[4], pk8[5], pk8[6], pk8[7]);
+      }
+      den = (den4[0] + den4[1]) + (den4[2] + den4[3]);
+      fence_proxy_async_smem();
+      mbar_arrive(&bars->phi_full);
+    }
+
 
     // barrier of the P V product two steps back (the one that frees P[w]): its stage alternates between w and w + 2,
     // its parity flips every second iteration; both are carried along instead of being recomputed from t
@@ -563,86 +656,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(&bars->p_full[w]);
-    }
-
-    // linear branch: this thread's 32 columns (warpgroup w -> columns 32 w ..) of phi(q) as bf16 A operand, partial
-    // denominator phi(q) . zeta_i on the side; computed in registers while the last P V products are still running.
-    // The query row comes from the Q tile in shared memory (64-byte rows, 64B swizzle: 16-byte chunk c of row r sits at
-    // chunk c ^ ((r >> 1) & 3)).  Every Q K^T product has completed once both warpgroups are here, which the issuer
-    // of the linear product checks through phi_full; the operand goes to K stages 2 and 3.
-    // The epilogue's loops over 16-column chunks are deliberately NOT unrolled: the kernel's code has to stay within
-    // the instruction cache of an SM, which its fully unrolled form exceeded several times over (the kernel was then
-    // bound by instruction fetch from the GPC-level cache, not by any arithmetic unit).
-    float den = 0.f;
-    const int swz = p_row & 7;
-    if (ok && p.k_marg > 0) {
-      ok = mbar_wait_far(&bars->q_full, 0, abort_flag, p.status, 307) && mbar_wait_far(&bars->z_full, 0, abort_flag, p.status, 308);
-      // the other warpgroup's last Q K^T may still be reading K stage 2 or 3: wait for the last two steps' products
-      for (int u = max(0, steps - 2); u < steps && ok; ++u)
-        ok = mbar_wait_far(&bars->k_free[u % kStages], (u / kStages) & 1, abort_flag, p.status, 310);
-      const uint8_t* qrow = smem + kOffQ + p_row * 64;
-      const int qswz = (p_row >> 1) & 3;
-      // phi = softmax over the components: any common shift of the exponents cancels in the ratio numerator /
-      // denominator.  448 * scale bounds every component of the block, so it serves as the shift without a pass over
-      // the row; only when exponents could then leave the fp32 range (block magnitudes in the hundreds) is the row's
-      // own maximum looked up.
-      const bool phi_softmax = p.phi == LITE3R_PHI_SOFTMAX;
-      const float cq = sq * kLog2e;
-      float shift = 448.f * cq;
-      if (phi_softmax && 896.f * cq > 100.f) {
-        float mxq[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll 1
-        for (int c4 = 0; c4 < 4; ++c4) {  // row maximum over the 64 components
-          const uint4 raw = *reinterpret_cast<const uint4*>(qrow + ((c4 ^ qswz) << 4));
-          const uint32_t words[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-          for (int xw = 0; xw < 4; ++xw) {
-            float fv[4];
-            e4m3x4_to_float(words[xw], fv);
-#pragma unroll
-            for (int y = 0; y < 4; ++y) mxq[y] = fmaxf(mxq[y], fv[y]);
-          }
-        }
-        shift = fmaxf(fmaxf(mxq[0], mxq[1]), fmaxf(mxq[2], mxq[3])) * cq;  // sq > 0 commutes with max
-      }
-      uint8_t* const phirow = smem + kOffPhi + p_row * 128;
-      float den4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 1
-      for (int cc = 0; cc < 2; ++cc) {  // this warpgroup's two chunks of 16 components
-        const int c4 = 2 * w + cc;
-        const uint4 raw = *reinterpret_cast<const uint4*>(qrow + ((c4 ^ qswz) << 4));
-        const uint32_t words[4] = {raw.x, raw.y, raw.z, raw.w};
-        const float4* zeta = reinterpret_cast<const float4*>(smem + kOffZeta + hf * 256 + c4 * 64);
-        uint32_t pk8[8];
-#pragma unroll
-        for (int xw = 0; xw < 4; ++xw) {
-          float fv[4];
-          e4m3x4_to_float(words[xw], fv);
-          const float4 z = zeta[xw];
-          const float zz[4] = {z.x, z.y, z.z, z.w};
-#pragma unroll
-          for (int y = 0; y < 4; y += 2) {
-            float e0, e1;
-            if (phi_softmax) {  // the softmax normaliser cancels in the ratio
-              e0 = ex2(fmaf(fv[y], cq, -shift));
-              e1 = ex2(fmaf(fv[y + 1], cq, -shift));
-            } else {
-              e0 = fv[y] > 0.f ? fmaf(fv[y], sq, 1.f) : ex2(fv[y] * cq);
-              e1 = fv[y + 1] > 0.f ? fmaf(fv[y + 1], sq, 1.f) : ex2(fv[y + 1] * cq);
-            }
-            const uint32_t pk = pack_bf162(e0, e1);
-            pk8[xw * 2 + (y >> 1)] = pk;
-            // the denominator uses the same rounded values as the MMA's numerator
-            den4[y] = fmaf(__uint_as_float(pk << 16), zz[y], den4[y]);
-            den4[y + 1] = fmaf(__uint_as_float(pk & 0xFFFF0000u), zz[y + 1], den4[y + 1]);
-          }
-        }
-        *reinterpret_cast<uint4*>(phirow + (((c4 * 2) ^ swz) << 4)) = make_uint4(pk8[0], pk8[1], pk8[2], pk8[3]);
-        *reinterpret_cast<uint4*>(phirow + (((c4 * 2 + 1) ^ swz) << 4)) = make_uint4(pk8[4], pk8[5], pk8[6], pk8[7]);
-      }
-      den = (den4[0] + den4[1]) + (den4[2] + den4[3]);
-      fence_proxy_async_smem();
-      mbar_arrive(&bars->phi_full);
     }
 
     // the two threads of a row (one per warpgroup) bring their row sums to the final reference and swap them together
