@@ -576,13 +576,15 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       const uint2 scal = lds_volatile_v2(scal_slot + (t & 7) * 16);
       const float c = __uint_as_float(scal.x);
       const int valid = static_cast<int>(scal.y);
-      uint32_t xa[32];
+      uint32_t xa[32], xb[32];
       float mx4[4];
       {
-        uint32_t xb[32];
         tmem_ld32(s_addr, xa);
         tmem_ld32(s_addr + 32, xb);
         tmem_wait_ld();
+        // the whole row of scores is in registers: the issuer may overwrite S[w] with step t+2 right away
+        tc_fence_before();
+        mbar_arrive(&bars->s_empty[w]);
         if (valid < kStepKeys) {
 #pragma unroll
           for (int k = 0; k < 32; ++k) {
@@ -634,16 +636,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         uint32_t packed[16];
         l += exp_half_row(xa, c, -m_ref, packed);
         tmem_st16(p_addr, packed);
-        tmem_ld32(s_addr + 32, xa);
-        tmem_wait_ld();
-        tc_fence_before();
-        mbar_arrive(&bars->s_empty[w]);  // the issuer may overwrite S[w] with step t+2
-        if (valid < kStepKeys) {
-#pragma unroll
-          for (int k = 0; k < 32; ++k)
-            if (32 + k >= valid) xa[k] = 0xFF800000u;
-        }
-        l += exp_half_row(xa, c, -m_ref, packed);
+        l += exp_half_row(xb, c, -m_ref, packed);
         tmem_st16(p_addr + 16, packed);
       }
       if (__any_sync(0xFFFFFFFFu, need)) {
