@@ -30,6 +30,14 @@ LITE3R_API lite3r_status lite3r_profile_stage_ms(float* ms);
 /* Number of kernel launches the library has enqueued since it was loaded (all threads). */
 LITE3R_API long long lite3r_launch_count(void);
 
+/* Test hook: which of its kernels lite3r_sla_plan (and a forward that builds its own plan) uses.  0 = chosen by the
+ * size of the problem (the default); 1 = eight rows per CTA with 64-bit keys in shared memory; 2 / 3 = eight / sixteen
+ * rows per CTA with single-precision scores in shared memory and exact keys recomputed for the entries at a
+ * selection threshold (what long rows get); 4 = four rows per CTA with staged column sums (what rows too long for
+ * the others get).  Every variant gives the same plan; a forced variant that does not fit the shape makes the plan call
+ * return LITE3R_ERR_UNSUPPORTED.  Process-wide. */
+LITE3R_API lite3r_status lite3r_plan_variant(int variant);
+
 /* Byte offsets, inside the workspace of lite3r_sla_forward, of its six parts, for tests that inspect intermediates
  * after a forward: offsets[0] per-key-block summaries, bf16 [tiles][4160] = ((H_j W)^T as [e][d] | z_j[d]), the
  * KV summary and normaliser of Algorithm 1 per block with the projection folded in; [1] per-query-block aggregates

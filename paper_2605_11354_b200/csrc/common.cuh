@@ -82,6 +82,7 @@ __device__ __forceinline__ float warp_sum(float v) {
 // One launch quantises `count` (1..3) source tensors of the same shape and dtype.
 lite3r_status launch_quantize(const lite3r_tensor* const* x, const lite3r_fp8* out, int count, const lite3r_shape& s,
                               cudaStream_t stream);
+void set_plan_variant(int variant);  // test hook, see lite3r_plan_variant
 lite3r_status launch_plan(const lite3r_fp8& q, const lite3r_fp8& k, const lite3r_shape& s, const Counts& c,
                           const lite3r_plan& plan, cudaStream_t stream);
 

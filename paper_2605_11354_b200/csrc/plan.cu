@@ -22,6 +22,8 @@
 //     row.  Two selections give the classes: the best k_crit are critical, the best Nb - k_neg are
 //     critical-or-marginal.
 //   Phase C (same warp): class row and ascending index lists, written with ballot prefix sums.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace lite3r {
@@ -482,6 +484,323 @@ __global__ void __launch_bounds__(R * 32) plan_kernel(const int* __restrict__ q_
   }
 }
 
+// The same plan with the scores kept in shared memory as single-precision values (4 bytes per key instead of an
+// 8-byte ordered key), for long rows: sixteen rows per CTA then fit where eight did, so the column sums of a (b, h)
+// are streamed half as often and twice as many warps hide the latencies of the selection and of the class pass.
+// The ranking stays the exact one.  The single-precision copy is a monotone (weakly order-preserving) image of the
+// exact score and only places a key in one of the 256 buckets; the few keys of a threshold bucket are decided by
+// their exact 64-bit keys, which are recomputed for them from the integer column sums (an int64 dot product, equal
+// to the tensor-core result as long as that is exact, i.e. below 2^53).
+// Warp w of the R = 8 or 16 warps: in phase A row tile w % (R / 8) (eight rows) against every (R / 8)-th group of
+// eight key blocks; in phases B and C row w.
+template <int R>
+__global__ void __launch_bounds__(R * 32) plan_compact_kernel(const int* __restrict__ q_colsum, const int* __restrict__ k_colsum,
+                                                               const float* __restrict__ k_scales, int tokens, int block,
+                                                               int nb, int k_crit, int k_marg, int k_neg,
+                                                               signed char* __restrict__ cls, int* __restrict__ crit_idx,
+                                                               int* __restrict__ marg_idx) {
+  constexpr int kRowTiles = R / 8;
+  constexpr int kGroups = R / kRowTiles;  // warps that share a row tile (= 8)
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int pitch = (nb + 3) & ~3;
+  float* s_val = reinterpret_cast<float*>(smem_raw);                                              // [R][pitch]
+  unsigned int* s_hist = reinterpret_cast<unsigned int*>(s_val + static_cast<size_t>(R) * pitch);  // [R][2][256]
+  unsigned long long* s_ckey = reinterpret_cast<unsigned long long*>(s_hist + R * 2 * kBuckets);   // [R][2][kMaxListed]
+  int* s_q = reinterpret_cast<int*>(s_ckey + R * 2 * kMaxListed);                                  // [R][64]
+  float2* s_range = reinterpret_cast<float2*>(s_q + R * kHeadDim);                                 // [kGroups][R]
+  unsigned short* s_idx = reinterpret_cast<unsigned short*>(s_range + kGroups * R);                // [R][2][kMaxListed]
+
+  const int row_tiles = (nb + R - 1) / R;
+  const int bh = blockIdx.x / row_tiles;
+  const int i0 = (blockIdx.x % row_tiles) * R;
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const size_t bh_rows = static_cast<size_t>(bh) * nb;
+  const bool block_pow2 = (block & (block - 1)) == 0;
+  const double inv_block = 1.0 / static_cast<double>(block);
+
+  // the ranking score from an exact dot product (same expression in phase A and for the recomputed keys)
+  auto ranking_score = [&](double dot, float ks, int j) {
+    const int valid = min(block, tokens - j * block);
+    const double num = dot * static_cast<double>(ks);
+    return ((valid == block && block_pow2) ? num * inv_block : num / static_cast<double>(valid)) + 0.0;
+  };
+
+  {
+    // Phase A: fp64 tensor-core products of the exactly widened int32 column sums (see plan_kernel).
+    const int tile = warp % kRowTiles, grp = warp / kRowTiles;
+    const int g = lane >> 2, t4 = lane & 3;
+    auto widen = [](int v) { return __int2double_rn(v); };  // exact; one instruction
+    auto load16 = [&](const int* base, size_t row, bool in, int4 dst[4]) {
+      const int4* src = reinterpret_cast<const int4*>(base + row * kHeadDim + 16 * t4);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) dst[q] = in ? __ldg(src + q) : make_int4(0, 0, 0, 0);
+    };
+    double q_frag[16];
+    {
+      int4 qv[4];
+      load16(q_colsum, bh_rows + i0 + 8 * tile + g, i0 + 8 * tile + g < nb, qv);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        q_frag[4 * q] = widen(qv[q].x);
+        q_frag[4 * q + 1] = widen(qv[q].y);
+        q_frag[4 * q + 2] = widen(qv[q].z);
+        q_frag[4 * q + 3] = widen(qv[q].w);
+      }
+    }
+    auto load_scales = [&](int j, float dst[2]) {
+#pragma unroll
+      for (int x = 0; x < 2; ++x) dst[x] = j + x < nb ? __ldg(k_scales + bh_rows + j + x) : 0.f;
+    };
+    int4 nxt[4];
+    float nxt_ks[2];
+    load16(k_colsum, bh_rows + grp * 8 + g, grp * 8 + g < nb, nxt);
+    load_scales(grp * 8 + 2 * t4, nxt_ks);
+    float lo = INFINITY, hi = -INFINITY;
+    float* const my_val = s_val + static_cast<size_t>(8 * tile + g) * pitch;
+    // key blocks in whole blocks of a power-of-two size divide by a multiplication that is exact, so the scale and
+    // the division fold into one factor per key block; only the last key block of a sequence can be shorter
+    const int last_full = (tokens % block == 0 && block_pow2) ? nb : (block_pow2 ? nb - 1 : 0);  // key blocks below this are whole
+#pragma unroll 2
+    for (int j0 = grp * 8; j0 < nb; j0 += 8 * kGroups) {
+      int4 cur[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) cur[q] = nxt[q];
+      const float cur_ks[2] = {nxt_ks[0], nxt_ks[1]};
+      if (j0 + 8 * kGroups < nb) {
+        load16(k_colsum, bh_rows + j0 + 8 * kGroups + g, j0 + 8 * kGroups + g < nb, nxt);
+        load_scales(j0 + 8 * kGroups + 2 * t4, nxt_ks);
+      }
+      double c[2][2] = {{0.0, 0.0}, {0.0, 0.0}};
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int vals[4] = {cur[q].x, cur[q].y, cur[q].z, cur[q].w};
+#pragma unroll
+        for (int y = 0; y < 4; ++y) {
+          const int st = 4 * q + y;
+          const double bv = widen(vals[y]);
+          asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+                       : "+d"(c[st & 1][0]), "+d"(c[st & 1][1])
+                       : "d"(q_frag[st]), "d"(bv));
+        }
+      }
+      if (j0 + 8 <= last_full) {  // all eight key blocks of the step exist and are whole (warp-uniform)
+        float tf[2];
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+          tf[x] = static_cast<float>((c[0][x] + c[1][x]) * (static_cast<double>(cur_ks[x]) * inv_block) + 0.0);
+          lo = fminf(lo, tf[x]);
+          hi = fmaxf(hi, tf[x]);
+        }
+        *reinterpret_cast<float2*>(my_val + j0 + 2 * t4) = make_float2(tf[0], tf[1]);
+      } else {
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+          const int j = j0 + 2 * t4 + x;
+          if (j < nb) {
+            const float tf = static_cast<float>(ranking_score(c[0][x] + c[1][x], cur_ks[x], j));
+            my_val[j] = tf;
+            lo = fminf(lo, tf);
+            hi = fmaxf(hi, tf);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int o = 1; o <= 2; o <<= 1) {
+      lo = fminf(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, o));
+      hi = fmaxf(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, o));
+    }
+    if (t4 == 0) s_range[grp * R + 8 * tile + g] = make_float2(lo, hi);
+  }
+  __syncthreads();
+  const int i = i0 + warp;
+  if (i >= nb) return;
+
+  // Phase B
+  const float* vals = s_val + static_cast<size_t>(warp) * pitch;
+  unsigned int* hist = s_hist + warp * 2 * kBuckets;
+  unsigned int* bucket_hist = hist + kBuckets;
+  float2 range = lane < kGroups ? s_range[lane * R + warp] : make_float2(INFINITY, -INFINITY);
+#pragma unroll
+  for (int o = 1; o < kGroups; o <<= 1) {
+    range.x = fminf(range.x, __shfl_xor_sync(0xFFFFFFFFu, range.x, o));
+    range.y = fmaxf(range.y, __shfl_xor_sync(0xFFFFFFFFu, range.y, o));
+  }
+  const float lo = __shfl_sync(0xFFFFFFFFu, range.x, 0), hi = __shfl_sync(0xFFFFFFFFu, range.y, 0);
+  // A key's place between the row's extremes on a 16-bit scale; its upper eight bits are the bucket of the first
+  // histogram, the lower eight refine a bucket that turns out too full to list.  Both are monotone in the score.
+  const float scale = hi > lo ? 65535.5f / (hi - lo) : 0.f;
+  auto fine = [&](int j) -> int { return min(65535, max(0, __float2int_rz((vals[j] - lo) * scale))); };
+  // exact 64-bit key of entry j of this row (the row's own column sums wait in shared memory)
+  int* const q_row = s_q + warp * kHeadDim;
+  q_row[lane] = __ldg(q_colsum + (bh_rows + i) * kHeadDim + lane);
+  q_row[lane + 32] = __ldg(q_colsum + (bh_rows + i) * kHeadDim + lane + 32);
+  const int4* const q4 = reinterpret_cast<const int4*>(q_row);
+  auto exact_key = [&](int j) -> unsigned long long {
+    const int4* const k4 = reinterpret_cast<const int4*>(k_colsum + (bh_rows + j) * kHeadDim);
+    long long dot = 0;
+#pragma unroll
+    for (int d = 0; d < kHeadDim / 4; ++d) {
+      const int4 a = q4[d], b = __ldg(k4 + d);
+      dot += static_cast<long long>(a.x) * b.x + static_cast<long long>(a.y) * b.y + static_cast<long long>(a.z) * b.z +
+             static_cast<long long>(a.w) * b.w;
+    }
+    return order_key(ranking_score(static_cast<double>(dot), __ldg(k_scales + bh_rows + j), j));
+  };
+#pragma unroll
+  for (int b = 0; b < 8; ++b) bucket_hist[lane + 32 * b] = 0u;
+  __syncwarp();
+  for (int j = lane; j < nb; j += 32) atomicAdd(&bucket_hist[fine(j) >> 8], 1u);
+  __syncwarp();
+
+  // A selection: entries whose place is above t_hi are selected, those inside [t_lo, t_hi] are decided by their exact
+  // keys (prefix / mask / take as in Selection), the rest are not.  Each selection leaves the entries of its
+  // threshold range (ascending index) and their exact keys behind for the class pass: keys_from 0 = no key needed
+  // (the whole range goes one way), 1 = listed, 2 = recompute (still too many to list after the refinement).
+  struct Chosen {
+    Selection s;
+    int t_lo, t_hi, keys_from;
+  };
+  auto select = [&](int k, unsigned long long* ckey, unsigned short* idx) -> Chosen {
+    Chosen r;
+    r.keys_from = 0;
+    r.s.prefix = 0ull;
+    r.s.mask = 0ull;
+    r.s.take = 0;
+    r.s.bucket = 0;
+    if (k <= 0) {
+      r.t_lo = r.t_hi = 65536;
+      return r;
+    }
+    if (k >= nb) {
+      r.t_lo = r.t_hi = -1;
+      return r;
+    }
+    const Located at = locate(bucket_hist, k, lane);
+    r.t_lo = at.bin << 8;
+    r.t_hi = r.t_lo + 255;
+    int remaining = k - at.above, size = at.size;
+    if (remaining == size) {
+      r.s.take = size;
+      return r;
+    }
+    if (size > kMaxListed) {  // refine: histogram of the lower eight bits inside the bucket
+#pragma unroll
+      for (int b = 0; b < 8; ++b) hist[lane + 32 * b] = 0u;
+      __syncwarp();
+      for (int j = lane; j < nb; j += 32) {
+        const int f = fine(j);
+        if ((f >> 8) == at.bin) atomicAdd(&hist[f & 255], 1u);
+      }
+      __syncwarp();
+      const Located at2 = locate(hist, remaining, lane);
+      __syncwarp();
+      r.t_lo = r.t_hi = (at.bin << 8) | at2.bin;
+      remaining -= at2.above;
+      size = at2.size;
+      if (remaining == size) {
+        r.s.take = size;
+        return r;
+      }
+    }
+    const int t_lo = r.t_lo, t_hi = r.t_hi;
+    if (size <= kMaxListed) {
+      const unsigned below = (1u << lane) - 1u;
+      int listed = 0;
+      for (int j0 = 0; j0 < nb; j0 += 32) {
+        const int j = j0 + lane;
+        const int f = j < nb ? fine(j) : -1;
+        const bool is = f >= t_lo && f <= t_hi;
+        const unsigned b = __ballot_sync(0xFFFFFFFFu, is);
+        if (is) idx[listed + __popc(b & below)] = static_cast<unsigned short>(j);
+        listed += __popc(b);
+      }
+      __syncwarp();
+      for (int c = lane; c < size; c += 32) ckey[c] = exact_key(idx[c]);
+      __syncwarp();
+      r.keys_from = 1;
+      radix_select([&](int c, unsigned long long& key) {
+        key = ckey[c];
+        return true;
+      }, size, remaining, hist, lane, r.s);
+    } else {  // more than kMaxListed entries in one of 65536 places (near-equal scores): every pass recomputes keys
+      r.keys_from = 2;
+      radix_select([&](int c, unsigned long long& key) {
+        const int f = fine(c);
+        if (f < t_lo || f > t_hi) return false;
+        key = exact_key(c);
+        return true;
+      }, nb, remaining, hist, lane, r.s);
+    }
+    return r;
+  };
+  unsigned long long* const ckey_c = s_ckey + warp * 2 * kMaxListed;
+  unsigned long long* const ckey_m = ckey_c + kMaxListed;
+  unsigned short* const idx_c = s_idx + warp * 2 * kMaxListed;
+  const Chosen cc = select(k_crit, ckey_c, idx_c);
+  const Chosen cm = select(nb - k_neg, ckey_m, idx_c + kMaxListed);
+  const Selection sc = cc.s, sm = cm.s;
+  const int from_c = cc.keys_from, from_m = cm.keys_from;
+
+  // Phase C
+  const size_t row = bh_rows + i;
+  signed char* out_cls = cls + row * nb;
+  int n_crit = 0, n_marg = 0, tie_c = 0, tie_m = 0, seen_c = 0, seen_m = 0;
+  const unsigned below = (1u << lane) - 1u;
+#pragma unroll 2
+  for (int j0 = 0; j0 < nb; j0 += 32) {
+    const int j = j0 + lane;
+    const bool in = j < nb;
+    const int f = in ? fine(j) : -2;
+    bool sel_c = in && f > cc.t_hi, sel_m = in && f > cm.t_hi;
+    const bool at_c = f >= cc.t_lo && f <= cc.t_hi, at_m = f >= cm.t_lo && f <= cm.t_hi;
+    if (__any_sync(0xFFFFFFFFu, at_c || at_m)) {
+      // the entries of a threshold bucket come by in the order in which the selection listed them
+      const unsigned b_at_c = __ballot_sync(0xFFFFFFFFu, at_c), b_at_m = __ballot_sync(0xFFFFFFFFu, at_m);
+      unsigned long long kc = 0ull, km = 0ull;
+      if (at_c && from_c != 0) kc = (from_c == 1 ? ckey_c[seen_c + __popc(b_at_c & below)] : exact_key(j)) & sc.mask;
+      if (at_m && from_m != 0) km = (from_m == 1 ? ckey_m[seen_m + __popc(b_at_m & below)] : exact_key(j)) & sm.mask;
+      seen_c += __popc(b_at_c);
+      seen_m += __popc(b_at_m);
+      const bool eq_c = at_c && kc == sc.prefix, eq_m = at_m && km == sm.prefix;
+      const unsigned b_eq_c = __ballot_sync(0xFFFFFFFFu, eq_c), b_eq_m = __ballot_sync(0xFFFFFFFFu, eq_m);
+      sel_c = sel_c || (at_c && kc > sc.prefix) || (eq_c && tie_c + __popc(b_eq_c & below) < sc.take);
+      sel_m = sel_m || (at_m && km > sm.prefix) || (eq_m && tie_m + __popc(b_eq_m & below) < sm.take);
+      tie_c += __popc(b_eq_c);
+      tie_m += __popc(b_eq_m);
+    }
+    const int c = !in ? -1 : (sel_c ? 2 : (sel_m ? 1 : 0));
+    if (in) out_cls[j] = static_cast<signed char>(c);
+    const unsigned m_crit = __ballot_sync(0xFFFFFFFFu, c == 2);
+    const unsigned m_marg = __ballot_sync(0xFFFFFFFFu, c == 1);
+    if (c == 2) crit_idx[row * k_crit + n_crit + __popc(m_crit & below)] = j;
+    if (c == 1 && marg_idx != nullptr) marg_idx[row * k_marg + n_marg + __popc(m_marg & below)] = j;
+    n_crit += __popc(m_crit);
+    n_marg += __popc(m_marg);
+  }
+}
+
+size_t plan_compact_smem_bytes(int nb, int rows) {
+  const size_t pitch = static_cast<size_t>((nb + 3) & ~3);
+  return rows * pitch * 4 + static_cast<size_t>(rows) * 2 * kBuckets * 4 + static_cast<size_t>(rows) * 2 * kMaxListed * 8 +
+         static_cast<size_t>(rows) * kHeadDim * 4 + static_cast<size_t>(8) * rows * sizeof(float2) +
+         static_cast<size_t>(rows) * 2 * kMaxListed * 2;
+}
+
+template <int R>
+lite3r_status launch_compact(const lite3r_fp8& q, const lite3r_fp8& k, const lite3r_shape& s, const Counts& c,
+                             const lite3r_plan& plan, int nb, cudaStream_t stream) {
+  const size_t smem = plan_compact_smem_bytes(nb, R);
+  lite3r_status st = ensure_dynamic_smem(plan_compact_kernel<R>, static_cast<int>(smem));
+  if (st != LITE3R_OK) return st;
+  const int row_tiles = ceil_div(nb, R);
+  plan_compact_kernel<R><<<s.batch * s.heads * row_tiles, R * 32, smem, stream>>>(q.colsum, k.colsum, k.scales, s.tokens,
+                                                                                   s.block, nb, c.k_crit, c.k_marg, c.k_neg,
+                                                                                   plan.cls, plan.crit_idx, plan.marg_idx);
+  return after_launch();
+}
+
 size_t plan_smem_bytes(int nb, int rows) {
   const size_t pitch = static_cast<size_t>((nb + 1) & ~1);
   const size_t common = rows * pitch * 8 + static_cast<size_t>(rows) * 2 * kBuckets * 4 +
@@ -507,10 +826,32 @@ lite3r_status launch_rows(const lite3r_fp8& q, const lite3r_fp8& k, const lite3r
 
 }  // namespace
 
+// Test hook: which kernel launch_plan takes (0 = by size, as described there).
+static std::atomic<int> g_plan_variant{0};
+void set_plan_variant(int variant) { g_plan_variant.store(variant, std::memory_order_relaxed); }
+
 lite3r_status launch_plan(const lite3r_fp8& q, const lite3r_fp8& k, const lite3r_shape& s, const Counts& c,
                           const lite3r_plan& plan, cudaStream_t stream) {
   const int nb = ceil_div(s.tokens, s.block);
   constexpr size_t kLimit = 227 * 1024;
+  switch (g_plan_variant.load(std::memory_order_relaxed)) {  // forced by a test; sizes that do not fit are refused
+    case 1: return plan_smem_bytes(nb, 8) <= kLimit ? launch_rows<8>(q, k, s, c, plan, nb, stream) : LITE3R_ERR_UNSUPPORTED;
+    case 2: return plan_compact_smem_bytes(nb, 8) <= kLimit && nb <= 65536 ? launch_compact<8>(q, k, s, c, plan, nb, stream) : LITE3R_ERR_UNSUPPORTED;
+    case 3: return plan_compact_smem_bytes(nb, 16) <= kLimit && nb <= 65536 ? launch_compact<16>(q, k, s, c, plan, nb, stream) : LITE3R_ERR_UNSUPPORTED;
+    case 4: return plan_smem_bytes(nb, 4) <= kLimit ? launch_rows<4>(q, k, s, c, plan, nb, stream) : LITE3R_ERR_UNSUPPORTED;
+    default: break;
+  }
+  // Long rows (where the 8-byte keys of eight rows would leave room for a single CTA per SM): single-precision scores in
+  // shared memory, sixteen rows per CTA when that still leaves every SM several CTAs to work on, else eight (index
+  // lists hold 16-bit positions: rows of up to 65536 blocks).
+  int sms = 0;
+  lite3r_status st = sm_count(&sms);
+  if (st != LITE3R_OK) return st;
+  if (plan_smem_bytes(nb, 8) > kLimit / 2 && nb <= 65536) {
+    const long long ctas16 = static_cast<long long>(s.batch) * s.heads * ceil_div(nb, 16);
+    if (ctas16 >= 4ll * sms && plan_compact_smem_bytes(nb, 16) <= kLimit) return launch_compact<16>(q, k, s, c, plan, nb, stream);
+    if (plan_compact_smem_bytes(nb, 8) <= kLimit) return launch_compact<8>(q, k, s, c, plan, nb, stream);
+  }
   // As many rows per CTA as the row keys allow: the staged key blocks are then shared by more rows.
   if (plan_smem_bytes(nb, 8) <= kLimit) return launch_rows<8>(q, k, s, c, plan, nb, stream);
   if (plan_smem_bytes(nb, 4) <= kLimit) return launch_rows<4>(q, k, s, c, plan, nb, stream);

@@ -202,12 +202,89 @@ def test_all_scores_tied_in_a_long_row():
 
 
 def test_plan_of_a_very_long_sequence():
-    """3000 blocks: the row keys of eight query blocks no longer fit in shared memory, so the plan kernel runs with
-    four rows per CTA, staged column sums and the whole selection in the radix select.  Quantiser and plan are
-    compared in full, the output on a few sampled query blocks."""
+    """3000 blocks: the 64-bit row keys of eight query blocks no longer fit in shared memory, so the plan runs on the
+    kernel that keeps single-precision scores and recomputes the exact keys at the selection thresholds.  Quantiser
+    and plan are compared in full, the output on a few sampled query blocks."""
     wl = small_workload("long", tokens=3000 * 64 - 17, heads=1, src_dtype="bf16", crit=0.01, neg=0.95)
     inputs = wk.make_inputs(wl)
     full_parity(wl, inputs, query_blocks=pu.sample_blocks(wl, [0], 6, seed=5))
+
+
+@pytest.fixture
+def plan_variant():
+    """Forces one of the plan kernels for the duration of a test (the library chooses by size otherwise)."""
+    yield lt.lite3r_plan_variant
+    lt.lite3r_plan_variant(0)
+
+
+def plan_only(inputs, wl, crit=None, neg=None):
+    """Quantises and plans on the GPU; returns the class matrix and the index lists as the oracle lays them out."""
+    crit = wl.crit if crit is None else crit
+    neg = wl.neg if neg is None else neg
+    eng = lt.SlaForward(wl.batch, wl.heads, wl.tokens, wl.block, crit, neg)
+    eng.quantize(*[pu.to_device(inputs[n], wl.src_dtype) for n in ("q", "k", "v")])
+    eng.make_plan()
+    torch.cuda.synchronize()
+    return eng
+
+
+@pytest.mark.parametrize("variant", [1, 2, 3, 4])
+def test_every_plan_kernel_on_ties_and_near_ties(variant, plan_variant):
+    """The four plan kernels (64-bit keys, single-precision scores with 8 or 16 rows per CTA, staged column sums) must
+    give the oracle's plan bit for bit on the cases that separate them: exact ties (duplicated key blocks), rows
+    whose scores are all equal (every entry in one place of the selection histogram: the keys are recomputed pass by
+    pass), a crowded histogram bucket that only the refinement separates, ragged last blocks, and empty classes."""
+    plan_variant(variant)
+    # duplicated key blocks in a ragged sequence of 300 blocks
+    wl = small_workload(f"var{variant}-ties", tokens=300 * 64 - 21, heads=2, src_dtype="f32", crit=0.1, neg=0.45)
+    inputs = wk.make_inputs(wl)
+    for dst, src in ((3, 1), (5, 1), (8, 2), (299, 7), (150, 149)):
+        n = min(64, wl.tokens - dst * 64)
+        inputs["k"][:, :, dst * 64:dst * 64 + n] = inputs["k"][:, :, src * 64:src * 64 + n]
+    for crit, neg in ((0.1, 0.45), (0.0, 0.5), (0.37, 0.63), (1.0, 0.0), (0.02, 0.0)):
+        eng = plan_only(inputs, wl, crit, neg)
+        ref = oracle_subset(inputs, wl, [0, 1], crit, neg, query_blocks=[])
+        flips, _ = pu.compare_plan(eng, ref["scores"], ref["cls"], [0, 1])
+        assert flips == 0, (variant, crit, neg, flips)
+    # all scores of every row equal, then nearly equal: keys that differ only far below single precision
+    wl = small_workload(f"var{variant}-flat", tokens=400 * 64, heads=1, src_dtype="f32", crit=0.2, neg=0.5)
+    inputs = wk.make_inputs(wl)
+    inputs["q"][:] = 0.0
+    eng = plan_only(inputs, wl)
+    ref = oracle_subset(inputs, wl, [0], query_blocks=[])
+    assert np.array_equal(eng.plan.cls.cpu().numpy(), ref["cls"])
+    # a crowded bucket: 390 key blocks with scores within 5 % of each other and ten a hundred times larger, which
+    # stretch the histogram's range so that the 390 share one of its 256 buckets (far more than the candidate list
+    # keeps) and only the 16-bit refinement separates them
+    g = np.random.default_rng(variant)
+    inputs["q"][:] = 1.0
+    level = (1.0 + 0.05 * g.uniform(-1.0, 1.0, 400)).astype(np.float32)
+    level[g.choice(400, 10, replace=False)] = 100.0
+    inputs["k"][0, 0] = np.repeat(level, 64)[:, None]
+    for crit, neg in ((0.2, 0.5), (0.5, 0.1), (0.02, 0.9)):
+        eng = plan_only(inputs, wl, crit, neg)
+        ref = oracle_subset(inputs, wl, [0], crit, neg, query_blocks=[])
+        flips, _ = pu.compare_plan(eng, ref["scores"], ref["cls"], [0])
+        assert flips == 0, (variant, crit, neg)
+
+
+@pytest.mark.parametrize("variant", [1, 2, 3, 4])
+def test_every_plan_kernel_on_random_shapes(variant, plan_variant):
+    plan_variant(variant)
+    rng = np.random.default_rng(100 + variant)
+    for case in range(10):
+        wl = wk.Workload(f"planvar{variant}-{case}", cfg_id=300 + case, batch=int(rng.integers(1, 3)),
+                         heads=int(rng.integers(1, 4)), tokens=int(rng.integers(1, 40000)), head_dim=64,
+                         block=int(rng.choice([64, 128])), crit=float(rng.choice([0.0, 0.02, 0.1, 0.3, 1.0])),
+                         neg=float(rng.choice([0.0, 0.2, 0.6, 0.9])), centres=int(rng.choice([0, 8, 64])), sigma=0.3,
+                         src_dtype="bf16")
+        inputs = wk.make_inputs(wl)
+        eng = plan_only(inputs, wl)
+        heads = list(range(wl.heads))
+        ref = oracle_subset(inputs, wl, heads, query_blocks=[])
+        flips, _ = pu.compare_plan(eng, ref["scores"], ref["cls"], heads)
+        if flips:
+            print(f"{wl.name}: {flips} class entries differ at pooled-score ties <= {pu.TIE_TOL}")
 
 
 # ------------------------------------------------------------------------------------------------ benchmark shapes
