@@ -53,6 +53,9 @@ aggregate_mma_kernel(const __grid_constant__ CUtensorMap map_s, const signed cha
     if (threadIdx.x == 0 && status != nullptr) atomicCAS(status, 0, 901);
     return;
   }
+  // The attention kernel that follows needs this kernel's results only at its very end: it may be scheduled as soon
+  // as every CTA of this grid has started (it waits for the grid's completion itself before it reads G and zeta).
+  sm100::launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_tile = blockIdx.x;           // 0..16, 256 summary columns each (the last one holds zeta)
   // Rows and keys are numbered through all (b, h): row R = (b h) Nb + i, key (b h) Nb + j, the row numbers of the class

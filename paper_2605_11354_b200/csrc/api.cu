@@ -94,6 +94,7 @@ static bool g_profile = false;
 static cudaEvent_t g_events[8] = {};
 static bool g_marked[8] = {};
 
+bool profile_enabled() { return g_profile; }
 void profile_mark(int idx, cudaStream_t stream) {
   if (!g_profile) return;
   if (idx == 0)

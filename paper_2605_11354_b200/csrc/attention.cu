@@ -260,11 +260,6 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           tma_load_2d(smem + kOffQ, &map_q, &bars->q_full, 0, static_cast<int>((bh_rows + i_q[0]) * 128));
           tma_load_2d(smem + kOffQ + 4096, &map_q, &bars->q_full, 0, static_cast<int>((bh_rows + i_q[0]) * 128 + 64));
         }
-        if (p.k_marg > 0) {  // the denominators of the linear branch have a place of their own: fetched right away
-          mbar_arrive_expect_tx(&bars->z_full, kHalves * 256);
-          for (int hf = 0; hf < kHalves; ++hf)
-            bulk_load(smem + kOffZeta + hf * 256, p.zeta + (bh_rows + i_q[hf]) * kHeadDim, 256, &bars->z_full);
-        }
       }
       const float sq0 = __ldg(p.q_scales + bh_rows + i_q[0]) * (kLog2e * 0.125f);
       const float sq1 = __ldg(p.q_scales + bh_rows + i_q[1]) * (kLog2e * 0.125f);
@@ -342,7 +337,13 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         // completed: well before the last P V products, so this load is off the tail's critical path.
         for (int u = max(0, steps - kStages); u < steps && ok; ++u)
           ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars->k_free[u % kStages], (u / kStages) & 1, abort_flag, p.status, 103, kBackoffNs));
+        // G and zeta come from the kernel enqueued just before this one, which may still be running when this kernel
+        // was launched to overlap with it: everything above reads older results only.
+        wait_for_prior_grid();
         if (ok && leader) {
+          mbar_arrive_expect_tx(&bars->z_full, kHalves * 256);
+          for (int hf = 0; hf < kHalves; ++hf)
+            bulk_load(smem + kOffZeta + hf * 256, p.zeta + (bh_rows + i_q[hf]) * kHeadDim, 256, &bars->z_full);
           mbar_arrive_expect_tx(&bars->g_full, kHalves * 8192);
           for (int hf = 0; hf < kHalves; ++hf)
             tma_load_2d(smem + kOffG + hf * 8192, &map_g, &bars->g_full, 0, static_cast<int>((bh_rows + i_q[hf]) * 64));
@@ -484,10 +485,10 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     };
 
     // linear branch, first part: this thread's 32 columns (warpgroup w -> columns 32 w ..) of phi(q) as bf16 A operand
-    // of the linear product, partial denominator phi(q) . zeta_i on the side.  It needs the Q tile and zeta_i only, so
-    // it is computed while the first key tiles are on their way and the softmax threads would be idle; the operand
-    // has a shared-memory region of its own and the linear product can then be issued as soon as the aggregated
-    // summaries have arrived and the last scores have been read.
+    // of the linear product.  It needs the Q tile only, so it is computed while the first key tiles are on their way
+    // and the softmax threads would be idle; the operand has a shared-memory region of its own and the linear product
+    // can then be issued as soon as the aggregated summaries have arrived and the last scores have been read.  The
+    // denominators phi(q) . zeta_i follow in the epilogue, from the operand's own rounded values.
     // The query row comes from the Q tile in shared memory (64-byte rows, 64B swizzle: 16-byte chunk c of row r sits at
     // chunk c ^ ((r >> 1) & 3)).
     // The loops over 16-column chunks here and in the epilogue are deliberately NOT unrolled: the kernel's code has to
@@ -496,7 +497,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     float den = 0.f;
     const int swz = p_row & 7;
     if (p.k_marg > 0) {
-      ok = mbar_wait_far(&bars->q_full, 0, abort_flag, p.status, 307) && mbar_wait_far(&bars->z_full, 0, abort_flag, p.status, 308);
+      ok = mbar_wait_far(&bars->q_full, 0, abort_flag, p.status, 307);
       const uint8_t* qrow = smem + kOffQ + p_row * 64;
       const int qswz = (p_row >> 1) & 3;
       // phi = softmax over the components: any common shift of the exponents cancels in the ratio numerator /
@@ -523,20 +524,16 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         shift = fmaxf(fmaxf(mxq[0], mxq[1]), fmaxf(mxq[2], mxq[3])) * cq;  // sq > 0 commutes with max
       }
       uint8_t* const phirow = smem + kOffPhi + p_row * 128;
-      float den4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 1
       for (int cc = 0; cc < 2; ++cc) {  // this warpgroup's two chunks of 16 components
         const int c4 = 2 * w + cc;
         const uint4 raw = *reinterpret_cast<const uint4*>(qrow + ((c4 ^ qswz) << 4));
         const uint32_t words[4] = {raw.x, raw.y, raw.z, raw.w};
-        const float4* zeta = reinterpret_cast<const float4*>(smem + kOffZeta + hf * 256 + c4 * 64);
         uint32_t pk8[8];
 #pragma unroll
         for (int xw = 0; xw < 4; ++xw) {
           float fv[4];
           e4m3x4_to_float(words[xw], fv);
-          const float4 z = zeta[xw];
-          const float zz[4] = {z.x, z.y, z.z, z.w};
 #pragma unroll
           for (int y = 0; y < 4; y += 2) {
             float e0, e1;
@@ -547,17 +544,12 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               e0 = fv[y] > 0.f ? fmaf(fv[y], sq, 1.f) : ex2(fv[y] * cq);
               e1 = fv[y + 1] > 0.f ? fmaf(fv[y + 1], sq, 1.f) : ex2(fv[y + 1] * cq);
             }
-            const uint32_t pk = pack_bf162(e0, e1);
-            pk8[xw * 2 + (y >> 1)] = pk;
-            // the denominator uses the same rounded values as the MMA's numerator
-            den4[y] = fmaf(__uint_as_float(pk << 16), zz[y], den4[y]);
-            den4[y + 1] = fmaf(__uint_as_float(pk & 0xFFFF0000u), zz[y + 1], den4[y + 1]);
+            pk8[xw * 2 + (y >> 1)] = pack_bf162(e0, e1);
           }
         }
         *reinterpret_cast<uint4*>(phirow + (((c4 * 2) ^ swz) << 4)) = make_uint4(pk8[0], pk8[1], pk8[2], pk8[3]);
         *reinterpret_cast<uint4*>(phirow + (((c4 * 2 + 1) ^ swz) << 4)) = make_uint4(pk8[4], pk8[5], pk8[6], pk8[7]);
       }
-      den = (den4[0] + den4[1]) + (den4[2] + den4[3]);
       fence_proxy_async_smem();
       mbar_arrive(&bars->phi_full);
     }
@@ -649,6 +641,31 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(&bars->p_full[w]);
+    }
+
+    // linear branch, second part: partial denominator phi(q) . zeta_i over this thread's 32 columns, with the same
+    // rounded values as the numerator's operand (read back from shared memory); zeta_i arrives with the aggregated
+    // summaries at the end of the producer's work
+    if (ok && p.k_marg > 0) {
+      ok = mbar_wait_far(&bars->z_full, 0, abort_flag, p.status, 308);
+      const uint8_t* const phirow = smem + kOffPhi + p_row * 128;
+      float den4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+      for (int ch = 0; ch < 4; ++ch) {  // 16-byte chunks of eight components
+        const int c8 = 4 * w + ch;
+        const uint4 raw = *reinterpret_cast<const uint4*>(phirow + ((c8 ^ swz) << 4));
+        const uint32_t words[4] = {raw.x, raw.y, raw.z, raw.w};
+        const float4* zeta = reinterpret_cast<const float4*>(smem + kOffZeta + hf * 256 + c8 * 32);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const float4 z = zeta[half];
+          den4[0] = fmaf(__uint_as_float(words[2 * half] << 16), z.x, den4[0]);
+          den4[1] = fmaf(__uint_as_float(words[2 * half] & 0xFFFF0000u), z.y, den4[1]);
+          den4[2] = fmaf(__uint_as_float(words[2 * half + 1] << 16), z.z, den4[2]);
+          den4[3] = fmaf(__uint_as_float(words[2 * half + 1] & 0xFFFF0000u), z.w, den4[3]);
+        }
+      }
+      den = (den4[0] + den4[1]) + (den4[2] + den4[3]);
     }
 
     // the two threads of a row (one per warpgroup) bring their row sums to the final reference and swap them together
@@ -807,6 +824,23 @@ lite3r_status launch(const AttentionLaunch& a, cudaStream_t stream) {
   st = ensure_dynamic_smem(attention_kernel<BS>, static_cast<int>(kSmemBytes));
   if (st != LITE3R_OK) return st;
   const int ctas = s.batch * s.heads * (BS == 64 ? (nb + 1) / 2 : nb);
+  if (a.overlap_prior) {
+    // programmatic dependent launch: the kernel may start while the preceding one (which announces it early) is
+    // still running, and waits for its completion itself before it reads that kernel's results
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(ctas));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, attention_kernel<BS>, map_q, map_k, map_v, map_g, p);
+    if (err != cudaSuccess) return record_cuda(err);
+    return after_launch();
+  }
   attention_kernel<BS><<<ctas, kThreads, kSmemBytes, stream>>>(map_q, map_k, map_v, map_g, p);
   return after_launch();
 }

@@ -24,6 +24,7 @@ lite3r_status after_launch();
 // Benchmark stage timing: records event `idx` (0..7; stage s runs from event 2s to 2s+1) on `stream` when
 // profiling is enabled.
 void profile_mark(int idx, cudaStream_t stream);
+bool profile_enabled();
 
 // Number of SMs of the current device (looked up once per device).
 lite3r_status sm_count(int* count);
@@ -119,6 +120,7 @@ struct AttentionLaunch {
   int out_dtype;  // lite3r_dtype of the output
   long long out_stride_b, out_stride_h, out_stride_n;
   int* device_status;
+  bool overlap_prior;  // the preceding launch in the stream produced only g16 and zeta: start before it has finished
 };
 lite3r_status launch_attention(const AttentionLaunch& a, cudaStream_t stream);
 

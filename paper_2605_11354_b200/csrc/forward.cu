@@ -160,6 +160,9 @@ lite3r_status run_forward(const ForwardArgs& a, int phases, cudaStream_t stream)
   att.out_stride_h = a.out_stride_h;
   att.out_stride_n = a.out_stride_n;
   att.device_status = a.device_status;
+  // With a linear branch the kernel enqueued just before the attention kernel is the aggregation, whose results the
+  // attention kernel needs only in its tail: the two may overlap (not while stage events sit between them).
+  att.overlap_prior = a.plan.k_marg > 0 && !profile_enabled();
   profile_mark(6, stream);
   st = launch_attention(att, stream);
   profile_mark(7, stream);
