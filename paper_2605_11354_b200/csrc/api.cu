@@ -148,6 +148,21 @@ lite3r_status make_tensor_map_3d(CUtensorMap* map, CUtensorMapDataType type, int
   return r == CUDA_SUCCESS ? LITE3R_OK : LITE3R_ERR_CUDA;
 }
 
+// Rank-4 map over a tensor whose innermost dimension is contiguous: extents dims[0..3], byte strides of dimensions
+// 1..3 (multiples of 16), box of box[0..3] elements.
+lite3r_status make_tensor_map_4d(CUtensorMap* map, CUtensorMapDataType type, const void* base, const uint64_t dims[4],
+                                 const uint64_t strides_bytes[3], const uint32_t box[4], CUtensorMapSwizzle swizzle) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return LITE3R_ERR_CUDA;
+  const cuuint64_t d[4] = {dims[0], dims[1], dims[2], dims[3]};
+  const cuuint64_t st[3] = {strides_bytes[0], strides_bytes[1], strides_bytes[2]};
+  const cuuint32_t bx[4] = {box[0], box[1], box[2], box[3]};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  const CUresult r = fn(map, type, 4, const_cast<void*>(base), d, st, bx, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle,
+                        CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? LITE3R_OK : LITE3R_ERR_CUDA;
+}
+
 Counts class_counts(int nb, double crit, double neg) {
   Counts c;
   if (crit == 0.0) {

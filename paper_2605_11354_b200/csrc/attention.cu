@@ -27,6 +27,8 @@
 // their waits block on mbarriers, nothing polls), warp 3 idle, warps 4-7 / 8-11 = softmax warpgroups 0 / 1.  The
 // control warps give registers back (setmaxnreg) so that a softmax thread can hold a whole row of scores.
 // Every wait is bounded (1 s); on expiry the CTA sets *device_status and all roles leave their loops.
+#include <utility>
+
 #include "common.cuh"
 #include "sm100.cuh"
 
@@ -89,6 +91,9 @@ struct AttnParams {
   void* out;
   long long out_stride_b, out_stride_h, out_stride_n;
   int heads, tokens, nb, k_crit, k_marg, phi, out_dtype;
+  // output through TMA stores (map_o): position of the token / head / batch dimension among the map's dimensions
+  // 1..3 (they are ordered by stride); tma_out = 0: plain stores
+  int tma_out, dim_token, dim_head, dim_batch;
   int* status;
 };
 
@@ -179,7 +184,7 @@ template <int BS>
 __global__ void __launch_bounds__(kThreads, 2)
 attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                  const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_g,
-                 const AttnParams p) {
+                 const __grid_constant__ CUtensorMap map_o, const AttnParams p) {
   constexpr bool kPair = (BS == 64);
   constexpr int kHalves = kPair ? 2 : 1;             // independent M=64 problems per CTA
   constexpr int kStepsPerBlock = BS / kStepKeys;     // 1 or 2
@@ -703,7 +708,14 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       const bool wide = p.out_dtype == LITE3R_F32;
       const bool to_bf16 = p.out_dtype == LITE3R_BF16;
       const uint32_t row_bytes = wide ? 256u : 128u;
-      uint8_t* const orow = smem + kOffOut + p_row * row_bytes;
+      // With TMA stores every warp stages its 32 half rows in a tile of its own (row = lane, 128 bytes with the 128B
+      // swizzle for fp32, 64 bytes with the 64B swizzle for the 16-bit types), which is the layout the store engine
+      // reads; otherwise whole rows of the 128-row tile, chunks swizzled by the row.
+      const bool tma_out = p.tma_out != 0;
+      const uint32_t half_bytes = wide ? 128u : 64u;
+      uint8_t* const warp_tile = smem + kOffOut + (warp - kCtrlWarps) * 4096;
+      const int tswz = wide ? (lane & 7) : ((lane >> 1) & 3);
+      uint8_t* const orow = tma_out ? warp_tile + lane * half_bytes : smem + kOffOut + p_row * row_bytes;
 #pragma unroll 1
       for (int cc = 0; cc < 2; ++cc) {  // 16 columns at a time
         float acc[16];
@@ -726,7 +738,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         if (wide) {
 #pragma unroll
           for (int ch = 0; ch < 4; ++ch)
-            *reinterpret_cast<float4*>(orow + (((w * 8 + cc * 4 + ch) ^ swz) << 4)) =
+            *reinterpret_cast<float4*>(orow + ((tma_out ? ((cc * 4 + ch) ^ tswz) : ((w * 8 + cc * 4 + ch) ^ swz)) << 4)) =
                 make_float4(acc[4 * ch], acc[4 * ch + 1], acc[4 * ch + 2], acc[4 * ch + 3]);
         } else {
 #pragma unroll
@@ -736,10 +748,33 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             for (int y = 0; y < 4; ++y)
               pk[y] = to_bf16 ? pack_bf162(acc[8 * ch + 2 * y], acc[8 * ch + 2 * y + 1])
                               : pack_half2(acc[8 * ch + 2 * y], acc[8 * ch + 2 * y + 1]);
-            *reinterpret_cast<uint4*>(orow + (((w * 4 + cc * 2 + ch) ^ swz) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            *reinterpret_cast<uint4*>(orow + ((tma_out ? ((cc * 2 + ch) ^ tswz) : ((w * 4 + cc * 2 + ch) ^ swz)) << 4)) =
+                make_uint4(pk[0], pk[1], pk[2], pk[3]);
           }
         }
       }
+      if (tma_out) {
+        // two boxes of 16 rows x 32 columns per warp: lanes 0-15 and 16-31 hold 16 consecutive tokens each (of the two
+        // query blocks of a pair, or of the two halves of the warp's 32 rows); rows past the end of the sequence are
+        // clipped by the store engine, the copy of the last block in an odd pair is not stored at all
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+#pragma unroll
+          for (int g2 = 0; g2 < 2; ++g2) {
+            const int token0 = kPair ? i_q[g2] * BS + quarter * 16 : i_q[0] * BS + quarter * 32 + 16 * g2;
+            if (token0 >= p.tokens || (kPair && g2 == 1 && i_q[1] == i_q[0])) continue;
+            int c[4] = {w * 32, 0, 0, 0};
+            c[p.dim_token] = token0;
+            c[p.dim_head] = h;
+            c[p.dim_batch] = bb;
+            tma_store_4d(&map_o, warp_tile + g2 * 16 * half_bytes, c[0], c[1], c[2], c[3]);
+          }
+          bulk_commit_group();
+          bulk_wait_group_read0();  // the tile must stay in place until the engine has read it
+        }
+        __syncwarp();
+      } else {
       __syncwarp();
       const int chunk_shift = wide ? 3 : 2;       // 8 or 4 chunks of 16 bytes per half row
       const int ch = lane & ((1 << chunk_shift) - 1);
@@ -762,6 +797,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         if (r_token < p.tokens && !(second_block_is_copy && r_hf == 1))
           *reinterpret_cast<uint4*>(out_bh + r_token * row_pitch) = val;
       }
+      }
     }
   }
 
@@ -782,10 +818,14 @@ lite3r_status launch(const AttentionLaunch& a, cudaStream_t stream) {
   // The four tensor maps depend on the buffers and the shape only; a caller that runs the same buffers again (the
   // usual serving loop) reuses the encoded maps of its previous call (one entry per calling thread).
   struct MapCache {
-    alignas(64) CUtensorMap q, k, v, g;
+    alignas(64) CUtensorMap q, k, v, g, o;
     const void* key[4] = {nullptr, nullptr, nullptr, nullptr};
     uint64_t tiles = 0;
     int block = 0;
+    // the output map
+    const void* out = nullptr;
+    long long out_strides[3] = {0, 0, 0};
+    int out_dims[3] = {0, 0, 0}, out_dtype = -1, out_ok = 0, dim_token = 1, dim_head = 2, dim_batch = 3;
   };
   thread_local MapCache cache;
   lite3r_status st;
@@ -803,8 +843,68 @@ lite3r_status launch(const AttentionLaunch& a, cudaStream_t stream) {
     cache.tiles = tiles;
     cache.block = BS;
   }
+  // The output goes through TMA stores when a tiled map can describe it: the token, head and batch dimensions ordered
+  // by stride (dimensions of extent 1 last), 16 tokens x 32 columns per box.  If the driver refuses the map the kernel
+  // falls back to plain stores.
+  if (cache.out != a.out || cache.out_dtype != a.out_dtype || cache.out_strides[0] != a.out_stride_n ||
+      cache.out_strides[1] != a.out_stride_h || cache.out_strides[2] != a.out_stride_b || cache.out_dims[0] != s.tokens ||
+      cache.out_dims[1] != s.heads || cache.out_dims[2] != s.batch) {
+    const int elem = a.out_dtype == LITE3R_F32 ? 4 : 2;
+    struct Dim {
+      long long stride;
+      int extent, which;  // which: 0 token, 1 head, 2 batch
+    } dm[3] = {{a.out_stride_n, s.tokens, 0}, {a.out_stride_h, s.heads, 1}, {a.out_stride_b, s.batch, 2}};
+    // order: extents above 1 by ascending stride, then the extent-1 dimensions (whose stride does not matter)
+    auto before = [](const Dim& x, const Dim& y) {
+      if ((x.extent > 1) != (y.extent > 1)) return x.extent > 1;
+      if (x.extent > 1 && x.stride != y.stride) return x.stride < y.stride;
+      return x.which < y.which;
+    };
+    for (int i = 0; i < 3; ++i)
+      for (int j = i + 1; j < 3; ++j)
+        if (before(dm[j], dm[i])) std::swap(dm[i], dm[j]);
+    uint64_t dims[4] = {kHeadDim, 0, 0, 0}, strides[3];
+    uint32_t box[4] = {32, 1, 1, 1};
+    uint64_t packed = static_cast<uint64_t>(kHeadDim) * elem;  // stride a dimension would have if packed after the previous ones
+    bool ok = (reinterpret_cast<uintptr_t>(a.out) & 15u) == 0;
+    for (int i = 0; i < 3; ++i) {
+      dims[i + 1] = static_cast<uint64_t>(dm[i].extent);
+      strides[i] = dm[i].extent > 1 ? static_cast<uint64_t>(dm[i].stride) * elem : packed;
+      ok = ok && strides[i] > 0 && (strides[i] & 15u) == 0;
+      packed = strides[i] * dims[i + 1];
+      if (dm[i].which == 0) {
+        box[i + 1] = 16;
+        cache.dim_token = i + 1;
+      } else if (dm[i].which == 1) {
+        cache.dim_head = i + 1;
+      } else {
+        cache.dim_batch = i + 1;
+      }
+    }
+    cache.out_ok = 0;
+    if (ok) {
+      const CUtensorMapDataType type = a.out_dtype == LITE3R_F32    ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                       : a.out_dtype == LITE3R_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
+                                                                    : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
+      const CUtensorMapSwizzle swz = a.out_dtype == LITE3R_F32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+      cache.out_ok = make_tensor_map_4d(&cache.o, type, a.out, dims, strides, box, swz) == LITE3R_OK ? 1 : 0;
+    }
+    cache.out = a.out;
+    cache.out_dtype = a.out_dtype;
+    cache.out_strides[0] = a.out_stride_n;
+    cache.out_strides[1] = a.out_stride_h;
+    cache.out_strides[2] = a.out_stride_b;
+    cache.out_dims[0] = s.tokens;
+    cache.out_dims[1] = s.heads;
+    cache.out_dims[2] = s.batch;
+  }
   const CUtensorMap &map_q = cache.q, &map_k = cache.k, &map_v = cache.v, &map_g = cache.g;
+  const CUtensorMap& map_o = cache.out_ok ? cache.o : cache.q;  // any valid map when it is not used
   AttnParams p;
+  p.tma_out = cache.out_ok;
+  p.dim_token = cache.dim_token;
+  p.dim_head = cache.dim_head;
+  p.dim_batch = cache.dim_batch;
   p.q_scales = a.q_scales;
   p.k_scales = a.k_scales;
   p.crit_idx = a.crit_idx;
@@ -837,11 +937,11 @@ lite3r_status launch(const AttentionLaunch& a, cudaStream_t stream) {
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const cudaError_t err = cudaLaunchKernelEx(&cfg, attention_kernel<BS>, map_q, map_k, map_v, map_g, p);
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, attention_kernel<BS>, map_q, map_k, map_v, map_g, map_o, p);
     if (err != cudaSuccess) return record_cuda(err);
     return after_launch();
   }
-  attention_kernel<BS><<<ctas, kThreads, kSmemBytes, stream>>>(map_q, map_k, map_v, map_g, p);
+  attention_kernel<BS><<<ctas, kThreads, kSmemBytes, stream>>>(map_q, map_k, map_v, map_g, map_o, p);
   return after_launch();
 }
 

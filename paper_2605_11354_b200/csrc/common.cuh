@@ -151,6 +151,8 @@ lite3r_status launch_qkv_project(const uint8_t* x_codes, const float* x_scales, 
 
 // The same for a 3-D tensor [planes][rows][inner] with a box of box_inner x box_rows x 1 (rows past the end of a plane
 // are zero-filled, so a tile never runs into the next plane).
+lite3r_status make_tensor_map_4d(CUtensorMap* map, CUtensorMapDataType type, const void* base, const uint64_t dims[4],
+                                 const uint64_t strides_bytes[3], const uint32_t box[4], CUtensorMapSwizzle swizzle);
 lite3r_status make_tensor_map_3d(CUtensorMap* map, CUtensorMapDataType type, int elem_bytes, const void* base,
                                  uint64_t inner, uint64_t rows, uint64_t planes, uint32_t box_inner, uint32_t box_rows,
                                  CUtensorMapSwizzle swizzle);
