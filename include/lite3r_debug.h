@@ -38,6 +38,11 @@ LITE3R_API long long lite3r_launch_count(void);
  * return LITE3R_ERR_UNSUPPORTED.  Process-wide. */
 LITE3R_API lite3r_status lite3r_plan_variant(int variant);
 
+/* Test hook: the attention kernel writes its output through TMA stores where a tiled tensor map can describe the
+ * output (always, for strides the forward accepts) and with plain vector stores otherwise.  on != 0 forces the plain
+ * stores, so that both ways can be compared; on == 0 restores the default.  Process-wide. */
+LITE3R_API lite3r_status lite3r_attention_plain_stores(int on);
+
 /* Byte offsets, inside the workspace of lite3r_sla_forward, of its six parts, for tests that inspect intermediates
  * after a forward: offsets[0] per-key-block summaries, bf16 [tiles][4160] = ((H_j W)^T as [e][d] | z_j[d]), the
  * KV summary and normaliser of Algorithm 1 per block with the projection folded in; [1] per-query-block aggregates

@@ -50,7 +50,7 @@ EXPORTS = ("lite3r_fp8_sizes", "lite3r_plan_sizes", "lite3r_forward_workspace", 
            "lite3r_sla_forward_begin", "lite3r_sla_forward_finish", "lite3r_forward_workspace_planned",
            "lite3r_workspace_layout", "lite3r_quantize_rows_fp8", "lite3r_linear_fp8", "lite3r_qkv_project_fp8",
            "lite3r_train_workspace", "lite3r_sla_linear_branch", "lite3r_mse_distill", "lite3r_proj_lin_backward",
-           "lite3r_plan_variant")
+           "lite3r_plan_variant", "lite3r_attention_plain_stores")
 STATIC_SCRATCH_BYTES = 32 << 20  # LITE3R_STATIC_SCRATCH_BYTES
 
 
@@ -123,6 +123,8 @@ def lib() -> C.CDLL:
     L.lite3r_launch_count.restype = C.c_longlong
     L.lite3r_plan_variant.argtypes = [C.c_int]
     L.lite3r_plan_variant.restype = C.c_int
+    L.lite3r_attention_plain_stores.argtypes = [C.c_int]
+    L.lite3r_attention_plain_stores.restype = C.c_int
     L.lite3r_profile_enable.argtypes = [C.c_int]
     L.lite3r_profile_enable.restype = C.c_int
     L.lite3r_profile_stage_ms.argtypes = [C.POINTER(C.c_float)]
@@ -154,6 +156,11 @@ def selftest_wait_expiry(status: torch.Tensor, limit_ns: int, stream=None) -> No
 
 def launch_count() -> int:
     return int(lib().lite3r_launch_count())
+
+
+def lite3r_attention_plain_stores(on: bool) -> None:
+    """Test hook: forces the attention kernel's plain-store output path."""
+    _check(lib().lite3r_attention_plain_stores(1 if on else 0), "lite3r_attention_plain_stores")
 
 
 def lite3r_plan_variant(variant: int) -> None:

@@ -585,6 +585,11 @@ int lite3r_last_cuda_error(void) { return g_last_cuda_error; }
 
 long long lite3r_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
+lite3r_status lite3r_attention_plain_stores(int on) {
+  lite3r::set_attention_plain_stores(on != 0 ? 1 : 0);
+  return LITE3R_OK;
+}
+
 lite3r_status lite3r_plan_variant(int variant) {
   if (variant < 0 || variant > 4) return LITE3R_ERR_INVALID_ARG;
   lite3r::set_plan_variant(variant);

@@ -27,6 +27,7 @@
 // their waits block on mbarriers, nothing polls), warp 3 idle, warps 4-7 / 8-11 = softmax warpgroups 0 / 1.  The
 // control warps give registers back (setmaxnreg) so that a softmax thread can hold a whole row of scores.
 // Every wait is bounded (1 s); on expiry the CTA sets *device_status and all roles leave their loops.
+#include <atomic>
 #include <utility>
 
 #include "common.cuh"
@@ -810,6 +811,9 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 }
 
 // ------------------------------------------------------------------------------------------------ host side
+// Test hook: non-zero makes the kernel write its output with plain stores even where a TMA map exists.
+std::atomic<int> g_plain_stores{0};
+
 template <int BS>
 lite3r_status launch(const AttentionLaunch& a, cudaStream_t stream) {
   const lite3r_shape& s = a.shape;
@@ -899,9 +903,10 @@ lite3r_status launch(const AttentionLaunch& a, cudaStream_t stream) {
     cache.out_dims[2] = s.batch;
   }
   const CUtensorMap &map_q = cache.q, &map_k = cache.k, &map_v = cache.v, &map_g = cache.g;
-  const CUtensorMap& map_o = cache.out_ok ? cache.o : cache.q;  // any valid map when it is not used
+  const bool tma_out = cache.out_ok != 0 && g_plain_stores.load(std::memory_order_relaxed) == 0;
+  const CUtensorMap& map_o = tma_out ? cache.o : cache.q;  // any valid map when it is not used
   AttnParams p;
-  p.tma_out = cache.out_ok;
+  p.tma_out = tma_out ? 1 : 0;
   p.dim_token = cache.dim_token;
   p.dim_head = cache.dim_head;
   p.dim_batch = cache.dim_batch;
@@ -946,6 +951,8 @@ lite3r_status launch(const AttentionLaunch& a, cudaStream_t stream) {
 }
 
 }  // namespace
+
+void set_attention_plain_stores(int on) { g_plain_stores.store(on, std::memory_order_relaxed); }
 
 lite3r_status launch_attention(const AttentionLaunch& a, cudaStream_t stream) {
   return a.shape.block == 64 ? launch<64>(a, stream) : launch<128>(a, stream);

@@ -123,6 +123,7 @@ struct AttentionLaunch {
   bool overlap_prior;  // the preceding launch in the stream produced only g16 and zeta: start before it has finished
 };
 lite3r_status launch_attention(const AttentionLaunch& a, cudaStream_t stream);
+void set_attention_plain_stores(int on);  // test hook, see lite3r_attention_plain_stores
 
 // Per-key-block summaries ((H_j W)^T | z_j) in bf16, one kSummaryRow-wide row per (b, h, key block).
 lite3r_status launch_summary(const lite3r_fp8& k, const lite3r_fp8& v, const float* proj, long long proj_head_stride,

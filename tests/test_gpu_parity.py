@@ -573,3 +573,39 @@ def test_step_replayed_as_a_cuda_graph():
     ref = eng.run(q, k, v, proj)
     torch.cuda.synchronize()
     assert torch.equal(out, ref) and not torch.equal(out, expected)
+
+
+@pytest.mark.parametrize("tokens,block,dtype,token_major", [(1000, 64, torch.float32, False), (7, 64, torch.float32, False),
+                                                            (1000, 128, torch.bfloat16, False), (129, 128, torch.float32, True),
+                                                            (1374, 64, torch.float16, True), (704, 64, torch.float32, False)])
+def test_plain_stores_and_tma_stores_write_the_same(tokens, block, dtype, token_major):
+    """The attention kernel's two ways of writing the output (TMA stores; plain vector stores, which it falls back to
+    when no tensor map can describe the output) must give the same bytes, ragged tails, odd block counts (the copy of
+    the last block in a pair is not stored), 16-bit types and token-major layouts included; and neither may touch
+    anything outside the rows and columns of the output."""
+    wl = small_workload(f"stores-{tokens}-{block}", tokens=tokens, block=block, batch=2, heads=3)
+    inputs = wk.make_inputs(wl)
+    eng, _ = pu.run_gpu(inputs, wl)
+    proj = torch.from_numpy(inputs["proj"]).cuda()
+    results = []
+    try:
+        for plain in (False, True):
+            lt.lite3r_attention_plain_stores(plain)
+            if token_major:  # [B, N, H, 80]: rows 80 wide, the kernel writes the first 64 columns
+                buf = torch.full((wl.batch, wl.tokens, wl.heads, 80), 7.0, dtype=dtype, device="cuda")
+                out = buf[..., :64].permute(0, 2, 1, 3)
+            else:
+                buf = torch.full((wl.batch, wl.heads, wl.tokens + 3, 64), 7.0, dtype=dtype, device="cuda")
+                out = buf[:, :, :wl.tokens]
+            eng.forward(proj, out=out)
+            torch.cuda.synchronize()
+            assert int(eng.status.item()) == 0
+            results.append(buf.clone())
+    finally:
+        lt.lite3r_attention_plain_stores(False)
+    assert torch.equal(results[0], results[1])
+    if token_major:
+        assert (results[0][..., 64:] == 7.0).all()
+    else:
+        assert (results[0][:, :, wl.tokens:] == 7.0).all()
+    assert torch.isfinite(results[0].float()).all()
