@@ -239,16 +239,18 @@ __global__ void __launch_bounds__(R * 32) plan_kernel(const int* __restrict__ q_
     auto widen = [](int v) {
       return __hiloint2double(0x43300000, v ^ static_cast<int>(0x80000000u)) - 4503601774854144.0;
     };
-    auto load16 = [&](const int* base, size_t row, bool in, int4 dst[4]) {
-      const int4* src = reinterpret_cast<const int4*>(base + row * kHeadDim + 16 * t4);
+    // `local` is a block index inside the (b, h); past the end the last block is read instead (its products land
+    // in rows or columns that are never stored), which keeps the loads free of predicates and zero fills
+    auto load16 = [&](const int* base, int local, int4 dst[4]) {
+      const int4* src = reinterpret_cast<const int4*>(base + (bh_rows + min(local, nb - 1)) * kHeadDim + 16 * t4);
 #pragma unroll
-      for (int q = 0; q < 4; ++q) dst[q] = in ? __ldg(src + q) : make_int4(0, 0, 0, 0);
+      for (int q = 0; q < 4; ++q) dst[q] = __ldg(src + q);
     };
     double q_frag[kTiles][16];
 #pragma unroll
     for (int m = 0; m < kTiles; ++m) {
       int4 qv[4];
-      load16(q_colsum, bh_rows + i0 + 8 * m + g, i0 + 8 * m + g < nb, qv);
+      load16(q_colsum, i0 + 8 * m + g, qv);
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         q_frag[m][4 * q] = widen(qv[q].x);
@@ -260,11 +262,11 @@ __global__ void __launch_bounds__(R * 32) plan_kernel(const int* __restrict__ q_
     // the scales of the two key blocks whose scores the lane ends up with travel with the column sums
     auto load_scales = [&](int j, float dst[2]) {
 #pragma unroll
-      for (int x = 0; x < 2; ++x) dst[x] = j + x < nb ? __ldg(k_scales + bh_rows + j + x) : 0.f;
+      for (int x = 0; x < 2; ++x) dst[x] = __ldg(k_scales + bh_rows + min(j + x, nb - 1));
     };
     int4 nxt[4];
     float nxt_ks[2];
-    load16(k_colsum, bh_rows + warp * 8 + g, warp * 8 + g < nb, nxt);
+    load16(k_colsum, warp * 8 + g, nxt);
     load_scales(warp * 8 + 2 * t4, nxt_ks);
     float lo[kTiles], hi[kTiles];  // range of the scores of row 8 m + g, as far as this lane sees them
 #pragma unroll
@@ -280,7 +282,7 @@ __global__ void __launch_bounds__(R * 32) plan_kernel(const int* __restrict__ q_
       for (int q = 0; q < 4; ++q) cur[q] = nxt[q];
       const float cur_ks[2] = {nxt_ks[0], nxt_ks[1]};
       if (j0 + 8 * R < nb) {
-        load16(k_colsum, bh_rows + j0 + 8 * R + g, j0 + 8 * R + g < nb, nxt);
+        load16(k_colsum, j0 + 8 * R + g, nxt);
         load_scales(j0 + 8 * R + 2 * t4, nxt_ks);
       }
       // per tile two accumulation chains (even / odd k-steps), which hide the MMA latency; four were slower
@@ -531,15 +533,17 @@ __global__ void __launch_bounds__(R * 32) plan_compact_kernel(const int* __restr
     const int tile = warp % kRowTiles, grp = warp / kRowTiles;
     const int g = lane >> 2, t4 = lane & 3;
     auto widen = [](int v) { return __int2double_rn(v); };  // exact; one instruction
-    auto load16 = [&](const int* base, size_t row, bool in, int4 dst[4]) {
-      const int4* src = reinterpret_cast<const int4*>(base + row * kHeadDim + 16 * t4);
+    // `local` is a block index inside the (b, h); past the end the last block is read instead (its products land
+    // in rows or columns that are never stored), which keeps the loads free of predicates and zero fills
+    auto load16 = [&](const int* base, int local, int4 dst[4]) {
+      const int4* src = reinterpret_cast<const int4*>(base + (bh_rows + min(local, nb - 1)) * kHeadDim + 16 * t4);
 #pragma unroll
-      for (int q = 0; q < 4; ++q) dst[q] = in ? __ldg(src + q) : make_int4(0, 0, 0, 0);
+      for (int q = 0; q < 4; ++q) dst[q] = __ldg(src + q);
     };
     double q_frag[16];
     {
       int4 qv[4];
-      load16(q_colsum, bh_rows + i0 + 8 * tile + g, i0 + 8 * tile + g < nb, qv);
+      load16(q_colsum, i0 + 8 * tile + g, qv);
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         q_frag[4 * q] = widen(qv[q].x);
@@ -550,11 +554,11 @@ __global__ void __launch_bounds__(R * 32) plan_compact_kernel(const int* __restr
     }
     auto load_scales = [&](int j, float dst[2]) {
 #pragma unroll
-      for (int x = 0; x < 2; ++x) dst[x] = j + x < nb ? __ldg(k_scales + bh_rows + j + x) : 0.f;
+      for (int x = 0; x < 2; ++x) dst[x] = __ldg(k_scales + bh_rows + min(j + x, nb - 1));
     };
     int4 nxt[4];
     float nxt_ks[2];
-    load16(k_colsum, bh_rows + grp * 8 + g, grp * 8 + g < nb, nxt);
+    load16(k_colsum, grp * 8 + g, nxt);
     load_scales(grp * 8 + 2 * t4, nxt_ks);
     float lo = INFINITY, hi = -INFINITY;
     float* const my_val = s_val + static_cast<size_t>(8 * tile + g) * pitch;
@@ -568,7 +572,7 @@ __global__ void __launch_bounds__(R * 32) plan_compact_kernel(const int* __restr
       for (int q = 0; q < 4; ++q) cur[q] = nxt[q];
       const float cur_ks[2] = {nxt_ks[0], nxt_ks[1]};
       if (j0 + 8 * kGroups < nb) {
-        load16(k_colsum, bh_rows + j0 + 8 * kGroups + g, j0 + 8 * kGroups + g < nb, nxt);
+        load16(k_colsum, j0 + 8 * kGroups + g, nxt);
         load_scales(j0 + 8 * kGroups + 2 * t4, nxt_ks);
       }
       double c[2][2] = {{0.0, 0.0}, {0.0, 0.0}};
