@@ -5,12 +5,12 @@
 //                   its epilogue: Q, K and V leave the kernel as e4m3 codes + per-(b, h, token-block) scales + column
 //                   sums in the library's own layout, so the separate quantiser pass over Q, K, V disappears.
 //
-// GEMM kernel: one CTA = one 128 x 128 output tile (128 tokens x 128 output columns = two heads of the projection).
+// GEMM kernel: persistent CTAs over 128 x 128 output tiles (128 tokens x 128 output columns = two heads of the projection).
 // Warp 0 = TMA producer (A = activation codes, B = weight codes, both K-major rows of 128 bytes, 128B swizzle, ring of
 // three stages), warp 1 = MMA issuer (four kind::f8f6f4 products of K = 32 per stage), warps 4-7 and 8-11 = epilogue of
 // the tile's first and second 64 columns (thread = token row = TMEM lane; two passes over the accumulator, maximum
 // then codes, so that a row of 64 values never has to stay in registers).  Two CTAs per SM, so one tile's epilogue
-// runs under the other's main loop.
+// runs under the other's main loop, and with two accumulators per CTA also under the CTA's own next tile.
 // Every mbarrier wait is bounded; on expiry the CTA sets *device_status and its roles leave their loops.
 #include <algorithm>
 
@@ -84,10 +84,12 @@ constexpr uint32_t kOffB = kTileM * kTileK;
 constexpr uint32_t kOffMisc = kStages * kStageBytes;  // column scales (512 B), bias (512 B), reduction slots
 constexpr uint32_t kOffBar = kOffMisc + 2048;
 constexpr uint32_t kSmemBytes = kOffBar + 256;  // 100608 B: two CTAs per SM
-constexpr uint32_t kTmemCols = 128;
+constexpr uint32_t kAccCols = 128;              // one accumulator (128 x 128 fp32)
+constexpr uint32_t kTmemCols = 2 * kAccCols;    // two of them: the products of the next tile run under this tile's epilogue
 
 struct Bars {
-  uint64_t full[kStages], empty[kStages], acc_full;
+  uint64_t full[kStages], empty[kStages];
+  uint64_t acc_full[2], acc_empty[2];  // accumulator written (issuer -> epilogue) / read out (epilogue -> issuer)
   uint32_t tmem_base;
   int abort;
 };
@@ -97,6 +99,7 @@ struct LinearParams {
   const float* w_scales;  // [d_out]
   const float* bias;      // [d_out] or null
   int rows, d_in, d_out;
+  int col_tiles, tiles;   // output tiles per row of tiles, and in all
   // plain output
   void* y;
   long long y_stride;  // elements
@@ -113,6 +116,12 @@ __device__ __forceinline__ void named_barrier_sync(int id, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
+// Persistent CTAs (two per SM) walk the output tiles blockIdx.x, blockIdx.x + gridDim.x, ... (tiles of one row of
+// tiles are neighbours, so the CTAs running at any time share their activation rows in L2).  The operand ring and the
+// two accumulators are never re-initialised: ring stages and barrier parities continue on a running count of K steps,
+// the accumulators alternate with the CTA's tile count.  The producer and the issuer run ahead into the next tile
+// while the epilogue warps drain the previous accumulator: with one tile per CTA the operand loads stopped during
+// every epilogue and the kernel was bound by the latency of its loads, not by the tensor pipe or the epilogue.
 __global__ void __launch_bounds__(kThreads, 2)
 linear_fp8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                   const LinearParams p) {
@@ -128,12 +137,20 @@ linear_fp8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // row tiles never run through a batch boundary in the fused form (a tile belongs to one sequence)
   const int tiles_per_seq = ((p.fused ? p.tokens : p.rows) + kTileM - 1) / kTileM;
-  const int row_tile = blockIdx.y;
-  const int seq = row_tile / tiles_per_seq, tile_in_seq = row_tile % tiles_per_seq;
-  const int row0 = p.fused ? seq * p.tokens + tile_in_seq * kTileM : row_tile * kTileM;
-  const int rows_valid = min(kTileM, (p.fused ? p.tokens : p.rows) - tile_in_seq * kTileM);
-  const int col0 = blockIdx.x * kTileN;
   const int k_steps = p.d_in / kTileK;
+  struct TileAt {
+    int seq, tile_in_seq, row0, rows_valid, col0;
+  };
+  auto tile_at = [&](int tile_id) {
+    TileAt t;
+    const int row_tile = tile_id / p.col_tiles;
+    t.col0 = (tile_id - row_tile * p.col_tiles) * kTileN;
+    t.seq = row_tile / tiles_per_seq;
+    t.tile_in_seq = row_tile - t.seq * tiles_per_seq;
+    t.row0 = p.fused ? t.seq * p.tokens + t.tile_in_seq * kTileM : row_tile * kTileM;
+    t.rows_valid = min(kTileM, (p.fused ? p.tokens : p.rows) - t.tile_in_seq * kTileM);
+    return t;
+  };
 
   float* const s_wscale = reinterpret_cast<float*>(smem + kOffMisc);
   float* const s_bias = s_wscale + kTileN;
@@ -144,19 +161,16 @@ linear_fp8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
       mbar_init(&bars->full[s], 1);
       mbar_init(&bars->empty[s], 1);
     }
-    mbar_init(&bars->acc_full, 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&bars->acc_full[b], 1);
+      mbar_init(&bars->acc_empty[b], 256);
+    }
     bars->abort = 0;
     mbar_fence_init();
   }
   if (warp == 1) {
     tmem_alloc(&bars->tmem_base, kTmemCols);
     tmem_relinquish();
-  }
-  if (threadIdx.x >= 128 && threadIdx.x < 256) {  // the tile's column scales and bias
-    const int c = threadIdx.x - 128;
-    const int col = col0 + c;
-    s_wscale[c] = col < p.d_out ? __ldg(p.w_scales + col) : 0.f;
-    s_bias[c] = (p.bias != nullptr && col < p.d_out) ? __ldg(p.bias + col) : 0.f;
   }
   tc_fence_before();
   __syncthreads();
@@ -168,14 +182,18 @@ linear_fp8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
       tma_prefetch_desc(&map_x);
       tma_prefetch_desc(&map_w);
       bool ok = true;
-      for (int k = 0; ok && k < k_steps; ++k) {
-        const int st = k % kStages;
-        if (k >= kStages)
-          ok = mbar_wait(&bars->empty[st], ((k - kStages) / kStages) & 1, abort_flag, p.status, 601, 32);
-        if (!ok) break;
-        mbar_arrive_expect_tx(&bars->full[st], kStageBytes);
-        tma_load_2d(smem + st * kStageBytes, &map_x, &bars->full[st], k * kTileK, row0);
-        tma_load_2d(smem + st * kStageBytes + kOffB, &map_w, &bars->full[st], k * kTileK, col0);
+      int kc = 0;  // K steps issued so far, through all tiles
+      for (int tile_id = blockIdx.x; ok && tile_id < p.tiles; tile_id += gridDim.x) {
+        const TileAt t = tile_at(tile_id);
+        for (int k = 0; ok && k < k_steps; ++k, ++kc) {
+          const int st = kc % kStages;
+          if (kc >= kStages)
+            ok = mbar_wait(&bars->empty[st], ((kc - kStages) / kStages) & 1, abort_flag, p.status, 601, 32);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&bars->full[st], kStageBytes);
+          tma_load_2d(smem + st * kStageBytes, &map_x, &bars->full[st], k * kTileK, t.row0);
+          tma_load_2d(smem + st * kStageBytes + kOffB, &map_w, &bars->full[st], k * kTileK, t.col0);
+        }
       }
     }
   } else if (warp == 1) {
@@ -184,34 +202,57 @@ linear_fp8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
       const uint64_t a_desc0 = smem_desc(smem_u32(smem), 16, 1024, kSwizzle128);
       const uint64_t b_desc0 = smem_desc(smem_u32(smem) + kOffB, 16, 1024, kSwizzle128);
       bool ok = true;
-      for (int k = 0; ok && k < k_steps; ++k) {
-        const int st = k % kStages;
-        ok = mbar_wait(&bars->full[st], (k / kStages) & 1, abort_flag, p.status, 602);
-        if (!ok) break;
+      int kc = 0, it = 0;
+      for (int tile_id = blockIdx.x; ok && tile_id < p.tiles; tile_id += gridDim.x, ++it) {
+        const int ab = it & 1;
+        // the accumulator was last used two tiles ago: wait until the epilogue warps have read it out
+        if (it >= 2) ok = mbar_wait(&bars->acc_empty[ab], ((it - 2) >> 1) & 1, abort_flag, p.status, 604);
         tc_fence_after();
-        const uint64_t off = static_cast<uint64_t>((st * kStageBytes) >> 4);
+        for (int k = 0; ok && k < k_steps; ++k, ++kc) {
+          const int st = kc % kStages;
+          ok = mbar_wait(&bars->full[st], (kc / kStages) & 1, abort_flag, p.status, 602);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t off = static_cast<uint64_t>((st * kStageBytes) >> 4);
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk)
-          mma_f8(tmem, a_desc0 + off + ((kk * 32) >> 4), b_desc0 + off + ((kk * 32) >> 4), idesc, (k > 0 || kk > 0) ? 1u : 0u);
-        mma_commit(&bars->empty[st]);
+          for (int kk = 0; kk < 4; ++kk)
+            mma_f8(tmem + ab * kAccCols, a_desc0 + off + ((kk * 32) >> 4), b_desc0 + off + ((kk * 32) >> 4), idesc,
+                   (k > 0 || kk > 0) ? 1u : 0u);
+          mma_commit(&bars->empty[st]);
+        }
+        if (ok) mma_commit(&bars->acc_full[ab]);
       }
-      if (ok) mma_commit(&bars->acc_full);
     }
   } else if (warp >= 4) {
     // ------------------------------------------------------------------------------------------ epilogue
     const int quarter = warp & 3;
     const int hh = (warp - 4) >> 2;     // which 64-column half of the tile this warpgroup owns
     const int r = quarter * 32 + lane;  // row of the tile = TMEM lane
+    const int tid = threadIdx.x - (4 + hh * 4) * 32;  // thread of the warpgroup
+    float* const wsc = s_wscale + hh * 64;
+    float* const bia = s_bias + hh * 64;
+    const int bar_id = 1 + hh;
+    bool ok = true;
+    int it = 0;
+    for (int tile_id = blockIdx.x; ok && tile_id < p.tiles; tile_id += gridDim.x, ++it) {
+    const TileAt ta = tile_at(tile_id);
+    const int row0 = ta.row0, rows_valid = ta.rows_valid, seq = ta.seq, tile_in_seq = ta.tile_in_seq;
+    const int ab = it & 1;
     const bool row_ok = r < rows_valid;
-    const uint32_t acc_addr = tmem + ((static_cast<uint32_t>(quarter) * 32u) << 16) + hh * 64;
+    const uint32_t acc_addr = tmem + ((static_cast<uint32_t>(quarter) * 32u) << 16) + ab * kAccCols + hh * 64;
     const float sx = row_ok ? __ldg(p.x_scales + row0 + r) : 0.f;
-    const float* const wsc = s_wscale + hh * 64;
-    const float* const bia = s_bias + hh * 64;
-    const int col = col0 + hh * 64;
-    bool ok = mbar_wait(&bars->acc_full, 0, abort_flag, p.status, 603);
+    const int col = ta.col0 + hh * 64;
+    // this warpgroup's 64 column scales and biases (the previous tile's were released by the barrier that ends a tile)
+    if (tid < 64) {
+      wsc[tid] = col + tid < p.d_out ? __ldg(p.w_scales + col + tid) : 0.f;
+      bia[tid] = (p.bias != nullptr && col + tid < p.d_out) ? __ldg(p.bias + col + tid) : 0.f;
+    }
+    named_barrier_sync(bar_id, 128);
+    ok = mbar_wait(&bars->acc_full[ab], (it >> 1) & 1, abort_flag, p.status, 603);
     tc_fence_after();
     ok = __all_sync(0xFFFFFFFFu, ok);
-    if (ok && col < p.d_out && !p.fused) {
+    if (!ok) break;
+    if (col < p.d_out && !p.fused) {
       // y = acc * (sx * sw) + b, written row by row (a thread owns 128 contiguous bytes per 32 fp32 columns)
       uint8_t* const yrow = static_cast<uint8_t*>(p.y) +
                             static_cast<long long>(row0 + r) * p.y_stride * (p.y_dtype == LITE3R_F32 ? 4 : 2);
@@ -220,6 +261,10 @@ linear_fp8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         uint32_t v[32];
         tmem_ld32(acc_addr + cb, v);
         tmem_wait_ld();
+        if (cb == 32) {  // the accumulator is in registers: the issuer may reuse it
+          tc_fence_before();
+          mbar_arrive(&bars->acc_empty[ab]);
+        }
         if (!row_ok) continue;
         float y[32];
 #pragma unroll
@@ -247,7 +292,7 @@ linear_fp8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
           }
         }
       }
-    } else if (ok && col < p.d_out) {
+    } else if (col < p.d_out) {
       // Fused block quantiser: this warpgroup's 64 columns are one head; each (head, token block) sub-tile gets its
       // maximum, scale, codes and column sums exactly as the stand-alone quantiser computes them from fp32 values.
       const int hd = p.heads * kHeadDim;
@@ -255,9 +300,7 @@ linear_fp8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
       const int blocks_in_tile = kTileM / p.block;            // 2 at block 64, 1 at block 128
       const int my_block = r / p.block;                       // token block of the tile this row is in
       const int block_first_warp = my_block * (p.block / 32);  // first warp (0..3) of that block in the warpgroup
-      const int bar_id = 1 + hh;
       float* const red = s_red + hh * 4;
-      uint8_t* const s_codes = smem + hh * kStageBytes;  // 128 rows x 64 bytes in stage hh (all products have completed)
       // pass 1: the row's largest magnitude, then the block's
       float amax = 0.f;
 #pragma unroll 1
@@ -276,21 +319,24 @@ linear_fp8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
       const float scale = __fdiv_rn(__fadd_rn(amax, 1e-8f), 448.0f);
       const int token_block = tile_in_seq * blocks_in_tile + my_block;
       const bool block_ok = token_block < p.nb;
-      const size_t tile_id = (static_cast<size_t>(seq) * p.heads + head) * p.nb + token_block;
-      if (block_ok && (r % p.block) == 0) p.scales[part][tile_id] = scale;
+      const size_t tile_out = (static_cast<size_t>(seq) * p.heads + head) * p.nb + token_block;
+      if (block_ok && (r % p.block) == 0) p.scales[part][tile_out] = scale;
       // pass 2: codes.  x / scale must be the IEEE quotient, but only its e4m3 rounding is kept: the quotient lies
       // between x * r_lo and x * r_hi (r = 1 / scale widened by 2^-20 either way) and rounding is monotone, so equal
       // codes of the two products are the quotient's code; otherwise the pair is redone with the division.
       const float rcp = __frcp_rn(scale);
       const float r_lo = rcp * (1.0f - 0x1p-20f), r_hi = rcp * (1.0f + 0x1p-20f);
       const bool want_colsum = p.colsum[part] != nullptr;
-      uint4* const gdst = reinterpret_cast<uint4*>(p.codes[part] + (tile_id * p.block + (r % p.block)) * kHeadDim);
-      uint4* const srow = reinterpret_cast<uint4*>(s_codes + r * 64);
+      uint4* const gdst = reinterpret_cast<uint4*>(p.codes[part] + (tile_out * p.block + (r % p.block)) * kHeadDim);
 #pragma unroll 1
       for (int cb = 0; cb < 64; cb += 32) {
         uint32_t v[32], packed[8];
         tmem_ld32(acc_addr + cb, v);
         tmem_wait_ld();
+        if (cb == 32) {  // the accumulator is in registers: the issuer may reuse it
+          tc_fence_before();
+          mbar_arrive(&bars->acc_empty[ab]);
+        }
 #pragma unroll
         for (int c = 0; c < 32; c += 4) {
           uint32_t two[2];
@@ -309,27 +355,30 @@ linear_fp8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
           gdst[cb / 16] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
           gdst[cb / 16 + 1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
         }
-        if (want_colsum) {  // 16-byte chunks rotated by the row so that the column readers below do not collide
-          srow[(cb / 16 + r) & 3] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-          srow[(cb / 16 + 1 + r) & 3] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
-        }
       }
       if (want_colsum) {
-        // one thread per (block, column) adds the code values of its column in units of 2^-9
+        // One thread per (block, column) adds the code values of its column in units of 2^-9, reading back the codes
+        // the warpgroup has just written (the barrier orders them; the loads go to L2, past the first-level cache).
         named_barrier_sync(bar_id, 128);
-        const int tid = threadIdx.x - (4 + hh * 4) * 32;
         if (tid < blocks_in_tile * 64) {
           const int blk = tid >> 6, cc = tid & 63;
-          int sum = 0;
-          for (int rr = 0; rr < p.block; ++rr) {
-            const int row = blk * p.block + rr;
-            sum += e4m3_units(s_codes[row * 64 + ((((cc >> 4) + row) & 3) << 4) + (cc & 15)]);
-          }
           const int tb = tile_in_seq * blocks_in_tile + blk;
-          if (tb < p.nb) p.colsum[part][((static_cast<size_t>(seq) * p.heads + head) * p.nb + tb) * kHeadDim + cc] = sum;
+          if (tb < p.nb) {
+            const size_t out_tile = (static_cast<size_t>(seq) * p.heads + head) * p.nb + tb;
+            const uint8_t* src = p.codes[part] + out_tile * p.block * kHeadDim + cc;
+            int sum = 0;
+#pragma unroll 8
+            for (int rr = 0; rr < p.block; ++rr) sum += e4m3_units(__ldcg(src + rr * kHeadDim));
+            p.colsum[part][out_tile * kHeadDim + cc] = sum;
+          }
         }
       }
+    } else {
+      tc_fence_before();
+      mbar_arrive(&bars->acc_empty[ab]);  // nothing to do for columns past the output
     }
+    named_barrier_sync(bar_id, 128);  // the column scales, biases and reduction slots are rewritten for the next tile
+    }  // tiles
   }
 
   tc_fence_before();
@@ -349,8 +398,13 @@ lite3r_status launch_gemm(const uint8_t* x_codes, const uint8_t* w_codes, const 
                                CU_TENSOR_MAP_SWIZZLE_128B)) != LITE3R_OK) return st;
   if ((st = ensure_dynamic_smem(linear_fp8_kernel, static_cast<int>(kSmemBytes))) != LITE3R_OK) return st;
   const int row_tiles = p.fused ? p.batch * ceil_div(p.tokens, kTileM) : ceil_div(p.rows, kTileM);
-  const dim3 grid(ceil_div(p.d_out, kTileN), row_tiles);
-  linear_fp8_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_x, map_w, p);
+  LinearParams q = p;
+  q.col_tiles = ceil_div(p.d_out, kTileN);
+  q.tiles = q.col_tiles * row_tiles;
+  int sms = 0;
+  if ((st = sm_count(&sms)) != LITE3R_OK) return st;
+  const int grid = q.tiles < 2 * sms ? q.tiles : 2 * sms;
+  linear_fp8_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_x, map_w, q);
   return after_launch();
 }
 
