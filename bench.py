@@ -555,6 +555,9 @@ def run_ours(args, wl):
             "e2e": {"value": e2e_flops / 1e12, "unit": UNIT, "h2d_bytes_per_step": in_bytes,
                     "d2h_bytes_per_step": out_bytes},
             "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline}
+    if world == 1 and args.no_per_config and args.projection:
+        # the qkv projection in front of this workload alone (what profiles of the FP8 GEMM are taken on)
+        line["per_config"] = [measure_projection(lt, wl, device, flush, peaks)]
     if world == 1 and not args.no_per_config:
         del dev, eng
         clocks_all = ClockSampler(local_rank)
@@ -579,6 +582,8 @@ def main():
     ap.add_argument("--oracle-blocks", type=int, default=512)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-config", action="store_true", help="skip the table over all configurations")
+    ap.add_argument("--projection", action="store_true",
+                    help="with --no-per-config: still measure the FP8 qkv projection in front of the workload")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     wl = wk.WORKLOADS[args.workload]
