@@ -5,12 +5,12 @@
 //                   its epilogue: Q, K and V leave the kernel as e4m3 codes + per-(b, h, token-block) scales + column
 //                   sums in the library's own layout, so the separate quantiser pass over Q, K, V disappears.
 //
-// GEMM kernel: persistent CTAs over 128 x 128 output tiles (128 tokens x 128 output columns = two heads of the projection).
-// Warp 0 = TMA producer (A = activation codes, B = weight codes, both K-major rows of 128 bytes, 128B swizzle, ring of
-// three stages), warp 1 = MMA issuer (four kind::f8f6f4 products of K = 32 per stage), warps 4-7 and 8-11 = epilogue of
-// the tile's first and second 64 columns (thread = token row = TMEM lane; two passes over the accumulator, maximum
-// then codes, so that a row of 64 values never has to stay in registers).  Two CTAs per SM, so one tile's epilogue
-// runs under the other's main loop, and with two accumulators per CTA also under the CTA's own next tile.
+// GEMM kernel: persistent CTAs (one per SM) over 128 x 256 output tiles (128 tokens x 256 output columns = four heads
+// of the projection).  Warp 0 = TMA producer (A = activation codes, B = weight codes, both K-major rows of 128 bytes,
+// 128B swizzle, ring of four stages), warp 1 = MMA issuer (four kind::f8f6f4 products of K = 32 per stage into one of
+// two accumulators), warps 4-19 = four epilogue warpgroups, one per 64 columns of the tile (thread = token row = TMEM
+// lane; two passes over the accumulator, maximum then codes, so that a row of 64 values never has to stay in
+// registers).  The products of the next tile run under the epilogue of this one.
 // Every mbarrier wait is bounded; on expiry the CTA sets *device_status and its roles leave their loops.
 #include <algorithm>
 
@@ -76,16 +76,18 @@ __global__ void __launch_bounds__(256) rowquant_kernel(const SrcT* __restrict__ 
 }
 
 // ------------------------------------------------------------------------------------------------ GEMM
-constexpr int kStages = 3;
-constexpr int kTileM = 128, kTileN = 128, kTileK = 128;  // K in bytes = e4m3 elements
-constexpr int kThreads = 384;  // 4 control warps + two epilogue warpgroups (one per 64-column half of the tile)
-constexpr uint32_t kStageBytes = kTileM * kTileK + kTileN * kTileK;  // 32 KB
+constexpr int kStages = 4;
+constexpr int kTileM = 128, kTileN = 256, kTileK = 128;  // K in bytes = e4m3 elements
+constexpr int kEpiGroups = kTileN / 64;                   // epilogue warpgroups, one per 64 columns (one head) of the tile
+constexpr int kThreads = 128 + kEpiGroups * 128;          // 4 control warps + the epilogue warpgroups
+constexpr uint32_t kStageBytes = kTileM * kTileK + kTileN * kTileK;  // 48 KB
 constexpr uint32_t kOffB = kTileM * kTileK;
-constexpr uint32_t kOffMisc = kStages * kStageBytes;  // column scales (512 B), bias (512 B), reduction slots
-constexpr uint32_t kOffBar = kOffMisc + 2048;
-constexpr uint32_t kSmemBytes = kOffBar + 256;  // 100608 B: two CTAs per SM
-constexpr uint32_t kAccCols = 128;              // one accumulator (128 x 128 fp32)
-constexpr uint32_t kTmemCols = 2 * kAccCols;    // two of them: the products of the next tile run under this tile's epilogue
+constexpr uint32_t kOffMisc = kStages * kStageBytes;  // column scales (1 KB), bias (1 KB), reduction slots, column sums
+constexpr uint32_t kOffBar = kOffMisc + 5120;  // + column sums (2 KB)
+constexpr uint32_t kSmemBytes = kOffBar + 256;  // 201984 B: one CTA per SM
+constexpr uint32_t kAccCols = kTileN;           // one accumulator (128 x 256 fp32)
+constexpr uint32_t kTmemCols = 2 * kAccCols;    // two of them (all of tensor memory): the products of the next tile run
+                                                // under this tile's epilogue
 
 struct Bars {
   uint64_t full[kStages], empty[kStages];
@@ -116,13 +118,13 @@ __device__ __forceinline__ void named_barrier_sync(int id, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
-// Persistent CTAs (two per SM) walk the output tiles blockIdx.x, blockIdx.x + gridDim.x, ... (tiles of one row of
+// Persistent CTAs (one per SM) walk the output tiles blockIdx.x, blockIdx.x + gridDim.x, ... (tiles of one row of
 // tiles are neighbours, so the CTAs running at any time share their activation rows in L2).  The operand ring and the
 // two accumulators are never re-initialised: ring stages and barrier parities continue on a running count of K steps,
 // the accumulators alternate with the CTA's tile count.  The producer and the issuer run ahead into the next tile
 // while the epilogue warps drain the previous accumulator: with one tile per CTA the operand loads stopped during
 // every epilogue and the kernel was bound by the latency of its loads, not by the tensor pipe or the epilogue.
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 1)
 linear_fp8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                   const LinearParams p) {
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -154,7 +156,8 @@ linear_fp8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
 
   float* const s_wscale = reinterpret_cast<float*>(smem + kOffMisc);
   float* const s_bias = s_wscale + kTileN;
-  float* const s_red = s_bias + kTileN;  // 16 floats
+  float* const s_red = s_bias + kTileN;  // 4 floats per epilogue warpgroup
+  int* const s_colsum = reinterpret_cast<int*>(s_red + 4 * kEpiGroups);  // 128 ints per epilogue warpgroup
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -163,7 +166,7 @@ linear_fp8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&bars->acc_full[b], 1);
-      mbar_init(&bars->acc_empty[b], 256);
+      mbar_init(&bars->acc_empty[b], kEpiGroups * 128);
     }
     bars->abort = 0;
     mbar_fence_init();
@@ -226,7 +229,7 @@ linear_fp8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
   } else if (warp >= 4) {
     // ------------------------------------------------------------------------------------------ epilogue
     const int quarter = warp & 3;
-    const int hh = (warp - 4) >> 2;     // which 64-column half of the tile this warpgroup owns
+    const int hh = (warp - 4) >> 2;     // which 64 columns of the tile this warpgroup owns
     const int r = quarter * 32 + lane;  // row of the tile = TMEM lane
     const int tid = threadIdx.x - (4 + hh * 4) * 32;  // thread of the warpgroup
     float* const wsc = s_wscale + hh * 64;
@@ -302,6 +305,9 @@ linear_fp8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
       const int block_first_warp = my_block * (p.block / 32);  // first warp (0..3) of that block in the warpgroup
       float* const red = s_red + hh * 4;
       // pass 1: the row's largest magnitude, then the block's
+      // (two columns per instruction: sx * sw and acc * (sx sw) + b as packed fp32 pairs, each lane rounded exactly
+      // as the scalar expression would be)
+      const uint64_t sx2 = pack_f32x2(sx, sx), neg0 = pack_f32x2(-0.f, -0.f);
       float amax = 0.f;
 #pragma unroll 1
       for (int cb = 0; cb < 64; cb += 32) {
@@ -309,7 +315,14 @@ linear_fp8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         tmem_ld32(acc_addr + cb, v);
         tmem_wait_ld();
 #pragma unroll
-        for (int c = 0; c < 32; ++c) amax = fmaxf(amax, fabsf(fmaf(__uint_as_float(v[c]), sx * wsc[cb + c], bia[cb + c])));
+        for (int c = 0; c < 32; c += 4) {
+          const ulonglong2 sw4 = *reinterpret_cast<const ulonglong2*>(wsc + cb + c);
+          const ulonglong2 b4 = *reinterpret_cast<const ulonglong2*>(bia + cb + c);
+          float y0, y1, y2, y3;
+          unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(v[c]), __uint_as_float(v[c + 1])), fma_f32x2(sx2, sw4.x, neg0), b4.x), y0, y1);
+          unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(v[c + 2]), __uint_as_float(v[c + 3])), fma_f32x2(sx2, sw4.y, neg0), b4.y), y2, y3);
+          amax = fmaxf(amax, fmaxf(fmaxf(fabsf(y0), fabsf(y1)), fmaxf(fabsf(y2), fabsf(y3))));
+        }
       }
       amax = warp_max(row_ok ? amax : 0.f);
       if (lane == 0) red[quarter] = amax;
@@ -326,6 +339,7 @@ linear_fp8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
       // codes of the two products are the quotient's code; otherwise the pair is redone with the division.
       const float rcp = __frcp_rn(scale);
       const float r_lo = rcp * (1.0f - 0x1p-20f), r_hi = rcp * (1.0f + 0x1p-20f);
+      const uint64_t r_lo2 = pack_f32x2(r_lo, r_lo), r_hi2 = pack_f32x2(r_hi, r_hi);
       const bool want_colsum = p.colsum[part] != nullptr;
       uint4* const gdst = reinterpret_cast<uint4*>(p.codes[part] + (tile_out * p.block + (r % p.block)) * kHeadDim);
 #pragma unroll 1
@@ -339,17 +353,27 @@ linear_fp8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         }
 #pragma unroll
         for (int c = 0; c < 32; c += 4) {
+          const ulonglong2 sw4 = *reinterpret_cast<const ulonglong2*>(wsc + cb + c);
+          const ulonglong2 b4 = *reinterpret_cast<const ulonglong2*>(bia + cb + c);
+          const unsigned long long sws[2] = {sw4.x, sw4.y}, bs[2] = {b4.x, b4.y};
           uint32_t two[2];
 #pragma unroll
           for (int h2 = 0; h2 < 2; ++h2) {
-            const float y0 = fmaf(__uint_as_float(v[c + 2 * h2]), sx * wsc[cb + c + 2 * h2], bia[cb + c + 2 * h2]);
-            const float y1 = fmaf(__uint_as_float(v[c + 2 * h2 + 1]), sx * wsc[cb + c + 2 * h2 + 1], bia[cb + c + 2 * h2 + 1]);
-            const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(y0 * r_lo, y1 * r_lo), __NV_SATFINITE, __NV_E4M3);
-            uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(y0 * r_hi, y1 * r_hi), __NV_SATFINITE, __NV_E4M3);
-            if (lo != hi) hi = quantise_pair(y0, y1, scale);
-            two[h2] = row_ok ? hi : 0u;
+            const uint64_t y2 = fma_f32x2(pack_f32x2(__uint_as_float(v[c + 2 * h2]), __uint_as_float(v[c + 2 * h2 + 1])),
+                                          fma_f32x2(sx2, sws[h2], neg0), bs[h2]);
+            float2 q_lo, q_hi;
+            unpack_f32x2(fma_f32x2(y2, r_lo2, neg0), q_lo.x, q_lo.y);
+            unpack_f32x2(fma_f32x2(y2, r_hi2, neg0), q_hi.x, q_hi.y);
+            const uint32_t lo = __nv_cvt_float2_to_fp8x2(q_lo, __NV_SATFINITE, __NV_E4M3);
+            uint32_t hi = __nv_cvt_float2_to_fp8x2(q_hi, __NV_SATFINITE, __NV_E4M3);
+            if (lo != hi) {
+              float y0, y1;
+              unpack_f32x2(y2, y0, y1);
+              hi = quantise_pair(y0, y1, scale);
+            }
+            two[h2] = hi;
           }
-          packed[c >> 2] = two[0] | (two[1] << 16);
+          packed[c >> 2] = row_ok ? (two[0] | (two[1] << 16)) : 0u;
         }
         if (block_ok) {  // rows past the sequence end inside an existing block are written as zeros
           gdst[cb / 16] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
@@ -357,20 +381,45 @@ linear_fp8_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         }
       }
       if (want_colsum) {
-        // One thread per (block, column) adds the code values of its column in units of 2^-9, reading back the codes
-        // the warpgroup has just written (the barrier orders them; the loads go to L2, past the first-level cache).
+        // Column sums of the code values (exact integers in units of 2^-9) from the codes the warpgroup has just written
+        // (the barrier orders them; the loads go to L2, past the first-level cache): a thread adds four columns over 16
+        // rows in fp32 (exact: at most 16 x 448 in steps of 2^-9), the eight row groups of the tile meet in shared memory.
+        int* const cs = s_colsum + hh * 128;  // [token block of the tile][64]
+        cs[tid] = 0;
+        named_barrier_sync(bar_id, 128);
+        {
+          const int cg = tid & 15, row_first = (tid >> 4) * 16;
+          const int blk = row_first / p.block;
+          const int tb = tile_in_seq * blocks_in_tile + blk;
+          if (tb < p.nb) {
+            const size_t out_tile = (static_cast<size_t>(seq) * p.heads + head) * p.nb + tb;
+            const uint32_t* src =
+                reinterpret_cast<const uint32_t*>(p.codes[part] + (out_tile * p.block + (row_first % p.block)) * kHeadDim) + cg;
+            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll 4
+            for (int rr = 0; rr < 16; ++rr) {
+              const uint32_t w4 = __ldcg(src + rr * (kHeadDim / 4));
+              const __half2_raw lo = __nv_cvt_fp8x2_to_halfraw2(static_cast<__nv_fp8x2_storage_t>(w4 & 0xFFFFu), __NV_E4M3);
+              const __half2_raw hi = __nv_cvt_fp8x2_to_halfraw2(static_cast<__nv_fp8x2_storage_t>(w4 >> 16), __NV_E4M3);
+              const float2 f01 = __half22float2(__half2(lo)), f23 = __half22float2(__half2(hi));
+              a0 += f01.x;
+              a1 += f01.y;
+              a2 += f23.x;
+              a3 += f23.y;
+            }
+            int* dst = cs + blk * 64 + cg * 4;
+            atomicAdd(dst, __float2int_rn(a0 * 512.f));
+            atomicAdd(dst + 1, __float2int_rn(a1 * 512.f));
+            atomicAdd(dst + 2, __float2int_rn(a2 * 512.f));
+            atomicAdd(dst + 3, __float2int_rn(a3 * 512.f));
+          }
+        }
         named_barrier_sync(bar_id, 128);
         if (tid < blocks_in_tile * 64) {
           const int blk = tid >> 6, cc = tid & 63;
           const int tb = tile_in_seq * blocks_in_tile + blk;
-          if (tb < p.nb) {
-            const size_t out_tile = (static_cast<size_t>(seq) * p.heads + head) * p.nb + tb;
-            const uint8_t* src = p.codes[part] + out_tile * p.block * kHeadDim + cc;
-            int sum = 0;
-#pragma unroll 8
-            for (int rr = 0; rr < p.block; ++rr) sum += e4m3_units(__ldcg(src + rr * kHeadDim));
-            p.colsum[part][out_tile * kHeadDim + cc] = sum;
-          }
+          if (tb < p.nb)
+            p.colsum[part][((static_cast<size_t>(seq) * p.heads + head) * p.nb + tb) * kHeadDim + cc] = cs[tid];
         }
       }
     } else {
@@ -403,7 +452,7 @@ lite3r_status launch_gemm(const uint8_t* x_codes, const uint8_t* w_codes, const 
   q.tiles = q.col_tiles * row_tiles;
   int sms = 0;
   if ((st = sm_count(&sms)) != LITE3R_OK) return st;
-  const int grid = q.tiles < 2 * sms ? q.tiles : 2 * sms;
+  const int grid = q.tiles < sms ? q.tiles : sms;
   linear_fp8_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_x, map_w, q);
   return after_launch();
 }
