@@ -635,7 +635,9 @@ __global__ void __launch_bounds__(R * 32) plan_compact_kernel(const int* __restr
   // A key's place between the row's extremes on a 16-bit scale; its upper eight bits are the bucket of the first
   // histogram, the lower eight refine a bucket that turns out too full to list.  Both are monotone in the score.
   const float scale = hi > lo ? 65535.5f / (hi - lo) : 0.f;
-  auto fine = [&](int j) -> int { return min(65535, max(0, __float2int_rz((vals[j] - lo) * scale))); };
+  // computed once, in the histogram pass, and left in place of the score (which nothing needs after that)
+  int* const places = reinterpret_cast<int*>(s_val + static_cast<size_t>(warp) * pitch);
+  auto fine = [&](int j) -> int { return places[j]; };
   // exact 64-bit key of entry j of this row (the row's own column sums wait in shared memory)
   int* const q_row = s_q + warp * kHeadDim;
   q_row[lane] = __ldg(q_colsum + (bh_rows + i) * kHeadDim + lane);
@@ -655,7 +657,11 @@ __global__ void __launch_bounds__(R * 32) plan_compact_kernel(const int* __restr
 #pragma unroll
   for (int b = 0; b < 8; ++b) bucket_hist[lane + 32 * b] = 0u;
   __syncwarp();
-  for (int j = lane; j < nb; j += 32) atomicAdd(&bucket_hist[fine(j) >> 8], 1u);
+  for (int j = lane; j < nb; j += 32) {
+    const int f = min(65535, max(0, __float2int_rz((vals[j] - lo) * scale)));
+    places[j] = f;
+    atomicAdd(&bucket_hist[f >> 8], 1u);
+  }
   __syncwarp();
 
   // A selection: entries whose place is above t_hi are selected, those inside [t_lo, t_hi] are decided by their exact
