@@ -668,17 +668,22 @@ __global__ void __launch_bounds__(R * 32) plan_compact_kernel(const int* __restr
   // keys (prefix / mask / take as in Selection), the rest are not.  Each selection leaves the entries of its
   // threshold range (ascending index) and their exact keys behind for the class pass: keys_from 0 = no key needed
   // (the whole range goes one way), 1 = listed, 2 = recompute (still too many to list after the refinement).
+  // The two selections of a row go through their stages together, so that the refinement and the listing each take
+  // one pass over the row for both.
   struct Chosen {
     Selection s;
-    int t_lo, t_hi, keys_from;
+    int t_lo, t_hi, keys_from, remaining, size;
+    bool refine, list;
   };
-  auto select = [&](int k, unsigned long long* ckey, unsigned short* idx) -> Chosen {
+  auto begin = [&](int k) -> Chosen {
     Chosen r;
     r.keys_from = 0;
     r.s.prefix = 0ull;
     r.s.mask = 0ull;
     r.s.take = 0;
     r.s.bucket = 0;
+    r.remaining = r.size = 0;
+    r.refine = r.list = false;
     if (k <= 0) {
       r.t_lo = r.t_hi = 65536;
       return r;
@@ -690,66 +695,91 @@ __global__ void __launch_bounds__(R * 32) plan_compact_kernel(const int* __restr
     const Located at = locate(bucket_hist, k, lane);
     r.t_lo = at.bin << 8;
     r.t_hi = r.t_lo + 255;
-    int remaining = k - at.above, size = at.size;
-    if (remaining == size) {
-      r.s.take = size;
-      return r;
-    }
-    if (size > kMaxListed) {  // refine: histogram of the lower eight bits inside the bucket
+    r.remaining = k - at.above;
+    r.size = at.size;
+    if (r.remaining == r.size)
+      r.s.take = r.size;
+    else if (r.size > kMaxListed)
+      r.refine = true;
+    else
+      r.list = true;
+    return r;
+  };
+  Chosen cc = begin(k_crit), cm = begin(nb - k_neg);
+  if (cc.refine || cm.refine) {  // histograms of the lower eight bits inside the two threshold buckets
 #pragma unroll
-      for (int b = 0; b < 8; ++b) hist[lane + 32 * b] = 0u;
-      __syncwarp();
-      for (int j = lane; j < nb; j += 32) {
-        const int f = fine(j);
-        if ((f >> 8) == at.bin) atomicAdd(&hist[f & 255], 1u);
-      }
-      __syncwarp();
-      const Located at2 = locate(hist, remaining, lane);
-      __syncwarp();
-      r.t_lo = r.t_hi = (at.bin << 8) | at2.bin;
-      remaining -= at2.above;
-      size = at2.size;
-      if (remaining == size) {
-        r.s.take = size;
-        return r;
-      }
+    for (int b = 0; b < 8; ++b) {
+      hist[lane + 32 * b] = 0u;
+      bucket_hist[lane + 32 * b] = 0u;  // the first histogram has served both selections
     }
-    const int t_lo = r.t_lo, t_hi = r.t_hi;
-    if (size <= kMaxListed) {
-      const unsigned below = (1u << lane) - 1u;
-      int listed = 0;
-      for (int j0 = 0; j0 < nb; j0 += 32) {
-        const int j = j0 + lane;
-        const int f = j < nb ? fine(j) : -1;
-        const bool is = f >= t_lo && f <= t_hi;
-        const unsigned b = __ballot_sync(0xFFFFFFFFu, is);
-        if (is) idx[listed + __popc(b & below)] = static_cast<unsigned short>(j);
-        listed += __popc(b);
-      }
-      __syncwarp();
-      for (int c = lane; c < size; c += 32) ckey[c] = exact_key(idx[c]);
-      __syncwarp();
+    __syncwarp();
+    const int bin_c = cc.refine ? cc.t_lo >> 8 : -1, bin_m = cm.refine ? cm.t_lo >> 8 : -1;
+    for (int j = lane; j < nb; j += 32) {
+      const int f = fine(j);
+      if ((f >> 8) == bin_c) atomicAdd(&hist[f & 255], 1u);
+      if ((f >> 8) == bin_m) atomicAdd(&bucket_hist[f & 255], 1u);
+    }
+    __syncwarp();
+    auto refined = [&](Chosen& r, const unsigned int* h) {
+      if (!r.refine) return;
+      const Located at2 = locate(h, r.remaining, lane);
+      r.t_lo = r.t_hi = (r.t_lo & ~255) | at2.bin;
+      r.remaining -= at2.above;
+      r.size = at2.size;
+      if (r.remaining == r.size)
+        r.s.take = r.size;
+      else if (r.size <= kMaxListed)
+        r.list = true;
+      else
+        r.keys_from = 2;  // more than kMaxListed entries in one of 65536 places (near-equal scores)
+    };
+    refined(cc, hist);
+    refined(cm, bucket_hist);
+    __syncwarp();
+  }
+  unsigned long long* const ckey_c = s_ckey + warp * 2 * kMaxListed;
+  unsigned long long* const ckey_m = ckey_c + kMaxListed;
+  unsigned short* const idx_c = s_idx + warp * 2 * kMaxListed;
+  unsigned short* const idx_m = idx_c + kMaxListed;
+  if (cc.list || cm.list) {  // positions of the entries inside the two threshold ranges, ascending
+    const unsigned below = (1u << lane) - 1u;
+    int listed_c = 0, listed_m = 0;
+    for (int j0 = 0; j0 < nb; j0 += 32) {
+      const int j = j0 + lane;
+      const int f = j < nb ? fine(j) : -1;
+      const bool is_c = cc.list && f >= cc.t_lo && f <= cc.t_hi, is_m = cm.list && f >= cm.t_lo && f <= cm.t_hi;
+      const unsigned b_c = __ballot_sync(0xFFFFFFFFu, is_c), b_m = __ballot_sync(0xFFFFFFFFu, is_m);
+      if (is_c) idx_c[listed_c + __popc(b_c & below)] = static_cast<unsigned short>(j);
+      if (is_m) idx_m[listed_m + __popc(b_m & below)] = static_cast<unsigned short>(j);
+      listed_c += __popc(b_c);
+      listed_m += __popc(b_m);
+    }
+    __syncwarp();
+    if (cc.list)
+      for (int c = lane; c < cc.size; c += 32) ckey_c[c] = exact_key(idx_c[c]);
+    if (cm.list)
+      for (int c = lane; c < cm.size; c += 32) ckey_m[c] = exact_key(idx_m[c]);
+    __syncwarp();
+  }
+  auto finish = [&](Chosen& r, const unsigned long long* ckey) {
+    if (r.list) {
       r.keys_from = 1;
       radix_select([&](int c, unsigned long long& key) {
         key = ckey[c];
         return true;
-      }, size, remaining, hist, lane, r.s);
-    } else {  // more than kMaxListed entries in one of 65536 places (near-equal scores): every pass recomputes keys
-      r.keys_from = 2;
+      }, r.size, r.remaining, hist, lane, r.s);
+    } else if (r.keys_from == 2) {  // every pass recomputes the keys it looks at
+      const int t_lo = r.t_lo, t_hi = r.t_hi;
       radix_select([&](int c, unsigned long long& key) {
         const int f = fine(c);
         if (f < t_lo || f > t_hi) return false;
         key = exact_key(c);
         return true;
-      }, nb, remaining, hist, lane, r.s);
+      }, nb, r.remaining, hist, lane, r.s);
     }
-    return r;
   };
-  unsigned long long* const ckey_c = s_ckey + warp * 2 * kMaxListed;
-  unsigned long long* const ckey_m = ckey_c + kMaxListed;
-  unsigned short* const idx_c = s_idx + warp * 2 * kMaxListed;
-  const Chosen cc = select(k_crit, ckey_c, idx_c);
-  const Chosen cm = select(nb - k_neg, ckey_m, idx_c + kMaxListed);
+  finish(cc, ckey_c);
+  finish(cm, ckey_m);
   const Selection sc = cc.s, sm = cm.s;
   const int from_c = cc.keys_from, from_m = cm.keys_from;
 
