@@ -44,7 +44,8 @@ __device__ __forceinline__ uint32_t quantise_pair(float a, float b, float scale)
   return __nv_cvt_float2_to_fp8x2(make_float2(__fdiv_rn(a, scale), __fdiv_rn(b, scale)), __NV_SATFINITE, __NV_E4M3);
 }
 
-// One warp per row: the row is read twice (maximum, then codes); the second read comes from L1 / L2.
+// One warp per row.  Rows of up to 1024 values are held in registers; longer ones are read twice (maximum, then codes;
+// the second read comes from L1 / L2).
 template <typename SrcT>
 __global__ void __launch_bounds__(256) rowquant_kernel(const SrcT* __restrict__ x, long long row_stride, int rows, int cols,
                                                        uint8_t* __restrict__ codes, float* __restrict__ scales) {
@@ -53,6 +54,54 @@ __global__ void __launch_bounds__(256) rowquant_kernel(const SrcT* __restrict__ 
   const int segs = cols >> 3;
   for (int row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; row < rows; row += warps) {
     const SrcT* src = x + static_cast<long long>(row) * row_stride;
+    if (segs <= 4 * 32) {
+      // rows of up to 1024 values stay in registers between the two sweeps (four 8-value segments per lane, all
+      // requested before the first is used): one pass over memory
+      float v[4][8];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        if (lane + 32 * q < segs) {
+          load8(src + (lane + 32 * q) * 8, v[q]);
+        } else {
+#pragma unroll
+          for (int c = 0; c < 8; ++c) v[q][c] = 0.f;
+        }
+      }
+      float amax = 0.f;
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+#pragma unroll
+        for (int c = 0; c < 8; ++c) amax = fmaxf(amax, fabsf(v[q][c]));
+      amax = warp_max(amax);
+      const float scale = __fdiv_rn(__fadd_rn(amax, 1e-8f), 448.0f);
+      if (lane == 0) scales[row] = scale;
+      uint8_t* dst = codes + static_cast<size_t>(row) * cols;
+      const float rcp = __frcp_rn(scale);
+      const uint64_t r_lo2 = pack_f32x2(rcp * (1.0f - 0x1p-20f), rcp * (1.0f - 0x1p-20f));
+      const uint64_t r_hi2 = pack_f32x2(rcp * (1.0f + 0x1p-20f), rcp * (1.0f + 0x1p-20f));
+      const uint64_t neg0 = pack_f32x2(-0.f, -0.f);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        if (lane + 32 * q >= segs) continue;
+        uint32_t two[4], differ = 0u;
+#pragma unroll
+        for (int c = 0; c < 8; c += 2) {
+          const uint64_t x2 = pack_f32x2(v[q][c], v[q][c + 1]);
+          float2 q_lo, q_hi;
+          unpack_f32x2(fma_f32x2(x2, r_lo2, neg0), q_lo.x, q_lo.y);
+          unpack_f32x2(fma_f32x2(x2, r_hi2, neg0), q_hi.x, q_hi.y);
+          const uint32_t lo = __nv_cvt_float2_to_fp8x2(q_lo, __NV_SATFINITE, __NV_E4M3);
+          two[c >> 1] = __nv_cvt_float2_to_fp8x2(q_hi, __NV_SATFINITE, __NV_E4M3);
+          differ |= lo ^ two[c >> 1];
+        }
+        if (differ != 0u) {  // next to a rounding boundary of the e4m3 grid: redone with the division
+#pragma unroll
+          for (int c = 0; c < 8; c += 2) two[c >> 1] = quantise_pair(v[q][c], v[q][c + 1], scale);
+        }
+        *reinterpret_cast<uint2*>(dst + (lane + 32 * q) * 8) = make_uint2(two[0] | (two[1] << 16), two[2] | (two[3] << 16));
+      }
+      continue;
+    }
     float amax = 0.f;
     for (int s = lane; s < segs; s += 32) {
       float v[8];
@@ -64,12 +113,31 @@ __global__ void __launch_bounds__(256) rowquant_kernel(const SrcT* __restrict__ 
     const float scale = __fdiv_rn(__fadd_rn(amax, 1e-8f), 448.0f);
     if (lane == 0) scales[row] = scale;
     uint8_t* dst = codes + static_cast<size_t>(row) * cols;
+    // x / scale must be the IEEE quotient, but only its e4m3 rounding is kept: the quotient lies between x * r_lo and
+    // x * r_hi (r = 1 / scale widened by 2^-20 either way) and rounding is monotone, so equal codes of the two products
+    // are the quotient's code; otherwise the eight values are redone with the division.
+    const float rcp = __frcp_rn(scale);
+    const uint64_t r_lo2 = pack_f32x2(rcp * (1.0f - 0x1p-20f), rcp * (1.0f - 0x1p-20f));
+    const uint64_t r_hi2 = pack_f32x2(rcp * (1.0f + 0x1p-20f), rcp * (1.0f + 0x1p-20f));
+    const uint64_t neg0 = pack_f32x2(-0.f, -0.f);
     for (int s = lane; s < segs; s += 32) {
       float v[8];
       load8(src + s * 8, v);
-      uint32_t two[4];
+      uint32_t two[4], differ = 0u;
 #pragma unroll
-      for (int c = 0; c < 8; c += 2) two[c >> 1] = quantise_pair(v[c], v[c + 1], scale);
+      for (int c = 0; c < 8; c += 2) {
+        const uint64_t x2 = pack_f32x2(v[c], v[c + 1]);
+        float2 q_lo, q_hi;
+        unpack_f32x2(fma_f32x2(x2, r_lo2, neg0), q_lo.x, q_lo.y);
+        unpack_f32x2(fma_f32x2(x2, r_hi2, neg0), q_hi.x, q_hi.y);
+        const uint32_t lo = __nv_cvt_float2_to_fp8x2(q_lo, __NV_SATFINITE, __NV_E4M3);
+        two[c >> 1] = __nv_cvt_float2_to_fp8x2(q_hi, __NV_SATFINITE, __NV_E4M3);
+        differ |= lo ^ two[c >> 1];
+      }
+      if (differ != 0u) {
+#pragma unroll
+        for (int c = 0; c < 8; c += 2) two[c >> 1] = quantise_pair(v[c], v[c + 1], scale);
+      }
       *reinterpret_cast<uint2*>(dst + s * 8) = make_uint2(two[0] | (two[1] << 16), two[2] | (two[3] << 16));
     }
   }
