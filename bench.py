@@ -37,7 +37,7 @@ DRAM_BYTES_PER_LAUNCH = {
     ("vggt8", "attention"): 86006528,
     ("vggt8", "plan"): 1485824,
     ("vggt8", "quantize_qkv"): 72634624,
-    ("vggt8", "summary"): 23863296,
+    ("vggt8", "summary"): 24797952,
     ("vggt8", "aggregation"): 23398144,
 }
 

@@ -261,20 +261,39 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) summary_kernel(const Sum
             }
           }
           if (p.phi == LITE3R_PHI_SOFTMAX) {
-            float mx4[4] = {x[0], x[1], x[2], x[3]};
-#pragma unroll
-            for (int d = 4; d < 64; ++d) mx4[d & 3] = fmaxf(mx4[d & 3], x[d]);
+            // Any common shift of the exponents cancels in the ratio.  448 * scale bounds every component of the block,
+            // so it serves as the shift without a pass over the row; only when exponents could then leave the fp32
+            // range (block magnitudes in the hundreds) is the row's own maximum looked up.  Arguments, sums and the
+            // normalisation run on pairs of components (packed fp32x2).
             const float c = sk * kLog2e;  // sk > 0 commutes with max
-            const float shift = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * c;
-            float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+            float shift = 448.f * c;
+            if (896.f * c > 100.f) {
+              float mx4[4] = {x[0], x[1], x[2], x[3]};
 #pragma unroll
-            for (int d = 0; d < 64; ++d) {
-              x[d] = ex2(fmaf(x[d], c, -shift));
-              sum4[d & 3] += x[d];
+              for (int d = 4; d < 64; ++d) mx4[d & 3] = fmaxf(mx4[d & 3], x[d]);
+              shift = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * c;
             }
-            const float inv = 1.f / ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
+            const uint64_t c2 = pack_f32x2(c, c), neg_shift2 = pack_f32x2(-shift, -shift);
+            uint64_t sum2[2] = {0ull, 0ull};  // bit pattern of (0.f, 0.f)
 #pragma unroll
-            for (int d = 0; d < 64; d += 2) pw[d >> 1] = float2_to_half2_bits(x[d] * inv, x[d + 1] * inv);
+            for (int d = 0; d < 64; d += 2) {
+              float a0, a1;
+              unpack_f32x2(fma_f32x2(pack_f32x2(x[d], x[d + 1]), c2, neg_shift2), a0, a1);
+              x[d] = ex2(a0);
+              x[d + 1] = ex2(a1);
+              sum2[(d >> 1) & 1] = add_f32x2(sum2[(d >> 1) & 1], pack_f32x2(x[d], x[d + 1]));
+            }
+            float s0, s1, s2, s3;
+            unpack_f32x2(sum2[0], s0, s1);
+            unpack_f32x2(sum2[1], s2, s3);
+            const float inv = 1.f / ((s0 + s1) + (s2 + s3));
+            const uint64_t inv2 = pack_f32x2(inv, inv), neg0 = pack_f32x2(-0.f, -0.f);  // x * inv + (-0) is x * inv
+#pragma unroll
+            for (int d = 0; d < 64; d += 2) {
+              float y0, y1;
+              unpack_f32x2(fma_f32x2(pack_f32x2(x[d], x[d + 1]), inv2, neg0), y0, y1);
+              pw[d >> 1] = float2_to_half2_bits(y0, y1);
+            }
           } else {
             const float c = sk * kLog2e;
 #pragma unroll
@@ -334,9 +353,13 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) summary_kernel(const Sum
           const float sv = __ldg(p.v_scales + tile);
           uint32_t hw[32];
 #pragma unroll
+          const uint64_t sv2 = pack_f32x2(sv, sv), neg0 = pack_f32x2(-0.f, -0.f);  // x * sv + (-0) is x * sv
           for (int e = 0; e < 32; e += 2) {
-            hw[e >> 1] = float2_to_half2_bits(__uint_as_float(lo[e]) * sv, __uint_as_float(lo[e + 1]) * sv);
-            hw[16 + (e >> 1)] = float2_to_half2_bits(__uint_as_float(hi[e]) * sv, __uint_as_float(hi[e + 1]) * sv);
+            float a0, a1, b0, b1;
+            unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(lo[e]), __uint_as_float(lo[e + 1])), sv2, neg0), a0, a1);
+            unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(hi[e]), __uint_as_float(hi[e + 1])), sv2, neg0), b0, b1);
+            hw[e >> 1] = float2_to_half2_bits(a0, a1);
+            hw[16 + (e >> 1)] = float2_to_half2_bits(b0, b1);
           }
           store_row_swizzled(smem + kOffV + hf * 8192, d_row, hw);
         }
