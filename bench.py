@@ -36,7 +36,7 @@ FP8_OVER_BF16 = 2.0  # nominal dense ratio (4.5 vs 2.25 PFLOP/s)
 DRAM_BYTES_PER_LAUNCH = {
     ("vggt8", "attention"): 87756288,
     ("vggt8", "plan"): 1485824,
-    ("vggt8", "quantize_qkv"): 72634624,
+    ("vggt8", "quantize_qkv"): 72396800,
     ("vggt8", "summary"): 24797952,
     ("vggt8", "aggregation"): 23398144,
 }

@@ -95,34 +95,53 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const __grid_constan
   const int stride = static_cast<int>(gridDim.x);
 
   // Copies this thread's segments of the next tile of the walk into ring slot `slot` (nothing once the walk has
-  // ended).  A position of the walk is (tensor, tile); it advances by the grid size.
-  int f_which = 0, f_tile = blockIdx.x;
-  while (f_tile >= tiles && f_which < batch.count) {
-    f_tile -= tiles;
+  // ended).  A position of the walk is (tensor, (b h), block); it advances by the grid size, which is split into whole
+  // (b h) and blocks once, so that no division sits in the per-tile path.  A full tile is copied with one running
+  // source pointer (one 64-bit add per pass); only a ragged last block takes the row-by-row form.
+  const int bh_total = tiles / nb;
+  const int step_bh = stride / nb, step_i = stride - step_bh * nb;
+  int f_which = 0, f_bh = static_cast<int>(blockIdx.x) / nb, f_i = static_cast<int>(blockIdx.x) - f_bh * nb;
+  while (f_bh >= bh_total && f_which < batch.count) {
+    f_bh -= bh_total;
     ++f_which;
   }
   auto fetch = [&](int slot) {
     if (f_which < batch.count) {
-      const int f_bh = f_tile / nb, f_i = f_tile - f_bh * nb;
       const int valid = min(BS, tokens - f_i * BS);
       const int b = f_bh / heads;
       const long long stride_n = batch.stride_n[f_which];
       const SrcT* src = static_cast<const SrcT*>(batch.x[f_which]) + b * batch.stride_b[f_which] +
                         (f_bh - b * heads) * batch.stride_h[f_which] + static_cast<long long>(f_i) * BS * stride_n + seg * 8;
+      uint8_t* const dst0 = ring + slot * kTileBytes + threadIdx.x * kSegBytes;
+      if (valid == BS) {
+        const uint8_t* g = reinterpret_cast<const uint8_t*>(src + row0 * stride_n);
+        const long long row_step = kRowsPerPass * stride_n * static_cast<long long>(sizeof(SrcT));
 #pragma unroll
-      for (int p = 0; p < kPasses; ++p) {
-        const int r = row0 + p * kRowsPerPass;
-        uint8_t* dst = ring + slot * kTileBytes + (p * kThreads + threadIdx.x) * kSegBytes;
-        const SrcT* g = src + (r < valid ? r : 0) * stride_n;  // rows past the end are zero-filled, not read
+        for (int p = 0; p < kPasses; ++p) {
 #pragma unroll
-        for (int q = 0; q < kSegBytes / 16; ++q)
-          cp_async16(dst + 16 * q, reinterpret_cast<const uint8_t*>(g) + 16 * q, r < valid ? 16u : 0u);
+          for (int q = 0; q < kSegBytes / 16; ++q) cp_async16(dst0 + p * kThreads * kSegBytes + 16 * q, g + 16 * q, 16u);
+          g += row_step;
+        }
+      } else {
+#pragma unroll
+        for (int p = 0; p < kPasses; ++p) {
+          const int r = row0 + p * kRowsPerPass;
+          const SrcT* g = src + (r < valid ? r : 0) * stride_n;  // rows past the end are zero-filled, not read
+#pragma unroll
+          for (int q = 0; q < kSegBytes / 16; ++q)
+            cp_async16(dst0 + p * kThreads * kSegBytes + 16 * q, reinterpret_cast<const uint8_t*>(g) + 16 * q, r < valid ? 16u : 0u);
+        }
       }
     }
     cp_async_commit();
-    f_tile += stride;
-    while (f_tile >= tiles && f_which < batch.count) {
-      f_tile -= tiles;
+    f_i += step_i;
+    f_bh += step_bh;
+    if (f_i >= nb) {
+      f_i -= nb;
+      ++f_bh;
+    }
+    while (f_bh >= bh_total && f_which < batch.count) {
+      f_bh -= bh_total;
       ++f_which;
     }
   };
